@@ -1,0 +1,163 @@
+/*
+ * meteora.h -- C ABI of the B200 (sm_100a) MeteoRA linear-layer forward.
+ *
+ * The layer (MeteoRA paper, Sec. 3.1, Eq. 2 and Eq. 3): every token x picks the k
+ * of N embedded LoRA adapters with the highest gate logits G(x) = Wg x, weighs them
+ * by a softmax over the k selected logits, and the output is
+ *
+ *     y = W0 x + sum_{i in topk(x)} w_i(x) * B_i (A_i x).
+ *
+ * Storage (all row-major, contiguous; the transposes of the paper's (n,d,r) and
+ * (n,r,h) adapter tensors of Sec. 3.3 so that every contraction runs along the
+ * contiguous axis):
+ *     x[T,d_in]  W0[d_out,d_in]  A[N,r,d_in]  B[N,d_out,r]  Wg[N,d_in]  y[T,d_out]
+ * in the element type named by meteora_shape_t::dtype (fp32, or bf16 with fp32
+ * accumulation and a single rounding of y).  No bias anywhere.  The LoRA scale
+ * alpha/r is folded into B by the caller (Eq. 1-2 carry no scale).
+ *
+ * Conventions for every entry point
+ *   - All tensor arguments are DEVICE pointers owned by the caller, 16-byte aligned,
+ *     unless an argument is explicitly marked "host".  The library allocates nothing,
+ *     keeps no pointer after a call returns, launches on `stream` (a cudaStream_t cast
+ *     to void*, NULL = default stream) and never synchronises, except where stated.
+ *   - Return value: METEORA_OK (0) or a negative meteora_status_t.  Arguments are
+ *     validated on the host before anything is launched; invalid arguments never reach
+ *     the device.  There is no CPU fallback and no other backend.
+ *   - Limits: 1 <= k <= METEORA_MAX_K, k <= N <= METEORA_MAX_N, 1 <= r <= METEORA_MAX_R,
+ *     T >= 0 (T == 0 is a no-op), T*k < 2^31, temperature > 0.
+ *   - Same inputs give bit-identical outputs from run to run (no floating-point atomics).
+ *   - Behaviour for NaN/Inf inputs is undefined but memory-safe (indices stay < N).
+ */
+#ifndef METEORA_H_
+#define METEORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define METEORA_MAX_N 64
+#define METEORA_MAX_K 8
+#define METEORA_MAX_R 64
+
+typedef enum { METEORA_F32 = 0, METEORA_BF16 = 1 } meteora_dtype_t;
+
+typedef enum {
+    METEORA_OK = 0,
+    METEORA_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, k > N, temperature <= 0 ... */
+    METEORA_ERR_UNSUPPORTED_SHAPE = -2,   /* a limit above is exceeded */
+    METEORA_ERR_MISALIGNED = -3,          /* a base pointer is not 16-byte aligned */
+    METEORA_ERR_WORKSPACE_TOO_SMALL = -4, /* workspace_bytes < meteora_workspace_bytes(shape) */
+    METEORA_ERR_CUDA = -5,                /* a CUDA runtime/driver call or a launch failed */
+    METEORA_ERR_TIMEOUT = -6              /* a bounded device-side wait expired (see meteora_workspace_status) */
+} meteora_status_t;
+
+typedef struct {
+    int T;               /* tokens (batch * sequence; tokens are independent, Sec. 3.3) */
+    int d_in;            /* input width  (paper: d) */
+    int d_out;           /* output width (paper: h) */
+    int N;               /* embedded adapters (paper: n) */
+    int r;               /* LoRA rank */
+    int k;               /* adapters selected per token */
+    meteora_dtype_t dtype;
+    float temperature;   /* divides the selected logits before the softmax (App. A.5); 1.0f = Eq. 3 as written */
+} meteora_shape_t;
+
+/*
+ * Gate, selection and weights (Sec. 3.1: G(x) = Wg x, the k highest logits form I(x);
+ * Eq. 3: softmax over the selected logits; App. A.1: k = 1 gives weight exactly 1).
+ *   x[T,d_in], Wg[N,d_in] in shape->dtype.  d_out and r of the shape are ignored.
+ *   topk_idx[T,k] int32: adapters by descending logit; equal logits keep the lower index first.
+ *   topk_w[T,k]   fp32 : the matching weights.
+ *   logits[T,N]   fp32 : optional (may be NULL).
+ * Logits are accumulated in fp32.
+ */
+int meteora_gate_topk(const void* x, const void* Wg, const meteora_shape_t* shape, int32_t* topk_idx,
+                      float* topk_w, float* logits, void* stream);
+
+/*
+ * Token -> adapter grouping (Sec. 3.3: the tokens that picked adapter i are gathered into one
+ * group per adapter).  Slot s = t*k + j has key topk_idx[s].
+ *   counts[N]    : slots per adapter.
+ *   offsets[N+1] : exclusive prefix sum of counts.
+ *   perm[T*k]    : slot numbers sorted by key, equal keys in ascending slot order (stable); the
+ *                  group of adapter e is perm[offsets[e] .. offsets[e+1]).
+ * Pure integer work; bit-exact.  Keys outside [0,N) are out of contract (clamped on the device).
+ */
+int meteora_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets,
+                  int32_t* perm, void* stream);
+
+/*
+ * The LoRA term of Eq. 2 alone, for a given routing:
+ *   delta[t,:] = sum_j topk_w[t,j] * B[topk_idx[t,j]] (A[topk_idx[t,j]] x[t]).
+ * The shrink (x A_i) runs adapter by adapter over the grouped slots (offsets, perm from
+ * meteora_route), the expand and weighted sum run token by token.
+ *   delta[T,d_out] fp32.  workspace: device scratch of at least meteora_workspace_bytes(shape).
+ */
+int meteora_lora_delta(const void* x, const void* A, const void* B, const int32_t* topk_idx,
+                       const float* topk_w, const int32_t* offsets, const int32_t* perm,
+                       const meteora_shape_t* shape, float* delta, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
+/*
+ * The whole layer, Eq. 2 with Eq. 3: gate, top-k, softmax over the selected, base product,
+ * gate-weighted LoRA sum, one rounding of y.
+ *   y[T,d_out] in shape->dtype.  workspace: device scratch of at least
+ *   meteora_workspace_bytes(shape); calls that share a workspace must not overlap in time.
+ * After the call the workspace holds the routing that was used (meteora_workspace_routing).
+ * bf16 shapes with d_in % 8 == 0 and r % 8 == 0 run on the tensor-core path (TMA + tcgen05);
+ * every other shape runs on a plain CUDA-core path with the same results up to rounding order.
+ */
+int meteora_linear_forward(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                           const meteora_shape_t* shape, void* y, void* workspace, size_t workspace_bytes,
+                           void* stream);
+
+/*
+ * Same as meteora_linear_forward with the activations in HOST memory: x_host[T,d_in] is copied to
+ * the device, the layer runs, y_host[T,d_out] is copied back, all on `stream` (pinned host memory
+ * makes the copies asynchronous).  Weights and workspace stay device pointers.  The call does not
+ * synchronise: y_host is valid once `stream` has been synchronised by the caller.
+ */
+int meteora_linear_forward_host(const void* x_host, const void* W0, const void* A, const void* B,
+                                const void* Wg, const meteora_shape_t* shape, void* y_host, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
+/* Upper bound of the scratch any of the calls above needs for this shape (0 on invalid shape). */
+size_t meteora_workspace_bytes(const meteora_shape_t* shape);
+
+/*
+ * Where meteora_linear_forward left its routing inside `workspace`: *topk_idx -> int32[T,k],
+ * *topk_w -> fp32[T,k] (device pointers into the workspace; valid until the workspace is reused).
+ */
+int meteora_workspace_routing(const meteora_shape_t* shape, void* workspace, int32_t** topk_idx, float** topk_w);
+
+/*
+ * Clears the status block at the head of a freshly allocated workspace (asynchronous, on `stream`).
+ * Call once before the workspace's first use; memory that is already zero needs no call.
+ */
+int meteora_workspace_init(void* workspace, void* stream);
+
+/*
+ * Reads the workspace's device status word (SYNCHRONISES `stream`): METEORA_OK, or
+ * METEORA_ERR_TIMEOUT if a bounded wait inside a kernel (an mbarrier of the TMA/tensor-core
+ * pipeline) gave up, in which case the outputs of that call are invalid.  The word is cleared.
+ */
+int meteora_workspace_status(void* workspace, void* stream);
+
+/*
+ * Tuning knobs for measurements (process-wide, not thread-safe): "splits" (split-K cluster size,
+ * 0 = automatic), "stages" (TMA ring depth, 0 = automatic), "tile_tokens" (tokens per tile, 0 =
+ * automatic), "force_simt" (1 = never take the tensor-core path), "pdl" (1 = overlap the chained
+ * kernels of a call by programmatic dependent launch).  Unknown names return
+ * METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
+ */
+int meteora_set_tuning(const char* name, int value);
+
+const char* meteora_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* METEORA_H_ */

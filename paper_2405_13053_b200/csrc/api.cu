@@ -1,0 +1,210 @@
+// C ABI of the library (declared in include/meteora.h): argument validation, workspace carve-up,
+// dispatch between the tensor-core path and the plain CUDA-core path.
+#include <string.h>
+
+#include "common.cuh"
+
+namespace meteora {
+
+Tuning& tuning() {
+    static Tuning t;
+    return t;
+}
+
+Workspace carve_workspace(const meteora_shape_t& s, void* base) {
+    Workspace ws;
+    uint8_t* p = (uint8_t*)base;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        uint8_t* q = p ? p + off : nullptr;
+        off += align_up(bytes, 256);
+        return q;
+    };
+    const size_t T = (size_t)s.T, es = elem_size(s.dtype);
+    int col_logits = 0;
+    ws.ld_u = tc_stacked_pitch(s, &col_logits);
+    ws.col_logits = col_logits;
+    ws.status = (int32_t*)take(64 * sizeof(int32_t));
+    ws.topk_idx = (int32_t*)take(T * s.k * sizeof(int32_t));
+    ws.topk_w = (float*)take(T * s.k * sizeof(float));
+    ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
+    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float));
+    ws.x_dev = take(T * s.d_in * es);
+    ws.y_dev = take(T * s.d_out * es);
+    ws.bytes = off;
+    return ws;
+}
+
+static int check_shape(const meteora_shape_t* s, bool need_out, bool need_r) {
+    if (!s) return METEORA_ERR_INVALID_ARG;
+    if (s->dtype != METEORA_F32 && s->dtype != METEORA_BF16) return METEORA_ERR_INVALID_ARG;
+    if (s->T < 0 || s->d_in <= 0 || s->N <= 0 || s->k <= 0 || s->k > s->N) return METEORA_ERR_INVALID_ARG;
+    if (!(s->temperature > 0.f)) return METEORA_ERR_INVALID_ARG;
+    if (need_out && s->d_out <= 0) return METEORA_ERR_INVALID_ARG;
+    if (need_r && s->r <= 0) return METEORA_ERR_INVALID_ARG;
+    if (s->N > METEORA_MAX_N || s->k > METEORA_MAX_K) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (need_r && s->r > METEORA_MAX_R) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if ((long long)s->T * s->k >= (1LL << 31)) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    return METEORA_OK;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+static int forward_device(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                          const meteora_shape_t& s, void* y, const Workspace& ws, cudaStream_t st) {
+    int rc;
+    if (tc_path_supported(s)) {
+        const bool pdl = tuning().pdl != 0;
+        if ((rc = launch_stacked_shrink_tc(x, A, Wg, s, ws, st)) != METEORA_OK) return rc;
+        if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, s, ws.topk_idx, ws.topk_w, ws.uw, pdl,
+                                             st)) != METEORA_OK)
+            return rc;
+        return launch_base_lora_tc(x, W0, B, s, ws, y, pdl, st);
+    }
+    if ((rc = launch_gate_topk(x, Wg, s, ws.topk_idx, ws.topk_w, nullptr, st)) != METEORA_OK) return rc;
+    if ((rc = launch_shrink_tokens(x, A, ws.topk_idx, ws.topk_w, s, ws.uw, st)) != METEORA_OK) return rc;
+    return launch_gemm_simt(x, W0, B, ws.topk_idx, ws.uw, s, y, st);
+}
+
+}  // namespace meteora
+
+using namespace meteora;
+
+extern "C" {
+
+int meteora_gate_topk(const void* x, const void* Wg, const meteora_shape_t* shape, int32_t* topk_idx,
+                      float* topk_w, float* logits, void* stream) {
+    int rc = check_shape(shape, false, false);
+    if (rc != METEORA_OK) return rc;
+    if (shape->T == 0) return METEORA_OK;
+    if (!x || !Wg || !topk_idx || !topk_w) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(Wg)) return METEORA_ERR_MISALIGNED;
+    return launch_gate_topk(x, Wg, *shape, topk_idx, topk_w, logits, (cudaStream_t)stream);
+}
+
+int meteora_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets,
+                  int32_t* perm, void* stream) {
+    if (T < 0 || k <= 0 || N <= 0 || k > N) return METEORA_ERR_INVALID_ARG;
+    if (N > METEORA_MAX_N || k > METEORA_MAX_K || (long long)T * k >= (1LL << 31))
+        return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (!counts || !offsets || (T > 0 && (!topk_idx || !perm))) return METEORA_ERR_INVALID_ARG;
+    return launch_route(topk_idx, T, k, N, counts, offsets, perm, (cudaStream_t)stream);
+}
+
+int meteora_lora_delta(const void* x, const void* A, const void* B, const int32_t* topk_idx,
+                       const float* topk_w, const int32_t* offsets, const int32_t* perm,
+                       const meteora_shape_t* shape, float* delta, void* workspace, size_t workspace_bytes,
+                       void* stream) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (shape->T == 0) return METEORA_OK;
+    if (!x || !A || !B || !topk_idx || !topk_w || !offsets || !perm || !delta || !workspace)
+        return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(A) || !aligned16(B) || !aligned16(delta) || !aligned16(workspace))
+        return METEORA_ERR_MISALIGNED;
+    const Workspace ws = carve_workspace(*shape, workspace);
+    if (workspace_bytes < ws.bytes) return METEORA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = launch_shrink_segments(x, A, offsets, perm, *shape, ws.uw, st)) != METEORA_OK) return rc;
+    return launch_expand(B, topk_idx, topk_w, ws.uw, *shape, delta, st);
+}
+
+int meteora_linear_forward(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                           const meteora_shape_t* shape, void* y, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (shape->T == 0) return METEORA_OK;
+    if (!x || !W0 || !A || !B || !Wg || !y || !workspace) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(Wg) || !aligned16(y) ||
+        !aligned16(workspace))
+        return METEORA_ERR_MISALIGNED;
+    const Workspace ws = carve_workspace(*shape, workspace);
+    if (workspace_bytes < ws.bytes) return METEORA_ERR_WORKSPACE_TOO_SMALL;
+    return forward_device(x, W0, A, B, Wg, *shape, y, ws, (cudaStream_t)stream);
+}
+
+int meteora_linear_forward_host(const void* x_host, const void* W0, const void* A, const void* B,
+                                const void* Wg, const meteora_shape_t* shape, void* y_host, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (shape->T == 0) return METEORA_OK;
+    if (!x_host || !W0 || !A || !B || !Wg || !y_host || !workspace) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(W0) || !aligned16(A) || !aligned16(B) || !aligned16(Wg) || !aligned16(workspace))
+        return METEORA_ERR_MISALIGNED;
+    const Workspace ws = carve_workspace(*shape, workspace);
+    if (workspace_bytes < ws.bytes) return METEORA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = elem_size(shape->dtype);
+    if (cudaMemcpyAsync(ws.x_dev, x_host, (size_t)shape->T * shape->d_in * es, cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return METEORA_ERR_CUDA;
+    if ((rc = forward_device(ws.x_dev, W0, A, B, Wg, *shape, ws.y_dev, ws, st)) != METEORA_OK) return rc;
+    if (cudaMemcpyAsync(y_host, ws.y_dev, (size_t)shape->T * shape->d_out * es, cudaMemcpyDeviceToHost, st) !=
+        cudaSuccess)
+        return METEORA_ERR_CUDA;
+    return METEORA_OK;
+}
+
+size_t meteora_workspace_bytes(const meteora_shape_t* shape) {
+    if (check_shape(shape, true, true) != METEORA_OK) return 0;
+    return carve_workspace(*shape, nullptr).bytes;
+}
+
+int meteora_workspace_routing(const meteora_shape_t* shape, void* workspace, int32_t** topk_idx, float** topk_w) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (!workspace || !topk_idx || !topk_w) return METEORA_ERR_INVALID_ARG;
+    const Workspace ws = carve_workspace(*shape, workspace);
+    *topk_idx = ws.topk_idx;
+    *topk_w = ws.topk_w;
+    return METEORA_OK;
+}
+
+int meteora_workspace_init(void* workspace, void* stream) {
+    if (!workspace) return METEORA_ERR_INVALID_ARG;
+    return cuda_status(cudaMemsetAsync(workspace, 0, 64 * sizeof(int32_t), (cudaStream_t)stream));
+}
+
+int meteora_workspace_status(void* workspace, void* stream) {
+    if (!workspace) return METEORA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return METEORA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return METEORA_ERR_CUDA;
+    if (word != 0) {
+        if (cudaMemsetAsync(workspace, 0, 64 * sizeof(int32_t), st) != cudaSuccess) return METEORA_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return METEORA_ERR_CUDA;
+        return METEORA_ERR_TIMEOUT;
+    }
+    return METEORA_OK;
+}
+
+int meteora_set_tuning(const char* name, int value) {
+    if (!name) return METEORA_ERR_INVALID_ARG;
+    Tuning& t = tuning();
+    if (!strcmp(name, "splits")) t.splits = value;
+    else if (!strcmp(name, "stages")) t.stages = value;
+    else if (!strcmp(name, "tile_tokens")) t.tile_tokens = value;
+    else if (!strcmp(name, "force_simt")) t.force_simt = value;
+    else if (!strcmp(name, "pdl")) t.pdl = value;
+    else return METEORA_ERR_INVALID_ARG;
+    return METEORA_OK;
+}
+
+const char* meteora_status_string(int status) {
+    switch (status) {
+        case METEORA_OK: return "ok";
+        case METEORA_ERR_INVALID_ARG: return "invalid argument";
+        case METEORA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case METEORA_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+        case METEORA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case METEORA_ERR_CUDA: return "CUDA error";
+        case METEORA_ERR_TIMEOUT: return "bounded device wait expired";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

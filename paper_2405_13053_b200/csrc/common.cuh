@@ -1,0 +1,123 @@
+// Shared declarations of the MeteoRA CUDA library (internal; the public C ABI is include/meteora.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "meteora.h"
+
+namespace meteora {
+
+// ---------------------------------------------------------------------------------------------
+// Workspace layout.  Every region starts on a 256-byte boundary.
+// ---------------------------------------------------------------------------------------------
+struct Workspace {
+    int32_t* status;    // [64]  word 0: error flag of bounded device waits; words 1..: where it gave up
+    int32_t* topk_idx;  // [T,k]
+    float* topk_w;      // [T,k]
+    float* uw;          // [T,k,r]   w_j * (A_{i_j} x): the shrunk, gate-weighted activations
+    float* u_all;       // [T,ld_u]  stacked shrink: every adapter's A_i x, then the gate logits
+    int ld_u;           // row pitch of u_all in floats
+    int col_logits;     // first logit column inside a u_all row
+    void* x_dev;        // [T,d_in]  staging for the host-buffer entry point
+    void* y_dev;        // [T,d_out]
+    size_t bytes;       // total
+};
+
+Workspace carve_workspace(const meteora_shape_t& s, void* base);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline size_t elem_size(meteora_dtype_t t) { return t == METEORA_BF16 ? 2 : 4; }
+
+// ---------------------------------------------------------------------------------------------
+// Kernel launchers (each returns a meteora_status_t).  All pointers are device pointers.
+// ---------------------------------------------------------------------------------------------
+// gate_topk.cu
+int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, int32_t* topk_idx, float* topk_w,
+                     float* logits, cudaStream_t st);
+int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, const meteora_shape_t& s,
+                               int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st);
+// route.cu
+int launch_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets, int32_t* perm,
+                 cudaStream_t st);
+// lora.cu
+int launch_shrink_segments(const void* x, const void* A, const int32_t* offsets, const int32_t* perm,
+                           const meteora_shape_t& s, float* u, cudaStream_t st);
+int launch_shrink_tokens(const void* x, const void* A, const int32_t* topk_idx, const float* topk_w,
+                         const meteora_shape_t& s, float* uw, cudaStream_t st);
+int launch_expand(const void* B, const int32_t* topk_idx, const float* topk_w, const float* u,
+                  const meteora_shape_t& s, float* delta, cudaStream_t st);
+// gemm_simt.cu
+int launch_gemm_simt(const void* x, const void* W0, const void* B, const int32_t* topk_idx, const float* uw,
+                     const meteora_shape_t& s, void* y, cudaStream_t st);
+// wgemm_tcgen05.cu
+bool tc_path_supported(const meteora_shape_t& s);
+int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits);  // row pitch (floats) of u_all
+int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const meteora_shape_t& s,
+                             const Workspace& ws, cudaStream_t st);
+int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
+                        void* y, bool pdl, cudaStream_t st);
+
+struct Tuning {
+    int splits = 0;
+    int stages = 0;
+    int tile_tokens = 0;
+    int force_simt = 0;
+    int pdl = 1;
+};
+Tuning& tuning();
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// 8 consecutive elements as fp32, from a 16-byte aligned address.
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 q = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 b = *reinterpret_cast<const float4*>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Dot product of two length-n vectors, spread over a warp; every lane returns the sum.
+// vec: n % 8 == 0 and both rows 16-byte aligned (128-bit loads); otherwise element by element.
+template <typename TI>
+__device__ __forceinline__ float warp_dot(const TI* __restrict__ a, const TI* __restrict__ b, int n, int lane,
+                                          bool vec) {
+    float acc = 0.f;
+    if (vec) {
+        for (int d = lane * 8; d < n; d += 256) {
+            float xa[8], xb[8];
+            load8(a + d, xa);
+            load8(b + d, xb);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc = fmaf(xa[i], xb[i], acc);
+        }
+    } else {
+        for (int d = lane; d < n; d += 32) acc = fmaf(to_f32(a[d]), to_f32(b[d]), acc);
+    }
+    return warp_sum(acc);
+}
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? METEORA_OK : METEORA_ERR_CUDA; }
+inline int last_launch_status() { return cuda_status(cudaGetLastError()); }
+
+}  // namespace meteora

@@ -1,0 +1,141 @@
+// Gate logits, top-k selection and softmax over the selected logits (Sec. 3.1, Eq. 3; temperature App. A.5).
+//
+// One warp owns one token.  Lane n (and lane n-32 for n >= 32) holds logit n; the k picks are
+// taken by k rounds of a warp-wide arg-max whose ordering is (logit descending, index ascending),
+// so equal logits always resolve to the lower adapter index.
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace meteora {
+
+constexpr int kGateWarps = 8;
+
+// v0 = logit[lane], v1 = logit[lane + 32]; entries at or beyond N are ignored.
+// On return lane j < k holds pick j (index and softmax weight).  Every lane runs the same code.
+__device__ __forceinline__ void warp_topk_softmax(float v0, float v1, int N, int k, float inv_tau, int lane,
+                                                  int& my_idx, float& my_w) {
+    bool taken0 = lane >= N, taken1 = lane + 32 >= N;
+    if (!(v0 > -CUDART_INF_F)) v0 = -CUDART_INF_F;  // NaN never wins a comparison; treat it as -inf
+    if (!(v1 > -CUDART_INF_F)) v1 = -CUDART_INF_F;
+    float first = 0.f, sum = 0.f, my_e = 0.f;
+    my_idx = 0;
+    for (int j = 0; j < k; ++j) {
+        float bv = -CUDART_INF_F;
+        int bi = 0x7FFFFFFF;
+        if (!taken0) { bv = v0; bi = lane; }
+        if (!taken1 && (bi == 0x7FFFFFFF || v1 > bv)) { bv = v1; bi = lane + 32; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        bi = min(bi, N - 1);
+        if (bi == lane) taken0 = true;
+        if (bi == lane + 32) taken1 = true;
+        if (j == 0) first = bv;
+        const float e = expf((bv - first) * inv_tau);
+        sum += e;
+        if (lane == j) { my_idx = bi; my_e = e; }
+    }
+    my_w = my_e / sum;
+}
+
+template <typename TI>
+__global__ void __launch_bounds__(kGateWarps * 32)
+k_gate_topk(const TI* __restrict__ x, const TI* __restrict__ Wg, int T, int d_in, int N, int k, float inv_tau,
+            int32_t* __restrict__ topk_idx, float* __restrict__ topk_w, float* __restrict__ logits) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * kGateWarps + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const bool vec = (d_in % 8) == 0;
+    const TI* xt = x + (size_t)t * d_in;
+    float v0 = 0.f, v1 = 0.f;
+    for (int n = 0; n < N; ++n) {
+        const float l = warp_dot(xt, Wg + (size_t)n * d_in, d_in, lane, vec);
+        if (n == lane) v0 = l;
+        if (n == lane + 32) v1 = l;
+    }
+    if (logits) {
+        if (lane < N) logits[(size_t)t * N + lane] = v0;
+        if (lane + 32 < N) logits[(size_t)t * N + lane + 32] = v1;
+    }
+    int idx;
+    float w;
+    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    if (lane < k) {
+        topk_idx[(size_t)t * k + lane] = idx;
+        topk_w[(size_t)t * k + lane] = w;
+    }
+}
+
+// Selection from the stacked shrink: row t of u_all holds A_i x for every adapter (N*r values)
+// and, from column col_logits on, the N gate logits.  Besides the picks and weights this writes
+// uw[t,j,:] = w_j * (A_{i_j} x), the activations the base product's epilogue expands.
+__global__ void __launch_bounds__(kGateWarps * 32)
+k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits, int T, int N, int r, int k,
+                      float inv_tau, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
+                      float* __restrict__ uw, int pdl) {
+    if (pdl) {
+        // Let the dependent launch (the base product) start streaming weights now; wait for the
+        // stacked shrink, which produced u_all, before reading it.
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * kGateWarps + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const float* row = u_all + (size_t)t * ld_u;
+    const float v0 = lane < N ? row[col_logits + lane] : 0.f;
+    const float v1 = lane + 32 < N ? row[col_logits + lane + 32] : 0.f;
+    int idx;
+    float w;
+    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    if (lane < k) {
+        topk_idx[(size_t)t * k + lane] = idx;
+        topk_w[(size_t)t * k + lane] = w;
+    }
+    for (int c0 = 0; c0 < k * r; c0 += 32) {
+        const int c = c0 + lane;
+        const int j = min(c / r, k - 1), p = c - j * r;
+        const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
+        const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
+        if (c < k * r) uw[(size_t)t * k * r + c] = wj * row[ij * r + p];
+    }
+}
+
+int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, int32_t* topk_idx, float* topk_w,
+                     float* logits, cudaStream_t st) {
+    if (s.T == 0) return METEORA_OK;
+    const int blocks = (s.T + kGateWarps - 1) / kGateWarps;
+    const float inv_tau = 1.0f / s.temperature;
+    if (s.dtype == METEORA_BF16)
+        k_gate_topk<__nv_bfloat16><<<blocks, kGateWarps * 32, 0, st>>>(
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)Wg, s.T, s.d_in, s.N, s.k, inv_tau, topk_idx, topk_w, logits);
+    else
+        k_gate_topk<float><<<blocks, kGateWarps * 32, 0, st>>>((const float*)x, (const float*)Wg, s.T, s.d_in, s.N,
+                                                               s.k, inv_tau, topk_idx, topk_w, logits);
+    return last_launch_status();
+}
+
+int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, const meteora_shape_t& s,
+                               int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st) {
+    if (s.T == 0) return METEORA_OK;
+    const int blocks = (s.T + kGateWarps - 1) / kGateWarps;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(kGateWarps * 32);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    const float inv_tau = 1.0f / s.temperature;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_select_from_stacked, u_all, ld_u, col_logits, s.T, s.N, s.r, s.k,
+                                       inv_tau, topk_idx, topk_w, uw, pdl ? 1 : 0);
+    return cuda_status(e);
+}
+
+}  // namespace meteora
