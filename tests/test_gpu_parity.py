@@ -1,0 +1,301 @@
+"""GPU parity: every entry point of the C ABI against the CPU oracle, element by element, on the same
+seeded inputs.  Tolerances (stated where used):
+  - indices, counts, offsets, perm: bit-exact (selections only where the logit gap exceeds 1e-3);
+  - fp32 layers: relative L2 <= 1e-4 (measured ~1e-6);
+  - bf16 layers: y relative L2 <= 1e-2 and max-abs <= 5e-2; fp32 intermediates (weights, delta) <= 1e-4,
+    since both sides read the same bf16 values and the GPU accumulates in fp32.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2405_13053_b200 import binding as mb
+from paper_2405_13053_b200 import workloads
+
+from .gpu_util import check_selection, max_abs, rel_l2, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def wl(T, d_in, d_out, N=5, r=8, k=2, dtype="bf16", seed=1, b_std=0.3, x_kind="normal", temperature=1.0):
+    return workloads.make_workload("t", T=T, d_in=d_in, d_out=d_out, N=N, r=r, k=k, dtype=dtype, x_kind=x_kind,
+                                   seed=seed, b_std=b_std, temperature=temperature)
+
+
+# ----------------------------------------------------------------------------------------- gate + top-k
+GATE_CASES = [
+    dict(T=64, d_in=256, d_out=8, N=4, k=2, dtype="f32"),
+    dict(T=37, d_in=136, d_out=8, N=28, k=2, dtype="bf16"),
+    dict(T=5, d_in=23, d_out=8, N=7, k=3, dtype="f32"),          # d_in not a multiple of 8: scalar loads
+    dict(T=19, d_in=72, d_out=8, N=40, k=8, dtype="bf16"),       # more than 32 adapters, k = 8
+    dict(T=9, d_in=64, d_out=8, N=64, k=1, dtype="f32"),         # top-1
+    dict(T=11, d_in=48, d_out=8, N=6, k=6, dtype="bf16"),        # k = N
+    dict(T=1, d_in=4096, d_out=8, N=28, k=2, dtype="bf16"),
+    dict(T=300, d_in=512, d_out=8, N=28, k=2, dtype="bf16", temperature=15.0),
+]
+
+
+@pytest.mark.parametrize("case", GATE_CASES, ids=lambda c: f"T{c['T']}d{c['d_in']}N{c['N']}k{c['k']}{c['dtype']}")
+def test_gate_topk_matches_oracle(case):
+    w = wl(**case)
+    x, Wg = to_dev(w, "x", "Wg")
+    idx, wts, logits = mb.meteora_gate_topk(x, Wg, w.k, w.temperature, want_logits=True)
+    torch.cuda.synchronize()
+    o_idx, o_w, o_logits = oracle.gate_topk(w["x"], w["Wg"], w.k, w.temperature)
+    np.testing.assert_allclose(logits.cpu().numpy(), o_logits, rtol=1e-4, atol=1e-5)
+    clear = check_selection(idx.cpu().numpy(), o_idx, o_logits, w.k)
+    assert clear.mean() > 0.9
+    g_w = wts.cpu().numpy()
+    np.testing.assert_allclose(g_w[clear], o_w[clear], rtol=1e-4, atol=1e-6)
+    np.testing.assert_allclose(g_w.sum(axis=1), 1.0, atol=1e-6)      # Eq. 3: weights sum to one
+    if w.k == 1:
+        assert np.all(g_w == 1.0)
+
+
+def test_gate_ties_resolve_to_lower_index():
+    w = wl(T=33, d_in=64, d_out=8, N=40, k=3, dtype="f32")
+    Wg = np.zeros_like(w["Wg"])
+    Wg[[3, 17, 35, 38], 0] = 7.0                                     # four exactly equal logits
+    x = w["x"].copy()
+    x[:, 0] = 1.0
+    idx, wts, _ = mb.meteora_gate_topk(torch.from_numpy(x).cuda(), torch.from_numpy(Wg).cuda(), 3)
+    o_idx, o_w, _ = oracle.gate_topk(x, Wg, 3)
+    np.testing.assert_array_equal(idx.cpu().numpy(), o_idx)
+    np.testing.assert_array_equal(o_idx[0], [3, 17, 35])
+    np.testing.assert_allclose(wts.cpu().numpy(), o_w, rtol=1e-6)
+
+
+# ----------------------------------------------------------------------------------------- routing
+def random_idx(T, k, N, seed, skew=False):
+    rng = np.random.default_rng(seed)
+    idx = np.stack([rng.permutation(N)[:k] for _ in range(T)]).astype(np.int32) if T else np.zeros((0, k), np.int32)
+    if skew and T > 4:
+        hot = rng.permutation(N)[:max(k, 3)]
+        idx[: 3 * T // 4] = np.stack([rng.permutation(hot)[:k] for _ in range(3 * T // 4)])
+    return idx
+
+
+@pytest.mark.parametrize("T,k,N,skew", [(0, 2, 4, False), (1, 1, 1, False), (1, 2, 28, False), (64, 2, 4, False),
+                                         (511, 2, 28, True), (512, 2, 28, True), (513, 2, 28, False),
+                                         (1500, 3, 64, True), (8192, 2, 28, True), (100, 8, 8, False)])
+def test_route_is_bit_exact(T, k, N, skew):
+    idx = random_idx(T, k, N, seed=T + k + N, skew=skew)
+    counts, offsets, perm = mb.meteora_route(torch.from_numpy(idx).cuda(), N)
+    torch.cuda.synchronize()
+    o_counts, o_offsets, o_perm = oracle.route(idx, N)
+    np.testing.assert_array_equal(counts.cpu().numpy(), o_counts)
+    np.testing.assert_array_equal(offsets.cpu().numpy(), o_offsets)
+    np.testing.assert_array_equal(perm.cpu().numpy(), o_perm)
+
+
+def test_route_all_tokens_to_one_adapter():
+    idx = np.tile(np.array([[5, 2]], np.int32), (2000, 1))
+    counts, offsets, perm = mb.meteora_route(torch.from_numpy(idx).cuda(), 28)
+    o = oracle.route(idx, 28)
+    for g, e in zip((counts, offsets, perm), o):
+        np.testing.assert_array_equal(g.cpu().numpy(), e)
+
+
+# ----------------------------------------------------------------------------------------- LoRA term
+DELTA_CASES = [
+    dict(T=64, d_in=256, d_out=256, N=4, r=8, k=2, dtype="f32"),
+    dict(T=77, d_in=136, d_out=200, N=28, r=8, k=2, dtype="bf16"),
+    dict(T=13, d_in=23, d_out=19, N=5, r=3, k=2, dtype="f32"),       # nothing aligned: scalar paths
+    dict(T=40, d_in=4096, d_out=320, N=28, r=16, k=2, dtype="bf16"),  # rank 16, several shared-memory chunks
+    dict(T=9, d_in=2304, d_out=64, N=6, r=12, k=3, dtype="f32"),      # rank not a multiple of 8
+    dict(T=300, d_in=512, d_out=96, N=28, r=8, k=1, dtype="bf16", x_kind="clusters"),
+]
+
+
+@pytest.mark.parametrize("case", DELTA_CASES, ids=lambda c: f"T{c['T']}d{c['d_in']}o{c['d_out']}r{c['r']}{c['dtype']}")
+def test_lora_delta_matches_oracle(case):
+    w = wl(**case)
+    o_idx, o_w, _ = oracle.gate_topk(w["x"], w["Wg"], w.k)
+    w32 = o_w.astype(np.float32)
+    x, A, B = to_dev(w, "x", "A", "B")
+    idx = torch.from_numpy(o_idx).cuda()
+    wts = torch.from_numpy(w32).cuda()
+    _, offsets, perm = mb.meteora_route(idx, w.N)
+    delta = mb.meteora_lora_delta(x, A, B, idx, wts, offsets, perm)
+    torch.cuda.synchronize()
+    ref = oracle.lora_delta(w["x"], w["A"], w["B"], o_idx, w32)
+    assert rel_l2(delta.cpu().numpy(), ref) <= 1e-4                  # fp32 accumulate on identical inputs
+    assert np.linalg.norm(ref) > 0
+
+
+def test_lora_delta_with_empty_adapters_and_single_hot_adapter():
+    w = wl(T=50, d_in=128, d_out=72, N=28, r=8, k=2, dtype="bf16")
+    o_idx = np.tile(np.array([[9, 27]], np.int32), (50, 1))          # 26 adapters receive no token
+    w32 = np.tile(np.array([[0.75, 0.25]], np.float32), (50, 1))
+    x, A, B = to_dev(w, "x", "A", "B")
+    idx = torch.from_numpy(o_idx).cuda()
+    _, offsets, perm = mb.meteora_route(idx, w.N)
+    delta = mb.meteora_lora_delta(x, A, B, idx, torch.from_numpy(w32).cuda(), offsets, perm)
+    ref = oracle.lora_delta(w["x"], w["A"], w["B"], o_idx, w32)
+    assert rel_l2(delta.cpu().numpy(), ref) <= 1e-4
+
+
+# ----------------------------------------------------------------------------------------- whole layer
+def run_forward(w, **kw):
+    x, W0, A, B, Wg = to_dev(w, "x", "W0", "A", "B", "Wg")
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, x.dtype, w.temperature)
+    ws = mb.alloc_workspace(shape)
+    y, idx, wts = mb.meteora_linear_forward(x, W0, A, B, Wg, w.k, w.temperature, workspace=ws, return_routing=True)
+    assert mb.meteora_workspace_status(ws) == 0
+    return y.float().cpu().numpy(), idx.cpu().numpy().copy(), wts.cpu().numpy().copy()
+
+
+def check_forward(w, y_tol, abs_tol=None, tokens=None):
+    """Compare the fused forward with the oracle; `tokens` restricts the y comparison to sampled rows."""
+    y, idx, wts = run_forward(w)
+    o_idx, o_w, o_logits = oracle.gate_topk(w["x"], w["Wg"], w.k, w.temperature)
+    clear = check_selection(idx, o_idx, o_logits, w.k)
+    np.testing.assert_allclose(wts[clear], o_w[clear], rtol=2e-3, atol=1e-5)
+    sel = np.arange(w.T) if tokens is None else np.asarray(tokens)
+    ref = oracle.linear_forward_routed(w["x"][sel], w["W0"], w["A"], w["B"], w["Wg"], idx[sel], w.temperature)
+    err = rel_l2(y[sel], ref)
+    assert err <= y_tol, err
+    if abs_tol is not None:
+        assert max_abs(y[sel], ref) <= abs_tol
+    return y, idx, err
+
+
+def test_config0_fp32():
+    w = workloads.config0()
+    _, _, err = check_forward(w, y_tol=1e-4)
+    assert err < 1e-5
+
+
+FORWARD_CASES = [
+    dict(T=13, d_in=24, d_out=20, N=5, r=3, k=2, dtype="f32"),                    # plain path, nothing aligned
+    dict(T=70, d_in=100, d_out=130, N=28, r=8, k=2, dtype="f32"),
+    dict(T=33, d_in=60, d_out=50, N=6, r=4, k=2, dtype="bf16"),                   # bf16 on the plain path (r % 8 != 0)
+    dict(T=37, d_in=136, d_out=200, N=28, r=8, k=2, dtype="bf16"),                # tensor-core path, ragged everywhere
+    dict(T=1, d_in=512, d_out=384, N=28, r=8, k=2, dtype="bf16"),
+    dict(T=129, d_in=1024, d_out=256, N=28, r=8, k=2, dtype="bf16"),
+    dict(T=300, d_in=2048, d_out=640, N=28, r=8, k=2, dtype="bf16"),              # two token tiles, ragged tail
+    dict(T=50, d_in=512, d_out=128, N=40, r=16, k=3, dtype="bf16"),               # 40 adapters, rank 16, top-3
+    dict(T=20, d_in=256, d_out=128, N=8, r=8, k=1, dtype="bf16"),                 # top-1
+    dict(T=24, d_in=256, d_out=136, N=4, r=8, k=4, dtype="bf16", temperature=20.0),  # k = N with temperature
+]
+
+
+@pytest.mark.parametrize("case", FORWARD_CASES,
+                         ids=lambda c: f"T{c['T']}d{c['d_in']}o{c['d_out']}N{c['N']}r{c['r']}k{c['k']}{c['dtype']}")
+def test_forward_small_shapes(case):
+    w = wl(**case)                                                   # B ~ N(0, 0.3): the LoRA term is as large as the base
+    if w.dtype == "f32":
+        check_forward(w, y_tol=1e-4)
+    else:
+        check_forward(w, y_tol=1e-2, abs_tol=5e-2 * max(1.0, float(np.abs(w["x"]).max())))
+
+
+@pytest.mark.parametrize("T", workloads.CONFIG1_T)
+def test_config1_decode_shapes(T):
+    w = workloads.config1(T)
+    y, idx, err = check_forward(w, y_tol=1e-2, abs_tol=5e-2)
+    assert err < 5e-3                                                # one bf16 rounding of y: ~2^-9 per element
+
+
+def test_zero_B_is_exactly_the_base_product_and_delta_is_visible():
+    w = wl(T=96, d_in=1024, d_out=384, N=28, r=8, k=2, dtype="bf16", b_std=0.3)
+    y, idx, _ = run_forward(w)
+    w0 = wl(T=96, d_in=1024, d_out=384, N=28, r=8, k=2, dtype="bf16", b_std=0.3)
+    w0.tensors["B"] = np.zeros_like(w["B"])
+    y0, _, _ = run_forward(w0)
+    base = w["x"].astype(np.float64) @ w["W0"].astype(np.float64).T
+    assert rel_l2(y0, base) < 5e-3                                   # Eq. 2 with B = 0
+    o_idx, o_w, _ = oracle.gate_topk(w["x"], w["Wg"], w.k)
+    ref_delta = oracle.lora_delta(w["x"], w["A"], w["B"], idx, o_w.astype(np.float32))
+    assert np.linalg.norm(ref_delta) > 0.3 * np.linalg.norm(base)    # the LoRA term is not hidden under the base
+    assert rel_l2(y - y0, ref_delta) <= 1e-2
+
+
+def test_forward_is_deterministic():
+    w = workloads.config1(32)
+    y1, i1, w1 = run_forward(w)
+    y2, i2, w2 = run_forward(w)
+    np.testing.assert_array_equal(y1, y2)
+    np.testing.assert_array_equal(i1, i2)
+    np.testing.assert_array_equal(w1, w2)
+
+
+def test_tensor_core_and_plain_paths_agree():
+    w = wl(T=45, d_in=512, d_out=264, N=28, r=8, k=2, dtype="bf16")
+    y_tc, i_tc, _ = run_forward(w)
+    mb.meteora_set_tuning("force_simt", 1)
+    try:
+        y_simt, i_simt, _ = run_forward(w)
+    finally:
+        mb.meteora_set_tuning("force_simt", 0)
+    same = np.all(i_tc == i_simt, axis=1)
+    assert same.mean() > 0.95
+    assert rel_l2(y_tc[same], y_simt[same]) < 5e-3
+
+
+@pytest.mark.parametrize("splits,stages", [(1, 2), (2, 3), (3, 4), (8, 2)])
+def test_split_k_cluster_sizes_agree_with_oracle(splits, stages):
+    w = wl(T=40, d_in=1536, d_out=200, N=28, r=8, k=2, dtype="bf16")
+    mb.meteora_set_tuning("splits", splits)
+    mb.meteora_set_tuning("stages", stages)
+    try:
+        check_forward(w, y_tol=1e-2)
+    finally:
+        mb.meteora_set_tuning("splits", 0)
+        mb.meteora_set_tuning("stages", 0)
+
+
+def test_host_buffer_entry_point():
+    w = workloads.config1(8)
+    _, W0, A, B, Wg = to_dev(w, "x", "W0", "A", "B", "Wg")
+    x_host = torch.from_numpy(w["x"]).to(torch.bfloat16).pin_memory()
+    y_host = torch.empty((w.T, w.d_out), dtype=torch.bfloat16).pin_memory()
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    ws = mb.alloc_workspace(shape)
+    mb.meteora_linear_forward_host(x_host, W0, A, B, Wg, w.k, y_host, ws)
+    assert mb.meteora_workspace_status(ws) == 0                      # synchronises
+    y_dev, _, _ = run_forward(w)
+    np.testing.assert_array_equal(y_host.float().numpy(), y_dev)
+
+
+# ----------------------------------------------------------------------------------------- full-size shapes
+@pytest.mark.parametrize("shape,T", [("gate_up", 512), ("down", 2048), ("kv", 8192)])
+def test_config2_prefill_sampled_rows(shape, T):
+    w = workloads.config2(shape, T)
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, 22)]))
+    check_forward(w, y_tol=1e-2, abs_tol=5e-2 * 8, tokens=rows)       # |x| reaches ~4 here, y ~ 4x larger than config 1
+
+
+@pytest.mark.parametrize("shape,T", [("qkvo", 64), ("gate_up", 1), ("down", 64)])
+def test_config3_sampled_rows(shape, T):
+    w = workloads.config3(shape, T)
+    rows = np.unique(np.concatenate([[0, T - 1], np.random.default_rng(6).integers(0, T, 14)]))
+    check_forward(w, y_tol=1e-2, abs_tol=5e-2 * 8, tokens=rows)
+
+
+# ----------------------------------------------------------------------------------------- error behaviour
+def test_errors_are_reported_not_launched():
+    w = workloads.config0()
+    x, W0, A, B, Wg = to_dev(w, "x", "W0", "A", "B", "Wg")
+    small = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(mb.MeteoraError) as e:
+        mb.meteora_linear_forward(x, W0, A, B, Wg, 2, workspace=small)
+    assert e.value.status == -4
+    with pytest.raises(mb.MeteoraError) as e:
+        mb.meteora_gate_topk(x, Wg, 5)
+    assert e.value.status == -1
+    with pytest.raises(mb.MeteoraError) as e:
+        mb.meteora_linear_forward(x, W0, A, B, Wg, 2, temperature=0.0)
+    assert e.value.status == -1
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.float32)
+    ws = mb.alloc_workspace(shape)
+    lib = mb.load_library()
+    import ctypes
+    rc = lib.meteora_linear_forward(x.data_ptr() + 4, W0.data_ptr(), A.data_ptr(), B.data_ptr(), Wg.data_ptr(),
+                                    ctypes.byref(shape), torch.empty_like(x).data_ptr(), ws.data_ptr(), ws.numel(),
+                                    None)
+    assert rc == -3
+    y = mb.meteora_linear_forward(x[:0].contiguous(), W0, A, B, Wg, 2)   # T = 0 is a no-op
+    assert y.shape == (0, w.d_out)
