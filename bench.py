@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the MeteoRA linear forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--tokens T]
+
+Workload (N = 1 and every rank of N > 1): the LLaMA3-8B q_proj-shaped MeteoRA linear, d_in = d_out = 4096,
+28 adapters of rank 8, top-2, bf16 with fp32 accumulation, a decode batch of T = 128 tokens.  One STEP is one
+pass of the whole layer (gate, top-k, softmax, shrink, base product, expand, store) over `--modules` = 16
+independent MeteoRA modules (own weights, own gate, own tokens), the way consecutive projections of a decoder
+are visited during decoding; their weights total ~0.6 GB, far beyond the 126 MB L2, so every step streams its
+weights from HBM.  value = (modules x T x K x ranks) tokens through a MeteoRA linear per second.
+
+The step is captured once into a CUDA graph (the library's launches are capturable: no allocation, no
+synchronisation) and replayed K times; `--launch stream` issues the same calls directly instead.
+One JSON line is printed by rank 0.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "MeteoRA-linear tokens/s at LLaMA3-8B shapes (N=28, r=8, k=2)"
+D_IN = D_OUT = 4096
+N_ADAPTERS, RANK, TOPK = 28, 8, 2
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
+NCU_TRAFFIC = {"kernel_sha": None, "bytes_per_launch": {}}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--tokens", type=int, default=128, help="decode batch T per module")
+    ap.add_argument("--modules", type=int, default=16, help="independent MeteoRA modules visited per step")
+    ap.add_argument("--launch", choices=["graph", "stream"], default="graph")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target length of the cpu_baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            p = json.load(fh)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_sha():
+    with open(os.path.join(ROOT, "paper_2405_13053_b200", "csrc", "wgemm_tcgen05.cu"), "rb") as fh:
+        return hashlib.sha256(fh.read()).hexdigest()[:16]
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            f = [c.strip() for c in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """The CPU oracle, as it stands, on this machine's host cores: each step is one module's T tokens."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2405_13053_b200 import workloads
+
+    T = args.tokens
+    w = workloads.config1(T)
+    cores = oracle.num_threads()
+    steps, warmup = args.steps, args.warmup
+    # bound the run: the oracle needs ~21 ms of one core per token at this shape
+    budget_steps = max(1, int(60.0 / max(0.021 * T / cores, 1e-3)))
+    steps = min(steps, budget_steps)
+    warmup = min(warmup, max(1, budget_steps // 10))
+    for _ in range(warmup):
+        oracle.linear_forward(w["x"], w["W0"], w["A"], w["B"], w["Wg"], w.k)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.linear_forward(w["x"], w["W0"], w["A"], w["B"], w["Wg"], w.k)
+    dt = time.perf_counter() - t0
+    value = T * steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": 1e3 * dt / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config1: 4096->4096 MeteoRA linear, N=28 r=8 k=2, bf16-valued inputs, T={T}",
+                       "sample": f"one module, {T} tokens per step"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{steps} steps of {T} tokens of one module"},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import build as lib_build
+    from paper_2405_13053_b200 import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        lib_build.build_library()
+    if world > 1:
+        dist.barrier()
+    lib = mb.load_library()
+    import ctypes
+
+    T, R, K, W = args.tokens, args.modules, args.steps, max(args.warmup, 3)
+    dt = torch.bfloat16
+    shape = mb.make_shape(T, D_IN, D_OUT, N_ADAPTERS, RANK, TOPK, dt)
+    es = 2
+
+    # ---- inputs: R independent modules (seeded), resident in HBM; pinned host copies of x / y for e2e
+    mods = []
+    host_w0 = None
+    for i in range(R):
+        w = workloads.make_workload(f"config1/T{T}/module{i}", T=T, d_in=D_IN, d_out=D_OUT, N=N_ADAPTERS, r=RANK,
+                                    k=TOPK, dtype="bf16", x_kind="rms", seed=1000 + 100 * i + 17 * rank)
+        if i == 0:
+            host_w0 = w
+        m = {n: torch.from_numpy(w[n]).to(dt).cuda() for n in ("x", "W0", "A", "B", "Wg")}
+        m["y"] = torch.empty((T, D_OUT), dtype=dt, device="cuda")
+        m["ws"] = mb.alloc_workspace(shape)
+        m["x_host"] = torch.from_numpy(w["x"]).to(dt).pin_memory()
+        m["y_host"] = torch.empty((T, D_OUT), dtype=dt).pin_memory()
+        mods.append(m)
+    torch.cuda.synchronize()
+
+    def call_device(m):
+        rc = lib.meteora_linear_forward(m["x"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(), m["B"].data_ptr(),
+                                        m["Wg"].data_ptr(), ctypes.byref(shape), m["y"].data_ptr(),
+                                        m["ws"].data_ptr(), m["ws"].numel(), torch.cuda.current_stream().cuda_stream)
+        if rc != 0:
+            raise mb.MeteoraError(rc, "meteora_linear_forward")
+
+    def call_host(m):
+        rc = lib.meteora_linear_forward_host(m["x_host"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(),
+                                             m["B"].data_ptr(), m["Wg"].data_ptr(), ctypes.byref(shape),
+                                             m["y_host"].data_ptr(), m["ws"].data_ptr(), m["ws"].numel(),
+                                             torch.cuda.current_stream().cuda_stream)
+        if rc != 0:
+            raise mb.MeteoraError(rc, "meteora_linear_forward_host")
+
+    def step_device():
+        for m in mods:
+            call_device(m)
+
+    def step_host():
+        for m in mods:
+            call_host(m)
+
+    def make_runner(step_fn):
+        """Capture one step into a CUDA graph; fall back to direct launches if capture is refused."""
+        if args.launch == "graph":
+            try:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    step_fn()                                  # tensor maps get encoded outside the capture
+                torch.cuda.current_stream().wait_stream(side)
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    step_fn()
+                return g.replay, "graph"
+            except Exception as e:                             # noqa: BLE001
+                sys.stderr.write(f"[bench] graph capture failed ({e}); using direct launches\n")
+                torch.cuda.synchronize()
+        return step_fn, "stream"
+
+    def timed(run, steps, warmup):
+        for _ in range(warmup):
+            run()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    def check_status():
+        for m in mods:
+            st = mb.meteora_workspace_status(m["ws"])
+            if st != 0:
+                raise mb.MeteoraError(st, "device status after the timed region")
+
+    # ---- device-resident timing (the headline value)
+    run_dev, mode = make_runner(step_device)
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    sampler = ClockSampler(uuid)
+    ms_total = timed(run_dev, K, W)
+    # keep the GPU under the same load a little longer if the region was too short for a clock sample
+    t_extra = time.time()
+    while time.time() - t_extra < 0.7:
+        run_dev()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    check_status()
+    tokens_per_step = R * T * world
+    value = tokens_per_step * K / (ms_total * 1e-3)
+
+    # ---- end to end: x from pinned host memory, y back to host, every step, through the host entry point
+    run_e2e, mode_e2e = make_runner(step_host)
+
+    def e2e_step():
+        run_e2e()
+        torch.cuda.current_stream().synchronize()          # the step's result is read on the host
+
+    ms_e2e = timed(e2e_step, K, W)
+    check_status()
+    e2e_value = tokens_per_step * K / (ms_e2e * 1e-3)
+
+    # ---- dominant kernel: event pairs around the base-product launch of every call, same launches
+    prof_steps = min(K, 50)
+    step_device()
+    torch.cuda.synchronize()
+    mb.meteora_profile_begin(prof_steps * R)
+    for _ in range(prof_steps):
+        step_device()
+    kernel_ms, kernel_launches = mb.meteora_profile_end()
+    check_status()
+
+    # ---- algorithmic bytes (adapters actually selected, from the realised routing of module 0)
+    idx0, _ = mb.meteora_workspace_routing(shape, mods[0]["ws"])
+    touched = int(torch.unique(idx0).numel())
+    bytes_kernel = (D_IN * D_OUT + touched * D_OUT * RANK + T * (D_IN + D_OUT)) * es
+    bytes_path = bytes_kernel + (N_ADAPTERS * D_IN + touched * RANK * D_IN) * es
+    peak, peak_kind = measured_peaks()
+    per_launch_s = kernel_ms * 1e-3 / max(kernel_launches, 1)
+    achieved = bytes_kernel / per_launch_s / 1e9
+    traffic = None
+    if NCU_TRAFFIC["kernel_sha"] == kernel_sha():
+        traffic = NCU_TRAFFIC["bytes_per_launch"].get(str(T))
+    per_call_s = ms_total * 1e-3 / (K * R)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"config1: LLaMA3-8B q_proj MeteoRA linear 4096->4096, N=28 r=8 k=2, bf16, "
+                               f"decode batch T={T}; step = {R} independent modules",
+                   "tokens_per_module": T, "modules_per_step": R, "launch": mode, "e2e_launch": mode_e2e,
+                   "l2": f"weights of the {R} modules total {R * bytes_path / 1e6:.0f} MB > 126 MB L2, "
+                         "so no weight is L2-resident between visits",
+                   "parallelism": f"token-sharded replicas x{world}, no collective"},
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": R * T * D_IN * es,
+                "d2h_bytes_per_step": R * T * D_OUT * es, "ms_per_step": ms_e2e / K},
+        "gpu_launches": 3 * R * K,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "k_wgemm (base product + LoRA epilogue)", "achieved": achieved,
+                     "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic, "algorithmic_bytes_per_launch": bytes_kernel,
+                     "us_per_launch": per_launch_s * 1e6, "launches_timed": kernel_launches},
+        "path_roofline": {"bound": "hbm", "algorithmic_bytes_per_call": bytes_path, "us_per_call": per_call_s * 1e6,
+                          "achieved": bytes_path / per_call_s / 1e9, "peak": peak, "unit": "GB/s",
+                          "frac": bytes_path / per_call_s / 1e9 / peak, "adapters_touched": touched},
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        cores = oracle.num_threads()
+        w = host_w0
+        n_tok, t_cpu, chunk = 0, 0.0, min(T, 32)
+        while t_cpu < args.cpu_seconds and n_tok < 16384:
+            sl = slice(n_tok % T, n_tok % T + chunk) if n_tok % T + chunk <= T else slice(0, chunk)
+            t0 = time.perf_counter()
+            oracle.linear_forward(w["x"][sl], w["W0"], w["A"], w["B"], w["Wg"], w.k)
+            t_cpu += time.perf_counter() - t0
+            n_tok += chunk
+        line["cpu_baseline"] = {"value": n_tok / t_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                "sample": f"{n_tok} tokens of module 0 in chunks of {chunk} ({t_cpu:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -147,6 +147,18 @@ int meteora_workspace_init(void* workspace, void* stream);
 int meteora_workspace_status(void* workspace, void* stream);
 
 /*
+ * Timing of the dominant kernel (the base product with its LoRA epilogue) for roofline reports.
+ * Between meteora_profile_begin and meteora_profile_end every tensor-core meteora_linear_forward
+ * records a CUDA event pair around that one launch on the caller's stream (up to max_launches
+ * pairs; the launch is not overlapped with its predecessor while timed).  meteora_profile_end
+ * SYNCHRONISES on the recorded events and returns the summed kernel time and the launch count.
+ * The events are created on first use and kept for the life of the process; not thread-safe; not
+ * to be used during stream capture.
+ */
+int meteora_profile_begin(int max_launches);
+int meteora_profile_end(float* total_ms, int* launches);
+
+/*
  * Tuning knobs for measurements (process-wide, not thread-safe): "splits" (split-K cluster size,
  * 0 = automatic), "stages" (TMA ring depth, 0 = automatic), "tile_tokens" (tokens per tile, 0 =
  * automatic), "force_simt" (1 = never take the tensor-core path), "pdl" (1 = overlap the chained

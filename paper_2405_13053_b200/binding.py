@@ -24,7 +24,8 @@ STATUS = {0: "METEORA_OK", -1: "METEORA_ERR_INVALID_ARG", -2: "METEORA_ERR_UNSUP
 
 EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_linear_forward",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
-           "meteora_workspace_init", "meteora_workspace_status", "meteora_set_tuning", "meteora_status_string"]
+           "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
+           "meteora_set_tuning", "meteora_status_string"]
 
 
 class MeteoraShape(ctypes.Structure):
@@ -62,6 +63,8 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_workspace_routing.argtypes = [shp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.meteora_workspace_init.argtypes = [vp, vp]
     lib.meteora_workspace_status.argtypes = [vp, vp]
+    lib.meteora_profile_begin.argtypes = [ci]
+    lib.meteora_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci)]
     lib.meteora_set_tuning.argtypes = [ctypes.c_char_p, ci]
     lib.meteora_status_string.argtypes = [ci]
     lib.meteora_status_string.restype = ctypes.c_char_p
@@ -231,6 +234,17 @@ def meteora_workspace_init(workspace: torch.Tensor) -> None:
 def meteora_workspace_status(workspace: torch.Tensor) -> int:
     """Synchronises the current stream; returns 0 or METEORA_ERR_TIMEOUT (-6)."""
     return int(load_library().meteora_workspace_status(workspace.data_ptr(), _stream()))
+
+
+def meteora_profile_begin(max_launches: int) -> None:
+    _check(load_library().meteora_profile_begin(int(max_launches)), "meteora_profile_begin")
+
+
+def meteora_profile_end() -> Tuple[float, int]:
+    """Synchronises; returns (summed milliseconds of the timed base-product launches, their count)."""
+    ms, n = ctypes.c_float(), ctypes.c_int()
+    _check(load_library().meteora_profile_end(ctypes.byref(ms), ctypes.byref(n)), "meteora_profile_end")
+    return float(ms.value), int(n.value)
 
 
 def meteora_set_tuning(name: str, value: int) -> None:

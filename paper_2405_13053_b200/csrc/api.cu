@@ -2,6 +2,8 @@
 // dispatch between the tensor-core path and the plain CUDA-core path.
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 
 namespace meteora {
@@ -48,6 +50,18 @@ static int check_shape(const meteora_shape_t* s, bool need_out, bool need_r) {
     return METEORA_OK;
 }
 
+// Optional timing of the dominant kernel (the base product with its LoRA epilogue): while a profile is
+// open every forward records a CUDA event pair around that launch on the caller's stream.
+struct Profile {
+    std::vector<cudaEvent_t> ev;   // 2 * capacity events
+    int used = 0;                  // pairs recorded
+    bool open = false;
+};
+static Profile& profile() {
+    static Profile p;
+    return p;
+}
+
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 static int forward_device(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
@@ -59,7 +73,12 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
         if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, s, ws.topk_idx, ws.topk_w, ws.uw, pdl,
                                              st)) != METEORA_OK)
             return rc;
-        return launch_base_lora_tc(x, W0, B, s, ws, y, pdl, st);
+        Profile& pf = profile();
+        const bool timed = pf.open && 2 * (pf.used + 1) <= (int)pf.ev.size();
+        if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
+        rc = launch_base_lora_tc(x, W0, B, s, ws, y, pdl && !timed, st);
+        if (timed) cudaEventRecord(pf.ev[2 * pf.used++ + 1], st);
+        return rc;
     }
     if ((rc = launch_gate_topk(x, Wg, s, ws.topk_idx, ws.topk_w, nullptr, st)) != METEORA_OK) return rc;
     if ((rc = launch_shrink_tokens(x, A, ws.topk_idx, ws.topk_w, s, ws.uw, st)) != METEORA_OK) return rc;
@@ -179,6 +198,37 @@ int meteora_workspace_status(void* workspace, void* stream) {
         if (cudaStreamSynchronize(st) != cudaSuccess) return METEORA_ERR_CUDA;
         return METEORA_ERR_TIMEOUT;
     }
+    return METEORA_OK;
+}
+
+int meteora_profile_begin(int max_launches) {
+    Profile& pf = profile();
+    if (max_launches <= 0 || max_launches > (1 << 20)) return METEORA_ERR_INVALID_ARG;
+    while ((int)pf.ev.size() < 2 * max_launches) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return METEORA_ERR_CUDA;
+        pf.ev.push_back(e);
+    }
+    pf.used = 0;
+    pf.open = true;
+    return METEORA_OK;
+}
+
+int meteora_profile_end(float* total_ms, int* launches) {
+    Profile& pf = profile();
+    if (!total_ms || !launches) return METEORA_ERR_INVALID_ARG;
+    pf.open = false;
+    float sum = 0.f;
+    for (int i = 0; i < pf.used; ++i) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(pf.ev[2 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, pf.ev[2 * i], pf.ev[2 * i + 1]) != cudaSuccess)
+            return METEORA_ERR_CUDA;
+        sum += ms;
+    }
+    *total_ms = sum;
+    *launches = pf.used;
+    pf.used = 0;
     return METEORA_OK;
 }
 
