@@ -30,7 +30,7 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     ws.topk_idx = (int32_t*)take(T * s.k * sizeof(int32_t));
     ws.topk_w = (float*)take(T * s.k * sizeof(float));
     ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
-    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float));
+    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (s.T <= 256 ? 4 : 1));   // up to 4 slices for decode batches
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);
     ws.bytes = off;
@@ -70,7 +70,7 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
     if (tc_path_supported(s)) {
         const bool pdl = tuning().pdl != 0;
         if ((rc = launch_stacked_shrink_tc(x, A, Wg, s, ws, st)) != METEORA_OK) return rc;
-        if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, s, ws.topk_idx, ws.topk_w, ws.uw, pdl,
+        if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, tc_stacked_zsplits(s), s, ws.topk_idx, ws.topk_w, ws.uw, pdl,
                                              st)) != METEORA_OK)
             return rc;
         Profile& pf = profile();

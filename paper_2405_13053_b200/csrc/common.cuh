@@ -17,7 +17,8 @@ struct Workspace {
     int32_t* topk_idx;  // [T,k]
     float* topk_w;      // [T,k]
     float* uw;          // [T,k,r]   w_j * (A_{i_j} x): the shrunk, gate-weighted activations
-    float* u_all;       // [T,ld_u]  stacked shrink: every adapter's A_i x, then the gate logits
+    float* u_all;       // [Z][T,ld_u]  stacked shrink: every adapter's A_i x, then the gate logits; Z partial
+                        //           copies (slices of the contraction axis) that the selection kernel adds up
     int ld_u;           // row pitch of u_all in floats
     int col_logits;     // first logit column inside a u_all row
     void* x_dev;        // [T,d_in]  staging for the host-buffer entry point
@@ -36,7 +37,7 @@ inline size_t elem_size(meteora_dtype_t t) { return t == METEORA_BF16 ? 2 : 4; }
 // gate_topk.cu
 int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, int32_t* topk_idx, float* topk_w,
                      float* logits, cudaStream_t st);
-int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, const meteora_shape_t& s,
+int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int zsplits, const meteora_shape_t& s,
                                int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st);
 // route.cu
 int launch_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets, int32_t* perm,
@@ -54,6 +55,7 @@ int launch_gemm_simt(const void* x, const void* W0, const void* B, const int32_t
 // wgemm_tcgen05.cu
 bool tc_path_supported(const meteora_shape_t& s);
 int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits);  // row pitch (floats) of u_all
+int tc_stacked_zsplits(const meteora_shape_t& s);                 // copies of u_all the stacked shrink writes (<= 4)
 int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const meteora_shape_t& s,
                              const Workspace& ws, cudaStream_t st);
 int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,

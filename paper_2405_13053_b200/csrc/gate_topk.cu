@@ -71,10 +71,12 @@ k_gate_topk(const TI* __restrict__ x, const TI* __restrict__ Wg, int T, int d_in
 }
 
 // Selection from the stacked shrink: row t of u_all holds A_i x for every adapter (N*r values)
-// and, from column col_logits on, the N gate logits.  Besides the picks and weights this writes
+// and, from column col_logits on, the N gate logits.  u_all comes as `zsplits` partial copies (slices
+// of the contraction axis, zstride floats apart) that are added here in slice order.  Besides the picks and weights this writes
 // uw[t,j,:] = w_j * (A_{i_j} x), the activations the base product's epilogue expands.
 __global__ void __launch_bounds__(kGateWarps * 32)
-k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits, int T, int N, int r, int k,
+k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits, int zsplits, size_t zstride, int T,
+                      int N, int r, int k,
                       float inv_tau, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
                       float* __restrict__ uw, int pdl) {
     if (pdl) {
@@ -87,8 +89,11 @@ k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits,
     const int t = blockIdx.x * kGateWarps + (threadIdx.x >> 5);
     if (t >= T) return;
     const float* row = u_all + (size_t)t * ld_u;
-    const float v0 = lane < N ? row[col_logits + lane] : 0.f;
-    const float v1 = lane + 32 < N ? row[col_logits + lane + 32] : 0.f;
+    float v0 = 0.f, v1 = 0.f;
+    for (int z = 0; z < zsplits; ++z) {
+        if (lane < N) v0 += row[z * zstride + col_logits + lane];
+        if (lane + 32 < N) v1 += row[z * zstride + col_logits + lane + 32];
+    }
     int idx;
     float w;
     warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
@@ -101,7 +106,11 @@ k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits,
         const int j = min(c / r, k - 1), p = c - j * r;
         const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
         const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
-        if (c < k * r) uw[(size_t)t * k * r + c] = wj * row[ij * r + p];
+        if (c < k * r) {
+            float u = 0.f;
+            for (int z = 0; z < zsplits; ++z) u += row[z * zstride + ij * r + p];
+            uw[(size_t)t * k * r + c] = wj * u;
+        }
     }
 }
 
@@ -119,7 +128,7 @@ int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, in
     return last_launch_status();
 }
 
-int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, const meteora_shape_t& s,
+int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int zsplits, const meteora_shape_t& s,
                                int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st) {
     if (s.T == 0) return METEORA_OK;
     const int blocks = (s.T + kGateWarps - 1) / kGateWarps;
@@ -133,7 +142,8 @@ int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, con
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     const float inv_tau = 1.0f / s.temperature;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_select_from_stacked, u_all, ld_u, col_logits, s.T, s.N, s.r, s.k,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_select_from_stacked, u_all, ld_u, col_logits, zsplits,
+                                       (size_t)s.T * ld_u, s.T, s.N, s.r, s.k,
                                        inv_tau, topk_idx, topk_w, uw, pdl ? 1 : 0);
     return cuda_status(e);
 }

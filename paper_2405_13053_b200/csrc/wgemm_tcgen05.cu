@@ -12,9 +12,9 @@
 // axis is split over a thread-block cluster and the partial accumulators are summed through distributed
 // shared memory in a fixed order (deterministic, no global scratch).
 //
-// Warp roles (192 threads): warp 0 lane 0 issues TMA loads into a ring of shared-memory stages, warp 1
-// owns the TMEM allocation and lane 0 issues tcgen05.mma, warps 2-5 run the epilogue (TMEM lane quarter
-// = warp id % 4).  Every mbarrier wait is bounded; on expiry the kernel records it in the status word
+// Warp roles (320 threads): warp 0 lane 0 issues TMA loads into a ring of shared-memory stages, warp 1
+// owns the TMEM allocation and lane 0 issues tcgen05.mma, warps 2-9 run the epilogue (TMEM lane quarter
+// = warp id % 4, two warps per quarter sharing the columns).  Every mbarrier wait is bounded; on expiry the kernel records it in the status word
 // and drains instead of hanging.
 #include <cuda.h>
 
@@ -28,10 +28,11 @@ namespace meteora {
 constexpr int kBM = 128;       // weight rows per tile (UMMA M)
 constexpr int kBK = 64;        // contraction elements per stage: one 128-byte swizzled row of bf16
 constexpr int kUmmaK = 16;     // contraction elements per tcgen05.mma (32 bytes of bf16)
-constexpr int kThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kThreads = 320;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2-9: epilogue
+constexpr int kEpiThreads = 256;
 constexpr int kWTileBytes = kBM * kBK * 2;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // about a second
+constexpr int kMaxZSplits = 4;
 
 enum { MODE_STACKED = 0, MODE_LORA = 1 };
 
@@ -39,6 +40,8 @@ struct WGemmParams {
     int T, K;            // tokens, contraction length
     int BN;              // tokens per tile (multiple of 16, <= 256)
     int splits;          // cluster size along the contraction axis
+    int zsplits;         // gridDim.z: further split of the contraction axis; slice z writes its own u_all copy
+    size_t u_all_zstride;   // floats between the u_all copies
     int ksteps;          // ceil(K / kBK)
     int stages;          // depth of the TMA ring
     int tmem_cols;       // power of two >= max(32, BN)
@@ -52,6 +55,10 @@ struct WGemmParams {
     const __nv_bfloat16* B;
     __nv_bfloat16* y;
     int d_out, N, r, k;
+    int epi_off;         // byte offset of the epilogue staging area behind the ring
+    int uw_off, slab_off;   // byte offsets of s_uw and the B slab inside that area
+    int slab_q;          // slab entries held in shared memory (0: read B from global memory)
+    int per_slot;        // slab indexed by slot t*k+j instead of by adapter
     int32_t* status;
     int pdl_wait;        // epilogue waits for the preceding grid before reading its results
     int pdl_trigger;     // let the dependent grid start as soon as this one is resident
@@ -128,14 +135,6 @@ __device__ __forceinline__ uint32_t cluster_rank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank) {
-    uint32_t remote;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-    return v;
-}
-
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, 128-byte swizzled
 // (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B): start address, leading byte offset unused
 // (1), stride byte offset 1024 (eight rows), descriptor version 1, swizzle mode 2 (128 B).
@@ -153,43 +152,164 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int bn) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Epilogue of one accumulator element: row of the launch's row space, token index, fp32 sum.
+// Epilogue.  The accumulator tile is parked in shared memory as part[t][row] (row fastest) by the four
+// epilogue warps; CTA `split` of the cluster then owns rows [128*split/S, 128*(split+1)/S) of the tile
+// and sums, in rank order, the S partial tiles of the cluster for those rows (its own through shared
+// memory, its peers' through distributed shared memory).  A thread finishes two adjacent rows of one
+// token at a time, so y is written as packed bf16 pairs, 4 bytes per thread, contiguous across lanes.
+//
+// What the LoRA expand needs is staged in shared memory while the main loop still streams W0:
+//   s_e[t][j]   adapter picked by token t at rank j,
+//   s_uw[t][j][:] = w_j * (A_e x_t)  (fp32, from the selection kernel),
+//   slab[q][row][:]  the B rows of this CTA's row slice, q = adapter (all N of them) or, when the tile
+//                    holds fewer (token, pick) slots than there are adapters, q = slot t*k+j.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void finish_element(const WGemmParams& p, int tile_m, int row_in_tile, int token,
-                                               float acc) {
-    if (token >= p.T) return;
-    if (p.mode == MODE_STACKED) {
-        int row, col;
-        if (tile_m < p.split_tile) {
-            row = tile_m * kBM + row_in_tile;
-            if (row >= p.rows0) return;
-            col = row;
-        } else {
-            row = (tile_m - p.split_tile) * kBM + row_in_tile;
-            if (row >= p.rows1) return;
-            col = p.col1 + row;
-        }
-        p.u_all[(size_t)token * p.ld_u + col] = acc;
+__device__ __forceinline__ float2 ld_part2(uint32_t local_addr, uint32_t rank, bool remote) {
+    float2 v;
+    if (remote) {
+        uint32_t a;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank));
+        asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
     } else {
-        const int o = tile_m * kBM + row_in_tile;
-        if (o >= p.d_out) return;
-        const int32_t* ti = p.topk_idx + (size_t)token * p.k;
-        const float* uq = p.uw + (size_t)token * p.k * p.r;
-        for (int j = 0; j < p.k; ++j) {
-            const int e = min(max(__ldg(ti + j), 0), p.N - 1);
-            const __nv_bfloat16* brow = p.B + ((size_t)e * p.d_out + o) * p.r;
-            for (int q = 0; q < p.r; q += 8) {
-                float bv[8];
-                load8(brow + q, bv);
-                const float4 u0 = __ldg(reinterpret_cast<const float4*>(uq + j * p.r + q));
-                const float4 u1 = __ldg(reinterpret_cast<const float4*>(uq + j * p.r + q + 4));
-                acc = fmaf(bv[0], u0.x, acc); acc = fmaf(bv[1], u0.y, acc);
-                acc = fmaf(bv[2], u0.z, acc); acc = fmaf(bv[3], u0.w, acc);
-                acc = fmaf(bv[4], u1.x, acc); acc = fmaf(bv[5], u1.y, acc);
-                acc = fmaf(bv[6], u1.z, acc); acc = fmaf(bv[7], u1.w, acc);
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(local_addr));
+    }
+    return v;
+}
+
+__device__ __forceinline__ void fma8(const uint4& b, const float4& u0, const float4& u1, float& acc) {
+    acc = fmaf(__uint_as_float(b.x << 16), u0.x, acc);
+    acc = fmaf(__uint_as_float(b.x & 0xFFFF0000u), u0.y, acc);
+    acc = fmaf(__uint_as_float(b.y << 16), u0.z, acc);
+    acc = fmaf(__uint_as_float(b.y & 0xFFFF0000u), u0.w, acc);
+    acc = fmaf(__uint_as_float(b.z << 16), u1.x, acc);
+    acc = fmaf(__uint_as_float(b.z & 0xFFFF0000u), u1.y, acc);
+    acc = fmaf(__uint_as_float(b.w << 16), u1.z, acc);
+    acc = fmaf(__uint_as_float(b.w & 0xFFFF0000u), u1.w, acc);
+}
+
+// Stage s_e, s_uw and the B slab of rows [row0, row0 + nrows) (epilogue threads only).
+__device__ __forceinline__ void stage_lora_operands(const WGemmParams& p, uint8_t* epi, int tok0, int ntok, int row0,
+                                                    int nrows, int etid) {
+    int* s_e = reinterpret_cast<int*>(epi);
+    float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off);
+    uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
+    const int slots = ntok * p.k;
+    for (int i = etid; i < slots; i += kEpiThreads)
+        s_e[i] = min(max(__ldg(p.topk_idx + (size_t)tok0 * p.k + i), 0), p.N - 1);
+    const float4* uw4 = reinterpret_cast<const float4*>(p.uw + (size_t)tok0 * p.k * p.r);
+    for (int i = etid; i < slots * p.r / 4; i += kEpiThreads) s_uw4[i] = __ldg(uw4 + i);
+    if (p.slab_q > 0) {
+        const int vpr = p.r >> 3;                      // 16-byte vectors per B row
+        const int vpe = nrows * vpr;                   // vectors per slab entry
+        const int nq = p.per_slot ? slots : p.N;
+        const int total = nq * vpe;
+        const uint4* Bv = reinterpret_cast<const uint4*>(p.B);
+        constexpr int U = 4;                           // independent loads in flight per thread
+        for (int v0 = etid; v0 < total; v0 += U * kEpiThreads) {
+            uint4 val[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * kEpiThreads;
+                val[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (v < total) {
+                    const int q = v / vpe, w = v - q * vpe;
+                    const int rr = w / vpr;
+                    const int e = p.per_slot ? min(max(__ldg(p.topk_idx + (size_t)tok0 * p.k + q), 0), p.N - 1) : q;
+                    if (row0 + rr < p.d_out) val[u] = __ldg(Bv + ((size_t)e * p.d_out + row0) * vpr + w);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * kEpiThreads;
+                if (v < total) slab[v] = val[u];
             }
         }
-        p.y[(size_t)token * p.d_out + o] = __float2bfloat16_rn(acc);
+    }
+}
+
+// One (row pair, token) result: add the LoRA expand and store.
+__device__ __forceinline__ void finish_pair(const WGemmParams& p, const uint8_t* epi, int tile_m, int row_in_tile,
+                                            int nrows, int pr, int t, int token, float a0, float a1) {
+    if (p.mode == MODE_STACKED) {
+        int row = tile_m * kBM + row_in_tile, limit = p.rows0, col = row;
+        if (tile_m >= p.split_tile) {
+            row = (tile_m - p.split_tile) * kBM + row_in_tile;
+            limit = p.rows1;
+            col = p.col1 + row;
+        }
+        float* dst = p.u_all + (size_t)blockIdx.z * p.u_all_zstride + (size_t)token * p.ld_u + col;
+        if (row + 1 < limit) {
+            *reinterpret_cast<float2*>(dst) = make_float2(a0, a1);
+        } else if (row < limit) {
+            dst[0] = a0;
+        }
+        return;
+    }
+    const int* s_e = reinterpret_cast<const int*>(epi);
+    const float4* s_uw4 = reinterpret_cast<const float4*>(epi + p.uw_off);
+    const uint4* slab = reinterpret_cast<const uint4*>(epi + p.slab_off);
+    const int vpr = p.r >> 3;
+    const int o = tile_m * kBM + row_in_tile;
+    for (int j = 0; j < p.k; ++j) {
+        const int slot = t * p.k + j;
+        const int e = s_e[slot];
+        for (int c = 0; c < vpr; ++c) {
+            uint4 b0, b1;
+            if (p.slab_q > 0) {
+                const int q = p.per_slot ? slot : e;
+                b0 = slab[(q * nrows + 2 * pr) * vpr + c];
+                b1 = slab[(q * nrows + 2 * pr + 1) * vpr + c];
+            } else {
+                const uint4* Bv = reinterpret_cast<const uint4*>(p.B) + ((size_t)e * p.d_out + o) * vpr + c;
+                b0 = o < p.d_out ? __ldg(Bv) : make_uint4(0u, 0u, 0u, 0u);
+                b1 = o + 1 < p.d_out ? __ldg(Bv + vpr) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            const float4 u0 = s_uw4[(slot * p.r >> 2) + 2 * c];
+            const float4 u1 = s_uw4[(slot * p.r >> 2) + 2 * c + 1];
+            fma8(b0, u0, u1, a0);
+            fma8(b1, u0, u1, a1);
+        }
+    }
+    __nv_bfloat16* dst = p.y + (size_t)token * p.d_out + o;
+    if (o + 1 < p.d_out && (p.d_out & 1) == 0) {
+        *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(a0, a1);
+    } else {
+        if (o < p.d_out) dst[0] = __float2bfloat16_rn(a0);
+        if (o + 1 < p.d_out) dst[1] = __float2bfloat16_rn(a1);
+    }
+}
+
+template <int S>
+__device__ __forceinline__ void reduce_and_finish(const WGemmParams& p, uint32_t ring, const uint8_t* epi, int tile_m,
+                                                  int split, int tok0, int ntok, int etid) {
+    constexpr int P = 64 / S;                 // row pairs of this CTA's slice
+    constexpr int TPP = kEpiThreads / P;      // tokens handled per pass of the epilogue threads
+    constexpr int NROWS = kBM / S;
+    constexpr int U = S >= 4 ? 2 : 4;         // tokens in flight per thread
+    const int pr = etid % P, tg = etid / P;
+    const int row_in_tile = NROWS * split + 2 * pr;
+
+    for (int t0 = tg; t0 < ntok; t0 += U * TPP) {
+        float2 part[U][S];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int t = min(t0 + u * TPP, ntok - 1);
+            const uint32_t addr = ring + (uint32_t)((t * kBM + row_in_tile) * 4);
+#pragma unroll
+            for (int q = 0; q < S; ++q) part[u][q] = ld_part2(addr, (uint32_t)q, S > 1);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int t = t0 + u * TPP;
+            if (t >= ntok) break;
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int q = 0; q < S; ++q) {
+                a0 += part[u][q].x;
+                a1 += part[u][q].y;
+            }
+            finish_pair(p, epi, tile_m, row_in_tile, NROWS, pr, t, tok0 + t, a0, a1);
+        }
     }
 }
 
@@ -203,16 +323,21 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const uint32_t stage_bytes = kWTileBytes + p.BN * 128;
     const uint32_t ring_bytes = p.stages * stage_bytes;
     const uint32_t bar_base = ring + ring_bytes;                 // full[stages], empty[stages], acc (8 bytes each)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + (2 * p.stages + 1) * 8);
     const uint32_t bar_acc = bar_base + 2 * p.stages * 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + (2 * p.stages + 1) * 8);
+    uint8_t* epi = ring_ptr + ring_bytes + p.epi_off;             // staging of the LoRA operands
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.splits;
     const int split = (int)cluster_rank();
     const int tile_m = blockIdx.x / S;
     const int tok0 = blockIdx.y * p.BN;
-    const int ks0 = (int)(((long long)p.ksteps * split) / S);
-    const int ks1 = (int)(((long long)p.ksteps * (split + 1)) / S);
+    const int ntok = min(p.BN, p.T - tok0);
+    // contraction range of this CTA: first cut by grid z, then by cluster rank
+    const int kz0 = (int)(((long long)p.ksteps * blockIdx.z) / p.zsplits);
+    const int kz1 = (int)(((long long)p.ksteps * (blockIdx.z + 1)) / p.zsplits);
+    const int ks0 = kz0 + (int)(((long long)(kz1 - kz0) * split) / S);
+    const int ks1 = kz0 + (int)(((long long)(kz1 - kz0) * (split + 1)) / S);
     const int nks = ks1 - ks0;
 
     if (p.pdl_trigger && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -245,7 +370,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
             const int row0 = (second ? tile_m - p.split_tile : tile_m) * kBM;
             int issued = 0;
             bool ok = true;
-            for (int i = 0; i < nks && ok; ++i) {
+            for (int i = 0; i < nks; ++i) {
                 const int s = i % p.stages, round = i / p.stages;
                 if (round > 0) ok = mbar_wait(bar_base + (p.stages + s) * 8, (round & 1) ^ 1);
                 if (!ok) break;
@@ -284,16 +409,14 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
                 atomicExch(p.status + 2, 200);
             }
         }
-    }
-    __syncwarp();
-
-    // ---------------------------------------------------------------------- epilogue
-    const bool epi = warp >= 2;
-    const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
-    const int etid = threadIdx.x - 64;            // 0..127 among the epilogue threads
-    bool acc_ok = true;
-    if (epi) {
+    } else {
+        // ------------------------------------------------------------------ epilogue warps, part 1
+        const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
+        const int etid = threadIdx.x - 64;
         if (p.pdl_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (p.mode == MODE_LORA)
+            stage_lora_operands(p, epi, tok0, ntok, tile_m * kBM + (kBM / S) * split, kBM / S, etid);
+        bool acc_ok = true;
         if (nks > 0) {
             acc_ok = mbar_wait(bar_acc, 0);
             if (!acc_ok && lane == 0) {
@@ -303,59 +426,38 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         }
         acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);   // keep the warp-collective TMEM loads convergent
         tc_fence_after();
+        // Park the accumulators in the ring, which is idle now: every load has landed and every MMA that
+        // read it has completed.
+        float* part = reinterpret_cast<float*>(ring_ptr);
+        const int row_in_tile = quad * 32 + lane;
+        const int half = ((p.BN / 16 + 1) / 2) * 16;            // warps 2-5 take columns [0, half), warps 6-9 the rest
+        const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
+        for (int c = c_begin; c < c_end; c += 16) {
+            float v[16];
+            if (nks > 0 && acc_ok) {
+                tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) part[(c + i) * kBM + row_in_tile] = v[i];
+        }
     }
+    __syncwarp();
+    if (S > 1) cluster_sync(); else __syncthreads();
 
-    if (S == 1) {
-        if (epi) {
-            const int row_in_tile = quad * 32 + lane;
-            for (int c = 0; c < p.BN; c += 16) {
-                float v[16];
-                if (nks > 0 && acc_ok) {
-                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                }
-                if (acc_ok) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) finish_element(p, tile_m, row_in_tile, tok0 + c + i, v[i]);
-                }
-            }
+    if (warp >= 2) {
+        const int etid = threadIdx.x - 64;
+        switch (S) {
+            case 1: reduce_and_finish<1>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
+            case 2: reduce_and_finish<2>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
+            case 4: reduce_and_finish<4>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
+            default: reduce_and_finish<8>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
         }
-    } else {
-        // Partial accumulators go to shared memory (the ring is idle now: every load has landed and every
-        // MMA that read it has completed), then each CTA of the cluster sums one slice of the 128 rows
-        // over all partials, in rank order, reading its peers through distributed shared memory.
-        float* part = reinterpret_cast<float*>(ring_ptr);          // part[t][row], row fastest
-        if (epi) {
-            const int row_in_tile = quad * 32 + lane;
-            for (int c = 0; c < p.BN; c += 16) {
-                float v[16];
-                if (nks > 0 && acc_ok) {
-                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                }
-#pragma unroll
-                for (int i = 0; i < 16; ++i) part[(c + i) * kBM + row_in_tile] = v[i];
-            }
-        }
-        cluster_sync();
-        if (epi && acc_ok) {
-            const int lo = (kBM * split) / S, hi = (kBM * (split + 1)) / S;
-            const int nrows = hi - lo;
-            const int items = nrows * p.BN;
-            for (int it = etid; it < items; it += kEpiThreads) {
-                const int t = it / nrows, rl = it - t * nrows;
-                const uint32_t addr = ring + (uint32_t)((t * kBM + lo + rl) * 4);
-                float acc = 0.f;
-                for (int q = 0; q < S; ++q) acc += ld_peer_f32(addr, (uint32_t)q);
-                finish_element(p, tile_m, lo + rl, tok0 + t, acc);
-            }
-        }
-        cluster_sync();   // nobody leaves while a peer may still read its partials
     }
+    __syncwarp();
+    if (S > 1) cluster_sync();   // nobody leaves while a peer may still read its partials
 
     tc_fence_before();
     __syncthreads();
@@ -452,35 +554,78 @@ int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits) {
     return a_tiles * kBM + (int)align_up((size_t)s.N, 32);
 }
 
+struct Plan;
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k);
+
 struct Plan {
-    int BN, n_tiles, splits, stages, tmem_cols;
+    int BN, n_tiles, splits, zsplits, stages, tmem_cols;
+    int epi_off, uw_off, slab_off, slab_q, per_slot;
     size_t smem;
 };
 
-static Plan make_plan(int row_tiles, int T, int K) {
+// Tile shape, split-K factor and shared-memory budget of one launch.
+//   - tokens per tile: the whole batch when it fits one UMMA N (<= 256), else 256;
+//   - split-K cluster size S in {1,2,4,8}: the largest that keeps one CTA per SM; if that leaves more
+//     than a quarter of the SMs idle, the next one (two CTAs per SM share the shared memory);
+//   - ring depth: whatever the shared memory left after the epilogue staging allows.
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k) {
     const Tuning& tn = tuning();
-    Plan pl;
+    Plan pl = {};
     const int ksteps = (K + kBK - 1) / kBK;
     int bn = tn.tile_tokens > 0 ? tn.tile_tokens : (T <= 256 ? (T + 15) / 16 * 16 : 256);
     bn = std::min(256, std::max(16, (bn + 15) / 16 * 16));
     pl.BN = bn;
     pl.n_tiles = (T + bn - 1) / bn;
     const int tiles = row_tiles * pl.n_tiles;
-    int splits = tn.splits > 0 ? tn.splits : std::max(1, sm_count() / tiles);
-    splits = std::min(std::min(splits, 8), ksteps);
+    const int sms = sm_count();
+    int splits = 1;
+    if (tn.splits > 0) {
+        splits = tn.splits >= 8 ? 8 : tn.splits >= 4 ? 4 : tn.splits >= 2 ? 2 : 1;
+    } else {
+        while (splits < 8 && tiles * splits * 2 <= sms) splits *= 2;
+        if (splits < 8 && tiles * splits * 4 < sms * 3 && tiles * splits * 2 <= 2 * sms) splits *= 2;
+    }
+    while (splits > 1 && splits > ksteps) splits /= 2;
     pl.splits = splits;
-    const int nks = (ksteps + splits - 1) / splits;
+    // The stacked shrink of a decode batch has only a handful of row tiles: cut its contraction axis
+    // further over grid z (every slice keeps at least two k-steps); the selection kernel adds the slices.
+    pl.zsplits = 1;
+    if (!lora && pl.n_tiles == 1) pl.zsplits = std::min(kMaxZSplits, std::max(1, ksteps / splits / 2));
+    const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
+    const bool two_per_sm = tiles * splits * pl.zsplits > sms;
+    const size_t total_budget = two_per_sm ? 112 * 1024 : 226 * 1024;
+
+    // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
+    const int tile_tokens = std::min(T, bn);
+    size_t epi_bytes = 0;
+    if (lora) {
+        pl.uw_off = (int)align_up((size_t)bn * k * 4, 16);
+        pl.slab_off = pl.uw_off + bn * k * r * 4;
+        pl.per_slot = tile_tokens * k <= N ? 1 : 0;
+        const int q = pl.per_slot ? tile_tokens * k : N;
+        const size_t slab_bytes = (size_t)q * (kBM / splits) * r * 2;
+        pl.slab_q = slab_bytes <= 64 * 1024 ? q : 0;
+        epi_bytes = pl.slab_off + (pl.slab_q > 0 ? slab_bytes : 0);
+    }
     const size_t stage_bytes = kWTileBytes + (size_t)bn * 128;
-    const size_t budget = (splits == 1 && tiles > sm_count()) ? 98 * 1024 : 200 * 1024;  // two CTAs per SM when tiles queue up
-    int stages = tn.stages > 0 ? tn.stages : (int)std::min<size_t>((size_t)nks, budget / stage_bytes);
+    const size_t part_bytes = (size_t)bn * kBM * 4;           // accumulators parked in the idle ring
+    const size_t fixed = 1024 + 256 + epi_bytes;               // alignment slack + barriers + staging
+    const int nks = ksteps_cta + 1;
+    int stages;
+    if (tn.stages > 0) {
+        stages = tn.stages;
+    } else {
+        const size_t avail = total_budget > fixed ? total_budget - fixed : 0;
+        stages = (int)std::min<size_t>((size_t)nks, avail / stage_bytes);
+    }
     stages = std::max(stages, 2);
-    if (splits > 1)   // the partial accumulators (bn * 512 bytes) are parked in the idle ring
-        while ((size_t)stages * stage_bytes < (size_t)bn * 512) ++stages;
+    while ((size_t)stages * stage_bytes < part_bytes) ++stages;
     pl.stages = stages;
     int cols = 32;
     while (cols < bn) cols *= 2;
     pl.tmem_cols = cols;
-    pl.smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 1) * 8 + 16;
+    pl.epi_off = (int)align_up((size_t)(2 * stages + 1) * 8 + 16, 16);
+    pl.smem = 1024 + (size_t)stages * stage_bytes + pl.epi_off + epi_bytes;
     return pl;
 }
 
@@ -497,7 +642,7 @@ static int launch_wgemm(const CUtensorMap& m0, const CUtensorMap& m1, const CUte
         smem_set[dev] = 227 * 1024;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(row_tiles * pl.splits, pl.n_tiles);
+    cfg.gridDim = dim3(row_tiles * pl.splits, pl.n_tiles, pl.zsplits);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
@@ -518,14 +663,26 @@ static int launch_wgemm(const CUtensorMap& m0, const CUtensorMap& m1, const CUte
     return cuda_status(cudaLaunchKernelEx(&cfg, k_wgemm, m0, m1, mx, p));
 }
 
+static int stacked_row_tiles(const meteora_shape_t& s) { return (s.N * s.r + kBM - 1) / kBM + 1; }
+
+int tc_stacked_zsplits(const meteora_shape_t& s) {
+    return make_plan(stacked_row_tiles(s), s.T, s.d_in, false, s.N, s.r, s.k).zsplits;
+}
+
 static void fill_common(WGemmParams& p, const Plan& pl, int T, int K, int32_t* status) {
     p.T = T;
     p.K = K;
     p.BN = pl.BN;
     p.splits = pl.splits;
+    p.zsplits = pl.zsplits;
     p.ksteps = (K + kBK - 1) / kBK;
     p.stages = pl.stages;
     p.tmem_cols = pl.tmem_cols;
+    p.epi_off = pl.epi_off;
+    p.uw_off = pl.uw_off;
+    p.slab_off = pl.slab_off;
+    p.slab_q = pl.slab_q;
+    p.per_slot = pl.per_slot;
     p.status = status;
 }
 
@@ -534,7 +691,7 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     const int a_rows = s.N * s.r;
     const int a_tiles = (a_rows + kBM - 1) / kBM;
     const int row_tiles = a_tiles + 1;
-    const Plan pl = make_plan(row_tiles, s.T, s.d_in);
+    const Plan pl = make_plan(row_tiles, s.T, s.d_in, false, s.N, s.r, s.k);
     CUtensorMap mA, mG, mX;
     int rc;
     if ((rc = get_tensor_map(A, s.d_in, a_rows, kBM, &mA)) != METEORA_OK) return rc;
@@ -547,6 +704,7 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     p.rows1 = s.N;
     p.mode = MODE_STACKED;
     p.u_all = ws.u_all;
+    p.u_all_zstride = (size_t)s.T * ws.ld_u;
     p.ld_u = ws.ld_u;
     p.col1 = ws.col_logits;
     p.pdl_wait = 0;
@@ -557,7 +715,7 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
 int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
                         void* y, bool pdl, cudaStream_t st) {
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
-    const Plan pl = make_plan(row_tiles, s.T, s.d_in);
+    const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     CUtensorMap mW, mX;
     int rc;
     if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, &mW)) != METEORA_OK) return rc;
