@@ -41,6 +41,7 @@ extern "C" {
 #define METEORA_MAX_N 64
 #define METEORA_MAX_K 8
 #define METEORA_MAX_R 64
+#define METEORA_STATIC_SCRATCH_FLOATS 65536 /* capacity of meteora_lora_delta_static: T * k * r may not exceed it */
 
 typedef enum { METEORA_F32 = 0, METEORA_BF16 = 1 } meteora_dtype_t;
 
@@ -100,6 +101,33 @@ int meteora_lora_delta(const void* x, const void* A, const void* B, const int32_
                        const float* topk_w, const int32_t* offsets, const int32_t* perm,
                        const meteora_shape_t* shape, float* delta, void* workspace, size_t workspace_bytes,
                        void* stream);
+
+/*
+ * meteora_lora_delta without a workspace.  (The paper has no counterpart: this entry point exists for the
+ * way the library is embedded, not for the method.)
+ *
+ * Who it is for: callers that cannot allocate device memory at the point where they need the LoRA term,
+ * and so have no workspace to pass: code running inside another framework's allocator lock or stream
+ * callback, serving loops whose memory pool is frozen after start-up, bindings that can launch but not
+ * allocate.  The scratch that meteora_lora_delta takes from its workspace (the shrunk activations, T*k*r
+ * floats) lives here in a fixed device array inside the library, METEORA_STATIC_SCRATCH_FLOATS floats
+ * (256 KB) on every GPU that loads the library, for the life of the process.  The call allocates nothing
+ * and frees nothing.
+ *
+ * Arguments, layouts and result are those of meteora_lora_delta (inputs and delta[T,d_out] fp32 are still
+ * the caller's).  Differences:
+ *   - T * k * r > METEORA_STATIC_SCRATCH_FLOATS returns METEORA_ERR_UNSUPPORTED_SHAPE and launches nothing;
+ *     larger problems need meteora_lora_delta and a workspace.
+ *   - The first call on each device looks up the device address of the built-in array (a runtime query,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left in it.  No
+ *     part of it needs clearing (every value is written before it is read within a call), but two calls
+ *     whose kernels can overlap on the GPU (different streams, no ordering between them) race on it: keep
+ *     calls on one device ordered.
+ */
+int meteora_lora_delta_static(const void* x, const void* A, const void* B, const int32_t* topk_idx,
+                              const float* topk_w, const int32_t* offsets, const int32_t* perm,
+                              const meteora_shape_t* shape, float* delta, void* stream);
 
 /*
  * The whole layer, Eq. 2 with Eq. 3: gate, top-k, softmax over the selected, base product,

@@ -22,7 +22,8 @@ STATUS = {0: "METEORA_OK", -1: "METEORA_ERR_INVALID_ARG", -2: "METEORA_ERR_UNSUP
           -3: "METEORA_ERR_MISALIGNED", -4: "METEORA_ERR_WORKSPACE_TOO_SMALL", -5: "METEORA_ERR_CUDA",
           -6: "METEORA_ERR_TIMEOUT"}
 
-EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_linear_forward",
+EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_lora_delta_static",
+           "meteora_linear_forward",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
            "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
            "meteora_set_tuning", "meteora_status_string"]
@@ -56,6 +57,7 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_gate_topk.argtypes = [vp, vp, shp, vp, vp, vp, vp]
     lib.meteora_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
     lib.meteora_lora_delta.argtypes = [vp, vp, vp, vp, vp, vp, vp, shp, vp, vp, sz, vp]
+    lib.meteora_lora_delta_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, shp, vp, vp]
     lib.meteora_linear_forward.argtypes = [vp, vp, vp, vp, vp, shp, vp, vp, sz, vp]
     lib.meteora_linear_forward_host.argtypes = [vp, vp, vp, vp, vp, shp, vp, vp, sz, vp]
     lib.meteora_workspace_bytes.argtypes = [shp]
@@ -165,6 +167,34 @@ def meteora_lora_delta(x, A, B, topk_idx, topk_w, offsets, perm, workspace: Opti
                                   _dev(perm, (T * k,), torch.int32, "perm"), ctypes.byref(shape),
                                   delta.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
            "meteora_lora_delta")
+    return delta
+
+
+STATIC_SCRATCH_FLOATS = 65536
+
+
+def meteora_lora_delta_static(x, A, B, topk_idx, topk_w, offsets, perm, out: Optional[torch.Tensor] = None
+                              ) -> torch.Tensor:
+    """meteora_lora_delta for callers that cannot allocate: the library's built-in 256 KB device array replaces
+    the workspace, so T*k*r must not exceed STATIC_SCRATCH_FLOATS (MeteoraError -2 otherwise).  Pass `out`
+    (fp32 [T,d_out]) to keep this wrapper from allocating the result as well.  Calls on one device share
+    the array: keep them ordered on the GPU.  Make the first call on a device outside stream capture."""
+    lib = load_library()
+    T, d_in = x.shape
+    N, r, _ = A.shape
+    d_out = B.shape[1]
+    k = topk_idx.shape[1]
+    shape = make_shape(T, d_in, d_out, N, r, k, x.dtype)
+    _dtype_code(x)
+    delta = out if out is not None else torch.empty((T, d_out), dtype=torch.float32, device=x.device)
+    _check(lib.meteora_lora_delta_static(_dev(x, (T, d_in), x.dtype, "x"), _dev(A, (N, r, d_in), x.dtype, "A"),
+                                         _dev(B, (N, d_out, r), x.dtype, "B"),
+                                         _dev(topk_idx, (T, k), torch.int32, "topk_idx"),
+                                         _dev(topk_w, (T, k), torch.float32, "topk_w"),
+                                         _dev(offsets, (N + 1,), torch.int32, "offsets"),
+                                         _dev(perm, (T * k,), torch.int32, "perm"), ctypes.byref(shape),
+                                         _dev(delta, (T, d_out), torch.float32, "delta"), _stream()),
+           "meteora_lora_delta_static")
     return delta
 
 
