@@ -189,7 +189,7 @@ int meteora_profile_end(float* total_ms, int* launches);
 /*
  * Tuning knobs for measurements (process-wide, not thread-safe): "splits" (split-K cluster size,
  * 0 = automatic), "stages" (TMA ring depth, 0 = automatic), "tile_tokens" (tokens per tile, 0 =
- * automatic), "force_simt" (1 = never take the tensor-core path), "pdl" (1 = overlap the chained
+ * automatic), "kc" (64-element k-chunks fetched per TMA copy: 1, 2 or 4; 0 = automatic), "force_simt" (1 = never take the tensor-core path), "pdl" (1 = overlap the chained
  * kernels of a call by programmatic dependent launch).  Unknown names return
  * METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
  */

@@ -65,6 +65,7 @@ struct Tuning {
     int splits = 0;
     int stages = 0;
     int tile_tokens = 0;
+    int kc = 0;
     int force_simt = 0;
     int pdl = 1;
 };

@@ -44,6 +44,8 @@ struct WGemmParams {
     size_t u_all_zstride;   // floats between the u_all copies
     int ksteps;          // ceil(K / kBK)
     int stages;          // depth of the TMA ring
+    int kc;              // k-steps (64-element chunks) per stage; > 1 only with the 3-D tensor maps
+    int maps3d;          // tensor maps are (64, rows, K/64) views: one TMA instruction fetches kc chunks
     int tmem_cols;       // power of two >= max(32, BN)
     int split_tile;      // row tiles >= split_tile read tensor map 1 (their rows restart at 0)
     int rows0, rows1;    // valid rows under tensor map 0 / 1
@@ -99,6 +101,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -320,7 +328,8 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;                 // 1024-byte aligned for the 128-byte swizzle
     uint8_t* ring_ptr = smem_raw + (ring - raw);
-    const uint32_t stage_bytes = kWTileBytes + p.BN * 128;
+    const uint32_t x_tile_bytes = p.BN * 128;
+    const uint32_t stage_bytes = p.kc * (kWTileBytes + x_tile_bytes);   // [kc W tiles][kc x tiles]
     const uint32_t ring_bytes = p.stages * stage_bytes;
     const uint32_t bar_base = ring + ring_bytes;                 // full[stages], empty[stages], acc (8 bytes each)
     const uint32_t bar_acc = bar_base + 2 * p.stages * 8;
@@ -339,6 +348,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const int ks0 = kz0 + (int)(((long long)(kz1 - kz0) * split) / S);
     const int ks1 = kz0 + (int)(((long long)(kz1 - kz0) * (split + 1)) / S);
     const int nks = ks1 - ks0;
+    const int niter = nks / p.kc;             // the host picks kc so that it divides every CTA's k-step count
 
     if (p.pdl_trigger && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -370,15 +380,21 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
             const int row0 = (second ? tile_m - p.split_tile : tile_m) * kBM;
             int issued = 0;
             bool ok = true;
-            for (int i = 0; i < nks; ++i) {
+            for (int i = 0; i < niter; ++i) {
                 const int s = i % p.stages, round = i / p.stages;
                 if (round > 0) ok = mbar_wait(bar_base + (p.stages + s) * 8, (round & 1) ^ 1);
                 if (!ok) break;
                 const uint32_t full = bar_base + s * 8;
                 const uint32_t dst = ring + s * stage_bytes;
+                const int kstep = ks0 + i * p.kc;
                 mbar_expect_tx(full, stage_bytes);
-                tma_load_2d(dst, tmW, (ks0 + i) * kBK, row0, full);
-                tma_load_2d(dst + kWTileBytes, &tmX, (ks0 + i) * kBK, tok0, full);
+                if (p.maps3d) {      // one instruction per operand brings kc consecutive 64-element chunks
+                    tma_load_3d(dst, tmW, 0, row0, kstep, full);
+                    tma_load_3d(dst + p.kc * kWTileBytes, &tmX, 0, tok0, kstep, full);
+                } else {
+                    tma_load_2d(dst, tmW, kstep * kBK, row0, full);
+                    tma_load_2d(dst + kWTileBytes, &tmX, kstep * kBK, tok0, full);
+                }
                 issued = i + 1;
             }
             if (!ok) {
@@ -391,16 +407,19 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(p.BN);
             bool ok = true;
-            for (int i = 0; i < nks; ++i) {
+            for (int i = 0; i < niter; ++i) {
                 const int s = i % p.stages, round = i / p.stages;
                 ok = mbar_wait(bar_base + s * 8, round & 1);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t wa = ring + s * stage_bytes;
-                const uint64_t da = smem_desc_sw128(wa), db = smem_desc_sw128(wa + kWTileBytes);
+                const uint32_t wa = ring + s * stage_bytes, xa = wa + p.kc * kWTileBytes;
+                for (int c = 0; c < p.kc; ++c) {
+                    const uint64_t da = smem_desc_sw128(wa + c * kWTileBytes);
+                    const uint64_t db = smem_desc_sw128(xa + c * x_tile_bytes);
 #pragma unroll
-                for (int kk = 0; kk < kBK / kUmmaK; ++kk)
-                    umma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (i | kk) != 0);
+                    for (int kk = 0; kk < kBK / kUmmaK; ++kk)
+                        umma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (i | c | kk) != 0);
+                }
                 umma_commit(bar_base + (p.stages + s) * 8);   // stage reusable once these MMAs have read it
             }
             umma_commit(bar_acc);                              // accumulators complete
@@ -489,9 +508,9 @@ static EncodeTiledFn encode_fn() {
 
 struct MapKey {
     const void* ptr;
-    int K, rows, box_rows;
+    int K, rows, box_rows, depth;   // depth 0: 2-D map; depth >= 1: 3-D map whose box holds `depth` chunks
     bool operator==(const MapKey& o) const {
-        return ptr == o.ptr && K == o.K && rows == o.rows && box_rows == o.box_rows;
+        return ptr == o.ptr && K == o.K && rows == o.rows && box_rows == o.box_rows && depth == o.depth;
     }
 };
 struct MapEntry {
@@ -499,13 +518,17 @@ struct MapEntry {
     CUtensorMap map;
 };
 
-// A [rows, K] row-major bf16 matrix as a 2-D tensor map whose box is kBK (128 bytes) x box_rows, 128-byte
-// swizzled; out-of-range rows and columns read as zero.  Encoded maps are cached by (pointer, shape).
-static int get_tensor_map(const void* ptr, int K, int rows, int box_rows, CUtensorMap* out) {
+// Tensor map of a [rows, K] row-major bf16 matrix, 128-byte swizzled, out-of-range elements read as zero.
+//   depth == 0: 2-D (K, rows), box = 64 elements (128 bytes) x box_rows.
+//   depth >= 1: 3-D view (64, rows, K/64) with strides (K*2, 128) bytes, box = 64 x box_rows x depth, so a
+//               single copy lands `depth` consecutive k-chunks as `depth` consecutive [box_rows][128 B]
+//               tiles.  Needs K % 64 == 0 (a ragged last chunk would run into the next row).
+// Encoded maps are cached by (pointer, shape).
+static int get_tensor_map(const void* ptr, int K, int rows, int box_rows, int depth, CUtensorMap* out) {
     static std::mutex mu;
     static std::vector<MapEntry> cache;
     static size_t next_evict = 0;
-    const MapKey key{ptr, K, rows, box_rows};
+    const MapKey key{ptr, K, rows, box_rows, depth};
     std::lock_guard<std::mutex> lock(mu);
     for (const MapEntry& e : cache)
         if (e.key == key) {
@@ -514,15 +537,26 @@ static int get_tensor_map(const void* ptr, int K, int rows, int box_rows, CUtens
         }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return METEORA_ERR_CUDA;
-    const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    const cuuint64_t gstride[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
-    const cuuint32_t estride[2] = {1, 1};
     MapEntry e;
     e.key = key;
-    const CUresult r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box,
-                          estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r;
+    if (depth == 0) {
+        const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+        const cuuint64_t gstride[1] = {(cuuint64_t)K * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+        const cuuint32_t estride[2] = {1, 1};
+        r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t gdim[3] = {(cuuint64_t)kBK, (cuuint64_t)rows, (cuuint64_t)(K / kBK)};
+        const cuuint64_t gstride[2] = {(cuuint64_t)K * 2, (cuuint64_t)kBK * 2};
+        const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)box_rows, (cuuint32_t)depth};
+        const cuuint32_t estride[3] = {1, 1, 1};
+        r = fn(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) return METEORA_ERR_CUDA;
     if (cache.size() < 256) {
         cache.push_back(e);
@@ -558,7 +592,7 @@ struct Plan;
 static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k);
 
 struct Plan {
-    int BN, n_tiles, splits, zsplits, stages, tmem_cols;
+    int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
     int epi_off, uw_off, slab_off, slab_q, per_slot;
     size_t smem;
 };
@@ -607,16 +641,33 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
         pl.slab_q = slab_bytes <= 64 * 1024 ? q : 0;
         epi_bytes = pl.slab_off + (pl.slab_q > 0 ? slab_bytes : 0);
     }
-    const size_t stage_bytes = kWTileBytes + (size_t)bn * 128;
+    const size_t chunk_bytes = kWTileBytes + (size_t)bn * 128;   // one k-step of both operands
     const size_t part_bytes = (size_t)bn * kBM * 4;           // accumulators parked in the idle ring
     const size_t fixed = 1024 + 256 + epi_bytes;               // alignment slack + barriers + staging
-    const int nks = ksteps_cta + 1;
+    const size_t avail = total_budget > fixed ? total_budget - fixed : 0;
+    // k-steps per stage: issuing a TMA copy costs about as much as moving 16 KB, so with the 3-D maps one
+    // instruction per operand fetches up to 4 consecutive k-steps, as long as that count divides every
+    // CTA's share of the contraction axis and at least three stages still fit.
+    pl.maps3d = (K % kBK) == 0 ? 1 : 0;
+    int kc = 1;
+    const int parts = splits * pl.zsplits;
+    if (pl.maps3d && ksteps % parts == 0) {
+        const int per = ksteps / parts;
+        for (int cand = 4; cand > 1; cand /= 2)
+            if (per % cand == 0 && 3 * cand * chunk_bytes <= avail) {
+                kc = cand;
+                break;
+            }
+        if (tn.kc > 0 && per % tn.kc == 0) kc = tn.kc;
+    }
+    pl.kc = kc;
+    const size_t stage_bytes = kc * chunk_bytes;
+    const int niter = (ksteps_cta + kc - 1) / kc + 1;
     int stages;
     if (tn.stages > 0) {
         stages = tn.stages;
     } else {
-        const size_t avail = total_budget > fixed ? total_budget - fixed : 0;
-        stages = (int)std::min<size_t>((size_t)nks, avail / stage_bytes);
+        stages = (int)std::min<size_t>((size_t)niter, avail / stage_bytes);
     }
     stages = std::max(stages, 2);
     while ((size_t)stages * stage_bytes < part_bytes) ++stages;
@@ -677,6 +728,8 @@ static void fill_common(WGemmParams& p, const Plan& pl, int T, int K, int32_t* s
     p.zsplits = pl.zsplits;
     p.ksteps = (K + kBK - 1) / kBK;
     p.stages = pl.stages;
+    p.kc = pl.kc;
+    p.maps3d = pl.maps3d;
     p.tmem_cols = pl.tmem_cols;
     p.epi_off = pl.epi_off;
     p.uw_off = pl.uw_off;
@@ -694,9 +747,9 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, false, s.N, s.r, s.k);
     CUtensorMap mA, mG, mX;
     int rc;
-    if ((rc = get_tensor_map(A, s.d_in, a_rows, kBM, &mA)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(Wg, s.d_in, s.N, kBM, &mG)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, a_rows, kBM, pl.maps3d ? pl.kc : 0, &mA)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Wg, s.d_in, s.N, kBM, pl.maps3d ? pl.kc : 0, &mG)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, pl.maps3d ? pl.kc : 0, &mX)) != METEORA_OK) return rc;
     WGemmParams p = {};
     fill_common(p, pl, s.T, s.d_in, ws.status);
     p.split_tile = a_tiles;
@@ -718,8 +771,8 @@ int launch_base_lora_tc(const void* x, const void* W0, const void* B, const mete
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     CUtensorMap mW, mX;
     int rc;
-    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, &mW)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, pl.maps3d ? pl.kc : 0, &mW)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, pl.maps3d ? pl.kc : 0, &mX)) != METEORA_OK) return rc;
     WGemmParams p = {};
     fill_common(p, pl, s.T, s.d_in, ws.status);
     p.split_tile = 0x7FFFFFFF;
