@@ -195,42 +195,74 @@ __device__ __forceinline__ void fma8(const uint4& b, const float4& u0, const flo
     acc = fmaf(__uint_as_float(b.w & 0xFFFF0000u), u1.w, acc);
 }
 
-// Stage s_e, s_uw and the B slab of rows [row0, row0 + nrows) (epilogue threads only).
+// Stage s_e, s_uw and the B slab of rows [row0, row0 + nrows) (epilogue threads only).  All global loads of
+// a batch are issued before any shared-memory store, so the arrays cost one memory round trip together
+// instead of one each (the loads queue behind the W0 stream and see microseconds of latency).
 __device__ __forceinline__ void stage_lora_operands(const WGemmParams& p, uint8_t* epi, int tok0, int ntok, int row0,
                                                     int nrows, int etid) {
     int* s_e = reinterpret_cast<int*>(epi);
     float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off);
     uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
     const int slots = ntok * p.k;
-    for (int i = etid; i < slots; i += kEpiThreads)
-        s_e[i] = min(max(__ldg(p.topk_idx + (size_t)tok0 * p.k + i), 0), p.N - 1);
+    const int n4 = slots * p.r / 4;
     const float4* uw4 = reinterpret_cast<const float4*>(p.uw + (size_t)tok0 * p.k * p.r);
-    for (int i = etid; i < slots * p.r / 4; i += kEpiThreads) s_uw4[i] = __ldg(uw4 + i);
-    if (p.slab_q > 0) {
-        const int vpr = p.r >> 3;                      // 16-byte vectors per B row
-        const int vpe = nrows * vpr;                   // vectors per slab entry
-        const int nq = p.per_slot ? slots : p.N;
-        const int total = nq * vpe;
-        const uint4* Bv = reinterpret_cast<const uint4*>(p.B);
-        constexpr int U = 4;                           // independent loads in flight per thread
-        for (int v0 = etid; v0 < total; v0 += U * kEpiThreads) {
-            uint4 val[U];
+    const int32_t* idx = p.topk_idx + (size_t)tok0 * p.k;
+    const int vpr = p.r >> 3;                      // 16-byte vectors per B row
+    const int vpe = nrows * vpr;                   // vectors per slab entry
+    const int nq = p.per_slot ? slots : p.N;
+    const int total = p.slab_q > 0 ? nq * vpe : 0;
+    const uint4* Bv = reinterpret_cast<const uint4*>(p.B);
+    constexpr int UE = 2, UU = 4, UB = 4;
+    int e_reg[UE];
+    float4 u_reg[UU];
+    uint4 b_reg[UB];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int v = v0 + u * kEpiThreads;
-                val[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (v < total) {
-                    const int q = v / vpe, w = v - q * vpe;
-                    const int rr = w / vpr;
-                    const int e = p.per_slot ? min(max(__ldg(p.topk_idx + (size_t)tok0 * p.k + q), 0), p.N - 1) : q;
-                    if (row0 + rr < p.d_out) val[u] = __ldg(Bv + ((size_t)e * p.d_out + row0) * vpr + w);
-                }
-            }
+    for (int u = 0; u < UE; ++u) {
+        const int i = etid + u * kEpiThreads;
+        e_reg[u] = i < slots ? __ldg(idx + i) : 0;
+    }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int v = v0 + u * kEpiThreads;
-                if (v < total) slab[v] = val[u];
-            }
+    for (int u = 0; u < UU; ++u) {
+        const int i = etid + u * kEpiThreads;
+        u_reg[u] = i < n4 ? __ldg(uw4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    auto load_b = [&](int v) {
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (v < total) {
+            const int q = v / vpe, w = v - q * vpe;
+            const int rr = w / vpr;
+            const int e = p.per_slot ? min(max(__ldg(idx + q), 0), p.N - 1) : q;
+            if (row0 + rr < p.d_out) val = __ldg(Bv + ((size_t)e * p.d_out + row0) * vpr + w);
+        }
+        return val;
+    };
+#pragma unroll
+    for (int u = 0; u < UB; ++u) b_reg[u] = load_b(etid + u * kEpiThreads);
+#pragma unroll
+    for (int u = 0; u < UE; ++u) {
+        const int i = etid + u * kEpiThreads;
+        if (i < slots) s_e[i] = min(max(e_reg[u], 0), p.N - 1);
+    }
+#pragma unroll
+    for (int u = 0; u < UU; ++u) {
+        const int i = etid + u * kEpiThreads;
+        if (i < n4) s_uw4[i] = u_reg[u];
+    }
+#pragma unroll
+    for (int u = 0; u < UB; ++u) {
+        const int v = etid + u * kEpiThreads;
+        if (v < total) slab[v] = b_reg[u];
+    }
+    // whatever did not fit into the first batch
+    for (int i = etid + UE * kEpiThreads; i < slots; i += kEpiThreads) s_e[i] = min(max(__ldg(idx + i), 0), p.N - 1);
+    for (int i = etid + UU * kEpiThreads; i < n4; i += kEpiThreads) s_uw4[i] = __ldg(uw4 + i);
+    for (int v0 = etid + UB * kEpiThreads; v0 < total; v0 += UB * kEpiThreads) {
+#pragma unroll
+        for (int u = 0; u < UB; ++u) b_reg[u] = load_b(v0 + u * kEpiThreads);
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            const int v = v0 + u * kEpiThreads;
+            if (v < total) slab[v] = b_reg[u];
         }
     }
 }
@@ -293,7 +325,7 @@ __device__ __forceinline__ void reduce_and_finish(const WGemmParams& p, uint32_t
     constexpr int P = 64 / S;                 // row pairs of this CTA's slice
     constexpr int TPP = kEpiThreads / P;      // tokens handled per pass of the epilogue threads
     constexpr int NROWS = kBM / S;
-    constexpr int U = S >= 4 ? 2 : 4;         // tokens in flight per thread
+    constexpr int U = S >= 8 ? 4 : 8;         // tokens in flight per thread: their partial loads go out together
     const int pr = etid % P, tg = etid / P;
     const int row_in_tile = NROWS * split + 2 * pr;
 
