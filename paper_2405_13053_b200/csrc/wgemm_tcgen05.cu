@@ -36,6 +36,21 @@ constexpr int kMaxZSplits = 4;
 
 enum { MODE_STACKED = 0, MODE_LORA = 1 };
 
+// Optional device timeline for tuning: built with -DMETEORA_TRACE, CTA 0 of a base-product launch writes the
+// low 31 bits of %globaltimer (ns) into status words 32 + slot at a few points.  Compiled out otherwise.
+#ifdef METEORA_TRACE
+#define METEORA_STAMP(p, slot)                                                      \
+    do {                                                                            \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && (p).mode == MODE_LORA) {          \
+            unsigned long long t_;                                                  \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                  \
+            (p).status[32 + (slot)] = (int)(t_ & 0x7FFFFFFF);                       \
+        }                                                                           \
+    } while (0)
+#else
+#define METEORA_STAMP(p, slot) do { } while (0)
+#endif
+
 struct WGemmParams {
     int T, K;            // tokens, contraction length
     int BN;              // tokens per tile (multiple of 16, <= 256)
@@ -383,6 +398,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const int niter = nks / p.kc;             // the host picks kc so that it divides every CTA's k-step count
 
     if (p.pdl_trigger && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 0) METEORA_STAMP(p, 0);      // start
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -455,6 +471,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
                 umma_commit(bar_base + (p.stages + s) * 8);   // stage reusable once these MMAs have read it
             }
             umma_commit(bar_acc);                              // accumulators complete
+            METEORA_STAMP(p, 1);                                // all MMAs issued
             if (!ok) {
                 atomicExch(p.status, 1);
                 atomicExch(p.status + 2, 200);
@@ -467,6 +484,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         if (p.pdl_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (p.mode == MODE_LORA)
             stage_lora_operands(p, epi, tok0, ntok, tile_m * kBM + (kBM / S) * split, kBM / S, etid);
+        if (etid == 0) METEORA_STAMP(p, 2);                     // LoRA operands staged
         bool acc_ok = true;
         if (nks > 0) {
             acc_ok = mbar_wait(bar_acc, 0);
@@ -476,6 +494,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
             }
         }
         acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);   // keep the warp-collective TMEM loads convergent
+        if (etid == 0) METEORA_STAMP(p, 3);                     // accumulators ready
         tc_fence_after();
         // Park the accumulators in the ring, which is idle now: every load has landed and every MMA that
         // read it has completed.
@@ -495,8 +514,10 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
             for (int i = 0; i < 16; ++i) part[(c + i) * kBM + row_in_tile] = v[i];
         }
     }
+    if (threadIdx.x == 64) METEORA_STAMP(p, 4);                 // accumulators parked
     __syncwarp();
     if (S > 1) cluster_sync(); else __syncthreads();
+    if (threadIdx.x == 64) METEORA_STAMP(p, 5);                 // partials of the cluster visible
 
     if (warp >= 2) {
         const int etid = threadIdx.x - 64;
@@ -507,8 +528,10 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
             default: reduce_and_finish<8>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
         }
     }
+    if (threadIdx.x == 64) METEORA_STAMP(p, 6);                 // this thread's outputs stored
     __syncwarp();
     if (S > 1) cluster_sync();   // nobody leaves while a peer may still read its partials
+    if (threadIdx.x == 64) METEORA_STAMP(p, 7);
 
     tc_fence_before();
     __syncthreads();
