@@ -66,6 +66,7 @@ struct Tuning {
     int stages = 0;
     int tile_tokens = 0;
     int kc = 0;
+    int simt_expand = 0;   // 1: keep the LoRA expand on CUDA cores even for rank 8
     int force_simt = 0;
     int pdl = 1;
 };

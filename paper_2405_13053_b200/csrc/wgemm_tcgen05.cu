@@ -76,6 +76,12 @@ struct WGemmParams {
     int uw_off, slab_off;   // byte offsets of s_uw and the B slab inside that area
     int slab_q;          // slab entries held in shared memory (0: read B from global memory)
     int per_slot;        // slab indexed by slot t*k+j instead of by adapter
+    // LoRA expand on the tensor cores (rank 8): CTA `split` of a tile owns adapters [split*na, split*na + na)
+    // and adds  sum_e B_e[rows, :] . U_e[:, tokens]  to its accumulator with na/2 extra MMAs.
+    int lora_mma;        // 1: the expand runs as MMAs, the epilogue only reduces and stores
+    int na;              // adapters per split, even (two 8-wide adapters per K = 16 MMA)
+    int us_in_ring;      // the token-side operand is too big for the staging area: build it in the idle ring
+    int us_off;          // byte offset of the token-side operand inside the staging area (slab at slab_off)
     int32_t* status;
     int pdl_wait;        // epilogue waits for the preceding grid before reading its results
     int pdl_trigger;     // let the dependent grid start as soon as this one is resident
@@ -167,6 +173,16 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     d |= (uint64_t)(1024 >> 4) << 32;
     d |= (uint64_t)1 << 46;
     d |= (uint64_t)2 << 61;
+    return d;
+}
+// Shared-memory matrix descriptor of an un-swizzled K-major bf16 operand made of 8-row x 16-byte core
+// matrices (128 contiguous bytes each): kstride = bytes between core matrices adjacent along K (leading
+// byte offset), mnstride = bytes between core matrices adjacent along M/N (stride byte offset).
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t kstride, uint32_t mnstride) {
+    uint64_t d = (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((kstride >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((mnstride >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
     return d;
 }
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, M = 128, N = bn.
@@ -282,6 +298,59 @@ __device__ __forceinline__ void stage_lora_operands(const WGemmParams& p, uint8_
     }
 }
 
+// Operands of the tensor-core expand (rank 8), both K-major without swizzle, K = adapter-major (8 elements
+// = 16 bytes per adapter):
+//   slab[a][row 0..127][8]   = B[a0 + a][tile rows]  -- in global memory the 8 rows x 16 bytes of a core
+//                              matrix are already 128 contiguous bytes, so this is a plain copy;
+//   us[a][t 0..BN)[8]        = bf16(w_j * A_e x_t) if token t picked adapter e = a0 + a at rank j, else 0.
+__device__ __forceinline__ void stage_slab_mma(const WGemmParams& p, uint8_t* epi, int a0, int tile_row0, int etid) {
+    uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
+    const uint4* Bv = reinterpret_cast<const uint4*>(p.B);
+    const int total = p.na * kBM;
+    constexpr int U = 4;
+    for (int v0 = etid; v0 < total; v0 += U * kEpiThreads) {
+        uint4 val[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int v = v0 + u * kEpiThreads;
+            const int a = v / kBM, row = v - a * kBM;
+            val[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (v < total && a0 + a < p.N && tile_row0 + row < p.d_out)
+                val[u] = __ldg(Bv + (size_t)(a0 + a) * p.d_out + tile_row0 + row);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int v = v0 + u * kEpiThreads;
+            if (v < total) slab[v] = val[u];
+        }
+    }
+}
+
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+__device__ __forceinline__ void stage_us_mma(const WGemmParams& p, uint4* us, int a0, int tok0, int ntok, int etid) {
+    const int total = p.na * p.BN;
+    for (int v = etid; v < total; v += kEpiThreads) us[v] = make_uint4(0u, 0u, 0u, 0u);
+    epi_barrier();
+    const int slots = ntok * p.k;
+    const int32_t* idx = p.topk_idx + (size_t)tok0 * p.k;
+    const float4* uw4 = reinterpret_cast<const float4*>(p.uw + (size_t)tok0 * p.k * 8);
+    for (int i = etid; i < slots; i += kEpiThreads) {
+        const int a = __ldg(idx + i) - a0;
+        if (a >= 0 && a < p.na) {
+            const float4 lo = __ldg(uw4 + 2 * i), hi = __ldg(uw4 + 2 * i + 1);
+            const __nv_bfloat162 q0 = __floats2bfloat162_rn(lo.x, lo.y), q1 = __floats2bfloat162_rn(lo.z, lo.w);
+            const __nv_bfloat162 q2 = __floats2bfloat162_rn(hi.x, hi.y), q3 = __floats2bfloat162_rn(hi.z, hi.w);
+            uint4 val;
+            val.x = *reinterpret_cast<const uint32_t*>(&q0);
+            val.y = *reinterpret_cast<const uint32_t*>(&q1);
+            val.z = *reinterpret_cast<const uint32_t*>(&q2);
+            val.w = *reinterpret_cast<const uint32_t*>(&q3);
+            us[a * p.BN + i / p.k] = val;
+        }
+    }
+}
+
 // One (row pair, token) result: add the LoRA expand and store.
 __device__ __forceinline__ void finish_pair(const WGemmParams& p, const uint8_t* epi, int tile_m, int row_in_tile,
                                             int nrows, int pr, int t, int token, float a0, float a1) {
@@ -305,7 +374,7 @@ __device__ __forceinline__ void finish_pair(const WGemmParams& p, const uint8_t*
     const uint4* slab = reinterpret_cast<const uint4*>(epi + p.slab_off);
     const int vpr = p.r >> 3;
     const int o = tile_m * kBM + row_in_tile;
-    for (int j = 0; j < p.k; ++j) {
+    for (int j = 0; j < (p.lora_mma ? 0 : p.k); ++j) {
         const int slot = t * p.k + j;
         const int e = s_e[slot];
         for (int c = 0; c < vpr; ++c) {
@@ -379,8 +448,10 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const uint32_t stage_bytes = p.kc * (kWTileBytes + x_tile_bytes);   // [kc W tiles][kc x tiles]
     const uint32_t ring_bytes = p.stages * stage_bytes;
     const uint32_t bar_base = ring + ring_bytes;                 // full[stages], empty[stages], acc (8 bytes each)
-    const uint32_t bar_acc = bar_base + 2 * p.stages * 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + (2 * p.stages + 1) * 8);
+    const uint32_t bar_acc = bar_base + 2 * p.stages * 8;       // accumulators complete
+    const uint32_t bar_main = bar_acc + 8;                      // main-loop MMAs complete: the ring is idle
+    const uint32_t bar_us = bar_acc + 16;                       // operands of the tensor-core expand are staged
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + (2 * p.stages + 3) * 8);
     uint8_t* epi = ring_ptr + ring_bytes + p.epi_off;             // staging of the LoRA operands
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -406,6 +477,8 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
             mbar_init(bar_base + (p.stages + s) * 8, 1);
         }
         mbar_init(bar_acc, 1);
+        mbar_init(bar_main, 1);
+        mbar_init(bar_us, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -470,6 +543,20 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
                 }
                 umma_commit(bar_base + (p.stages + s) * 8);   // stage reusable once these MMAs have read it
             }
+            if (p.lora_mma && ok) {
+                // LoRA expand as a K extension of the same accumulation: na/2 MMAs of K = 16 (two adapters)
+                umma_commit(bar_main);
+                ok = mbar_wait(bar_us, 0);
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t slab_a = smem_u32(epi + p.slab_off);
+                    const uint32_t us_a = p.us_in_ring ? ring : smem_u32(epi + p.us_off);
+                    const uint32_t ka = kBM * 16, kb = p.BN * 16;      // bytes from one adapter to the next
+                    for (int m = 0; m < p.na / 2; ++m)
+                        umma_bf16(tmem_base, smem_desc_plain(slab_a + 2 * m * ka, ka, 128),
+                                  smem_desc_plain(us_a + 2 * m * kb, kb, 128), idesc, (niter | m) != 0);
+                }
+            }
             umma_commit(bar_acc);                              // accumulators complete
             METEORA_STAMP(p, 1);                                // all MMAs issued
             if (!ok) {
@@ -482,11 +569,28 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         const int quad = warp & 3;                    // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
         const int etid = threadIdx.x - 64;
         if (p.pdl_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (p.mode == MODE_LORA)
+        if (p.mode == MODE_LORA && p.lora_mma) {
+            const int a0 = split * p.na;
+            stage_slab_mma(p, epi, a0, tile_m * kBM, etid);
+            bool ring_ok = true;
+            if (p.us_in_ring) {                                 // the token-side operand goes where the ring was
+                ring_ok = mbar_wait(bar_main, 0);
+                if (!ring_ok && lane == 0) {
+                    atomicExch(p.status, 1);
+                    atomicExch(p.status + 4, 350);
+                }
+            }
+            uint4* us = reinterpret_cast<uint4*>(p.us_in_ring ? ring_ptr : epi + p.us_off);
+            stage_us_mma(p, us, a0, tok0, ntok, etid);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+            epi_barrier();
+            if (etid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_us) : "memory");
+        } else if (p.mode == MODE_LORA) {
             stage_lora_operands(p, epi, tok0, ntok, tile_m * kBM + (kBM / S) * split, kBM / S, etid);
+        }
         if (etid == 0) METEORA_STAMP(p, 2);                     // LoRA operands staged
         bool acc_ok = true;
-        if (nks > 0) {
+        if (nks > 0 || p.lora_mma) {
             acc_ok = mbar_wait(bar_acc, 0);
             if (!acc_ok && lane == 0) {
                 atomicExch(p.status, 1);
@@ -504,7 +608,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
         for (int c = c_begin; c < c_end; c += 16) {
             float v[16];
-            if (nks > 0 && acc_ok) {
+            if ((nks > 0 || p.lora_mma) && acc_ok) {
                 tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
             } else {
 #pragma unroll
@@ -648,7 +752,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
 
 struct Plan {
     int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
-    int epi_off, uw_off, slab_off, slab_q, per_slot;
+    int epi_off, uw_off, slab_off, slab_q, per_slot, lora_mma, na, us_in_ring, us_off;
     size_t smem;
 };
 
@@ -687,7 +791,19 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
     const int tile_tokens = std::min(T, bn);
     size_t epi_bytes = 0;
-    if (lora) {
+    size_t us_bytes = 0;
+    if (lora && r == 8 && !tn.simt_expand) {
+        // expand on the tensor cores: B rows of this split's adapters for all 128 rows, and the masked,
+        // gate-weighted shrink outputs of the tile's tokens as the other operand
+        pl.lora_mma = 1;
+        pl.na = ((N + splits - 1) / splits + 1) / 2 * 2;
+        pl.slab_off = 0;
+        const size_t slab_bytes = (size_t)pl.na * kBM * 16;
+        us_bytes = (size_t)pl.na * bn * 16;
+        pl.us_in_ring = us_bytes > 32 * 1024 ? 1 : 0;
+        pl.us_off = (int)slab_bytes;
+        epi_bytes = slab_bytes + (pl.us_in_ring ? 0 : us_bytes);
+    } else if (lora) {
         pl.uw_off = (int)align_up((size_t)bn * k * 4, 16);
         pl.slab_off = pl.uw_off + bn * k * r * 4;
         pl.per_slot = tile_tokens * k <= N ? 1 : 0;
@@ -726,11 +842,13 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     }
     stages = std::max(stages, 2);
     while ((size_t)stages * stage_bytes < part_bytes) ++stages;
+    if (pl.us_in_ring)
+        while ((size_t)stages * stage_bytes < us_bytes) ++stages;
     pl.stages = stages;
     int cols = 32;
     while (cols < bn) cols *= 2;
     pl.tmem_cols = cols;
-    pl.epi_off = (int)align_up((size_t)(2 * stages + 1) * 8 + 16, 16);
+    pl.epi_off = (int)align_up((size_t)(2 * stages + 3) * 8 + 16, 128);
     pl.smem = 1024 + (size_t)stages * stage_bytes + pl.epi_off + epi_bytes;
     return pl;
 }
@@ -791,6 +909,10 @@ static void fill_common(WGemmParams& p, const Plan& pl, int T, int K, int32_t* s
     p.slab_off = pl.slab_off;
     p.slab_q = pl.slab_q;
     p.per_slot = pl.per_slot;
+    p.lora_mma = pl.lora_mma;
+    p.na = pl.na;
+    p.us_in_ring = pl.us_in_ring;
+    p.us_off = pl.us_off;
     p.status = status;
 }
 
