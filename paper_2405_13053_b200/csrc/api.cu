@@ -30,7 +30,7 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     ws.topk_idx = (int32_t*)take(T * s.k * sizeof(int32_t));
     ws.topk_w = (float*)take(T * s.k * sizeof(float));
     ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
-    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (s.T <= 256 ? 4 : 1));   // up to 4 slices for decode batches
+    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (s.T <= 256 ? 32 : 1));   // up to 32 slices for decode batches
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);
     ws.bytes = off;

@@ -32,7 +32,7 @@ constexpr int kThreads = 320;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2-9
 constexpr int kEpiThreads = 256;
 constexpr int kWTileBytes = kBM * kBK * 2;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // about a second
-constexpr int kMaxZSplits = 4;
+constexpr int kMaxZSplits = 32;
 
 enum { MODE_STACKED = 0, MODE_LORA = 1 };
 
@@ -601,11 +601,35 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         if (etid == 0) METEORA_STAMP(p, 3);                     // accumulators ready
         tc_fence_after();
         // Park the accumulators in the ring, which is idle now: every load has landed and every MMA that
-        // read it has completed.
+        // read it has completed.  (The stacked shrink without split-K stores them straight to u_all: lane =
+        // row = column of u_all, so a warp writes 128 contiguous bytes per token.)
         float* part = reinterpret_cast<float*>(ring_ptr);
         const int row_in_tile = quad * 32 + lane;
         const int half = ((p.BN / 16 + 1) / 2) * 16;            // warps 2-5 take columns [0, half), warps 6-9 the rest
         const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
+        if (p.mode == MODE_STACKED && S == 1) {
+            int row = tile_m * kBM + row_in_tile, limit = p.rows0, col = row;
+            if (tile_m >= p.split_tile) {
+                row = (tile_m - p.split_tile) * kBM + row_in_tile;
+                limit = p.rows1;
+                col = p.col1 + row;
+            }
+            float* dst = p.u_all + (size_t)blockIdx.z * p.u_all_zstride + (size_t)tok0 * p.ld_u + col;
+            for (int c = c_begin; c < c_end; c += 16) {
+                float v[16];
+                if (nks > 0 && acc_ok) {
+                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                }
+                if (row < limit) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c + i < ntok) dst[(size_t)(c + i) * p.ld_u] = v[i];
+                }
+            }
+        } else
         for (int c = c_begin; c < c_end; c += 16) {
             float v[16];
             if ((nks > 0 || p.lora_mma) && acc_ok) {
@@ -623,7 +647,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     if (S > 1) cluster_sync(); else __syncthreads();
     if (threadIdx.x == 64) METEORA_STAMP(p, 5);                 // partials of the cluster visible
 
-    if (warp >= 2) {
+    if (warp >= 2 && !(p.mode == MODE_STACKED && S == 1)) {
         const int etid = threadIdx.x - 64;
         switch (S) {
             case 1: reduce_and_finish<1>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
@@ -783,10 +807,20 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     // The stacked shrink of a decode batch has only a handful of row tiles: cut its contraction axis
     // further over grid z (every slice keeps at least two k-steps); the selection kernel adds the slices.
     pl.zsplits = 1;
-    if (!lora && pl.n_tiles == 1) pl.zsplits = std::min(kMaxZSplits, std::max(1, ksteps / splits / 2));
+    if (!lora && pl.n_tiles == 1) {
+        // decode-batch stacked shrink: every CTA takes a slice of the contraction axis of one row tile and
+        // writes its partial straight to u_all[z]; no cluster, no reduction here (the selection adds them).
+        splits = tn.splits > 0 ? splits : 1;
+        pl.splits = splits;
+        pl.zsplits = std::min(kMaxZSplits, std::max(1, ksteps / splits / 2));
+    }
     const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
-    const size_t total_budget = two_per_sm ? 112 * 1024 : 226 * 1024;
+    // Decode batches run as a chain stacked shrink -> selection -> base product overlapped by programmatic
+    // dependent launch: a base-product CTA and a shrink CTA must fit on one SM together (227 KB, 512 TMEM
+    // columns), so the shrink keeps to 60 KB and the base product to 160 KB.
+    const bool decode = pl.n_tiles == 1 && T <= 256;
+    const size_t total_budget = two_per_sm ? 112 * 1024 : decode ? (lora ? 160 * 1024 : 60 * 1024) : 226 * 1024;
 
     // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
     const int tile_tokens = std::min(T, bn);
