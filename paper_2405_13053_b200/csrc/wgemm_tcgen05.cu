@@ -818,9 +818,9 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
     // Decode batches run as a chain stacked shrink -> selection -> base product overlapped by programmatic
     // dependent launch: a base-product CTA and a shrink CTA must fit on one SM together (227 KB, 512 TMEM
-    // columns), so the shrink keeps to 60 KB and the base product to 160 KB.
+    // columns), so the shrink keeps to ~64 KB and the base product to 156 KB.
     const bool decode = pl.n_tiles == 1 && T <= 256;
-    const size_t total_budget = two_per_sm ? 112 * 1024 : decode ? (lora ? 160 * 1024 : 60 * 1024) : 226 * 1024;
+    const size_t total_budget = two_per_sm ? 112 * 1024 : decode ? (lora ? 156 * 1024 : 60 * 1024) : 226 * 1024;
 
     // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
     const int tile_tokens = std::min(T, bn);
@@ -852,14 +852,14 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     const size_t avail = total_budget > fixed ? total_budget - fixed : 0;
     // k-steps per stage: issuing a TMA copy costs about as much as moving 16 KB, so with the 3-D maps one
     // instruction per operand fetches up to 4 consecutive k-steps, as long as that count divides every
-    // CTA's share of the contraction axis and at least three stages still fit.
+    // CTA's share of the contraction axis and at least two stages still fit.
     pl.maps3d = (K % kBK) == 0 ? 1 : 0;
     int kc = 1;
     const int parts = splits * pl.zsplits;
     if (pl.maps3d && ksteps % parts == 0) {
         const int per = ksteps / parts;
         for (int cand = 4; cand > 1; cand /= 2)
-            if (per % cand == 0 && 3 * cand * chunk_bytes <= avail) {
+            if (per % cand == 0 && 2 * cand * chunk_bytes <= avail) {
                 kc = cand;
                 break;
             }
