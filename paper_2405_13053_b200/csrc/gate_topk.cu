@@ -89,6 +89,58 @@ k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits,
     const int t = blockIdx.x * kGateWarps + (threadIdx.x >> 5);
     if (t >= T) return;
     const float* row = u_all + (size_t)t * ld_u;
+    if (zsplits > 1 && zsplits <= 32 && r == 8 && k <= 4) {
+        // Many partial copies: lane z reads slice z, so all loads of a phase are in flight at once (one
+        // memory round trip instead of one per slice); the slices are then added across lanes by a
+        // butterfly, the same order for every token and every run.
+        const float* mine = row + (size_t)min(lane, zsplits - 1) * zstride;
+        const bool live = lane < zsplits;
+        float v0 = 0.f, v1 = 0.f;
+        for (int n0 = 0; n0 < N; n0 += 32) {
+            float vals[32];
+#pragma unroll
+            for (int n = 0; n < 32; ++n) vals[n] = (live && n0 + n < N) ? mine[col_logits + n0 + n] : 0.f;
+#pragma unroll
+            for (int n = 0; n < 32; ++n) {
+                if (n0 + n < N) {                       // uniform across the warp
+                    const float sum = warp_sum(vals[n]);
+                    if (lane == n) { if (n0 == 0) v0 = sum; else v1 = sum; }
+                }
+            }
+        }
+        int idx;
+        float w;
+        warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+        if (lane < k) {
+            topk_idx[(size_t)t * k + lane] = idx;
+            topk_w[(size_t)t * k + lane] = w;
+        }
+        float4 part[4][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
+            const float4* src = reinterpret_cast<const float4*>(mine + ij * 8);
+            const bool on = live && j < k;
+            part[j][0] = on ? src[0] : make_float4(0.f, 0.f, 0.f, 0.f);
+            part[j][1] = on ? src[1] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float out = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (j < k) {                                // uniform across the warp
+                const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
+                const float e[8] = {part[j][0].x, part[j][0].y, part[j][0].z, part[j][0].w,
+                                    part[j][1].x, part[j][1].y, part[j][1].z, part[j][1].w};
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float sum = warp_sum(e[q]);
+                    if (lane == j * 8 + q) out = wj * sum;
+                }
+            }
+        }
+        if (lane < k * 8) uw[(size_t)t * k * 8 + lane] = out;
+        return;
+    }
     float v0 = 0.f, v1 = 0.f;
     for (int z = 0; z < zsplits; ++z) {
         if (lane < N) v0 += row[z * zstride + col_logits + lane];
