@@ -239,6 +239,8 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "stages")) t.stages = value;
     else if (!strcmp(name, "tile_tokens")) t.tile_tokens = value;
     else if (!strcmp(name, "kc")) t.kc = value;
+    else if (!strcmp(name, "zmax")) t.zmax = value;
+    else if (!strcmp(name, "stacked_direct")) t.stacked_direct = value;
     else if (!strcmp(name, "simt_expand")) t.simt_expand = value;
     else if (!strcmp(name, "force_simt")) t.force_simt = value;
     else if (!strcmp(name, "pdl")) t.pdl = value;

@@ -66,6 +66,8 @@ struct Tuning {
     int stages = 0;
     int tile_tokens = 0;
     int kc = 0;
+    int zmax = 0;          // cap on the contraction slices of the decode-batch stacked shrink (0: automatic)
+    int stacked_direct = 0;  // 1: decode-batch stacked shrink without clusters, slices stored directly
     int simt_expand = 0;   // 1: keep the LoRA expand on CUDA cores even for rank 8
     int force_simt = 0;
     int pdl = 1;

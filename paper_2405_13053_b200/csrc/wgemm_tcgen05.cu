@@ -808,19 +808,19 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     // further over grid z (every slice keeps at least two k-steps); the selection kernel adds the slices.
     pl.zsplits = 1;
     if (!lora && pl.n_tiles == 1) {
-        // decode-batch stacked shrink: every CTA takes a slice of the contraction axis of one row tile and
-        // writes its partial straight to u_all[z]; no cluster, no reduction here (the selection adds them).
-        splits = tn.splits > 0 ? splits : 1;
-        pl.splits = splits;
-        pl.zsplits = std::min(kMaxZSplits, std::max(1, ksteps / splits / 2));
+        // Decode-batch stacked shrink (a handful of row tiles): cut the contraction axis further over grid z,
+        // every slice keeping at least two k-steps; the selection kernel adds the slices.  With the
+        // "stacked_direct" knob there is no cluster at all: up to 32 slices, each stored straight to u_all[z].
+        if (tn.stacked_direct) {
+            splits = tn.splits > 0 ? splits : 1;
+            pl.splits = splits;
+        }
+        const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits) : (tn.stacked_direct ? kMaxZSplits : 4);
+        pl.zsplits = std::min(zcap, std::max(1, ksteps / splits / 2));
     }
     const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
-    // Decode batches run as a chain stacked shrink -> selection -> base product overlapped by programmatic
-    // dependent launch: a base-product CTA and a shrink CTA must fit on one SM together (227 KB, 512 TMEM
-    // columns), so the shrink keeps to ~64 KB and the base product to 156 KB.
-    const bool decode = pl.n_tiles == 1 && T <= 256;
-    const size_t total_budget = two_per_sm ? 112 * 1024 : decode ? (lora ? 156 * 1024 : 60 * 1024) : 226 * 1024;
+    const size_t total_budget = two_per_sm ? 112 * 1024 : 226 * 1024;
 
     // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
     const int tile_tokens = std::min(T, bn);
