@@ -859,7 +859,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     if (pl.maps3d && ksteps % parts == 0) {
         const int per = ksteps / parts;
         for (int cand = 4; cand > 1; cand /= 2)
-            if (per % cand == 0 && 2 * cand * chunk_bytes <= avail) {
+            if (per % cand == 0 && (size_t)std::max(2, tn.stages) * cand * chunk_bytes <= avail) {
                 kc = cand;
                 break;
             }
