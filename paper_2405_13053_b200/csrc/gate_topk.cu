@@ -6,41 +6,11 @@
 #include <math_constants.h>
 
 #include "common.cuh"
+#include "select.cuh"
 
 namespace meteora {
 
 constexpr int kGateWarps = 8;
-
-// v0 = logit[lane], v1 = logit[lane + 32]; entries at or beyond N are ignored.
-// On return lane j < k holds pick j (index and softmax weight).  Every lane runs the same code.
-__device__ __forceinline__ void warp_topk_softmax(float v0, float v1, int N, int k, float inv_tau, int lane,
-                                                  int& my_idx, float& my_w) {
-    bool taken0 = lane >= N, taken1 = lane + 32 >= N;
-    if (!(v0 > -CUDART_INF_F)) v0 = -CUDART_INF_F;  // NaN never wins a comparison; treat it as -inf
-    if (!(v1 > -CUDART_INF_F)) v1 = -CUDART_INF_F;
-    float first = 0.f, sum = 0.f, my_e = 0.f;
-    my_idx = 0;
-    for (int j = 0; j < k; ++j) {
-        float bv = -CUDART_INF_F;
-        int bi = 0x7FFFFFFF;
-        if (!taken0) { bv = v0; bi = lane; }
-        if (!taken1 && (bi == 0x7FFFFFFF || v1 > bv)) { bv = v1; bi = lane + 32; }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
-            const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        bi = min(bi, N - 1);
-        if (bi == lane) taken0 = true;
-        if (bi == lane + 32) taken1 = true;
-        if (j == 0) first = bv;
-        const float e = expf((bv - first) * inv_tau);
-        sum += e;
-        if (lane == j) { my_idx = bi; my_e = e; }
-    }
-    my_w = my_e / sum;
-}
 
 template <typename TI>
 __global__ void __launch_bounds__(kGateWarps * 32)
@@ -88,82 +58,7 @@ k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits,
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * kGateWarps + (threadIdx.x >> 5);
     if (t >= T) return;
-    const float* row = u_all + (size_t)t * ld_u;
-    if (zsplits > 1 && zsplits <= 32 && r == 8 && k <= 4) {
-        // Many partial copies: lane z reads slice z, so all loads of a phase are in flight at once (one
-        // memory round trip instead of one per slice); the slices are then added across lanes by a
-        // butterfly, the same order for every token and every run.
-        const float* mine = row + (size_t)min(lane, zsplits - 1) * zstride;
-        const bool live = lane < zsplits;
-        float v0 = 0.f, v1 = 0.f;
-        for (int n0 = 0; n0 < N; n0 += 32) {
-            float vals[32];
-#pragma unroll
-            for (int n = 0; n < 32; ++n) vals[n] = (live && n0 + n < N) ? mine[col_logits + n0 + n] : 0.f;
-#pragma unroll
-            for (int n = 0; n < 32; ++n) {
-                if (n0 + n < N) {                       // uniform across the warp
-                    const float sum = warp_sum(vals[n]);
-                    if (lane == n) { if (n0 == 0) v0 = sum; else v1 = sum; }
-                }
-            }
-        }
-        int idx;
-        float w;
-        warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
-        if (lane < k) {
-            topk_idx[(size_t)t * k + lane] = idx;
-            topk_w[(size_t)t * k + lane] = w;
-        }
-        float4 part[4][2];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
-            const float4* src = reinterpret_cast<const float4*>(mine + ij * 8);
-            const bool on = live && j < k;
-            part[j][0] = on ? src[0] : make_float4(0.f, 0.f, 0.f, 0.f);
-            part[j][1] = on ? src[1] : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        float out = 0.f;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (j < k) {                                // uniform across the warp
-                const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
-                const float e[8] = {part[j][0].x, part[j][0].y, part[j][0].z, part[j][0].w,
-                                    part[j][1].x, part[j][1].y, part[j][1].z, part[j][1].w};
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float sum = warp_sum(e[q]);
-                    if (lane == j * 8 + q) out = wj * sum;
-                }
-            }
-        }
-        if (lane < k * 8) uw[(size_t)t * k * 8 + lane] = out;
-        return;
-    }
-    float v0 = 0.f, v1 = 0.f;
-    for (int z = 0; z < zsplits; ++z) {
-        if (lane < N) v0 += row[z * zstride + col_logits + lane];
-        if (lane + 32 < N) v1 += row[z * zstride + col_logits + lane + 32];
-    }
-    int idx;
-    float w;
-    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
-    if (lane < k) {
-        topk_idx[(size_t)t * k + lane] = idx;
-        topk_w[(size_t)t * k + lane] = w;
-    }
-    for (int c0 = 0; c0 < k * r; c0 += 32) {
-        const int c = c0 + lane;
-        const int j = min(c / r, k - 1), p = c - j * r;
-        const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
-        const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
-        if (c < k * r) {
-            float u = 0.f;
-            for (int z = 0; z < zsplits; ++z) u += row[z * zstride + ij * r + p];
-            uw[(size_t)t * k * r + c] = wj * u;
-        }
-    }
+    select_token<false>(u_all, ld_u, col_logits, zsplits, zstride, t, N, r, k, inv_tau, lane, topk_idx, topk_w, uw);
 }
 
 int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, int32_t* topk_idx, float* topk_w,
