@@ -162,8 +162,9 @@ size_t meteora_workspace_bytes(const meteora_shape_t* shape);
 int meteora_workspace_routing(const meteora_shape_t* shape, void* workspace, int32_t** topk_idx, float** topk_w);
 
 /*
- * Clears the status block at the head of a freshly allocated workspace (asynchronous, on `stream`).
- * Call once before the workspace's first use; memory that is already zero needs no call.
+ * Clears the 4 KB header of a freshly allocated workspace (status words and the counters the
+ * single-launch decode kernel synchronises on), asynchronously on `stream`.  Call once before the
+ * workspace's first use; memory that is already zero needs no call.
  */
 int meteora_workspace_init(void* workspace, void* stream);
 
@@ -185,6 +186,13 @@ int meteora_workspace_status(void* workspace, void* stream);
  */
 int meteora_profile_begin(int max_launches);
 int meteora_profile_end(float* total_ms, int* launches);
+
+/*
+ * Writes a one-line description of how meteora_linear_forward will run this shape (path, launches,
+ * CTAs, split factor, tile, ring depth) into buf, followed by the number of single-launch decode
+ * kernels the driver has refused so far in this process.  Host-only; for logs and benchmark records.
+ */
+int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_bytes);
 
 /*
  * Tuning knobs for measurements (process-wide, not thread-safe): "splits" (split-K cluster size,

@@ -26,7 +26,7 @@ EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_
            "meteora_linear_forward",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
            "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
-           "meteora_set_tuning", "meteora_status_string"]
+           "meteora_describe_plan", "meteora_set_tuning", "meteora_status_string"]
 
 
 class MeteoraShape(ctypes.Structure):
@@ -67,6 +67,7 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_workspace_status.argtypes = [vp, vp]
     lib.meteora_profile_begin.argtypes = [ci]
     lib.meteora_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci)]
+    lib.meteora_describe_plan.argtypes = [shp, ctypes.c_char_p, sz]
     lib.meteora_set_tuning.argtypes = [ctypes.c_char_p, ci]
     lib.meteora_status_string.argtypes = [ci]
     lib.meteora_status_string.restype = ctypes.c_char_p
@@ -275,6 +276,12 @@ def meteora_profile_end() -> Tuple[float, int]:
     ms, n = ctypes.c_float(), ctypes.c_int()
     _check(load_library().meteora_profile_end(ctypes.byref(ms), ctypes.byref(n)), "meteora_profile_end")
     return float(ms.value), int(n.value)
+
+
+def meteora_describe_plan(shape: MeteoraShape) -> str:
+    buf = ctypes.create_string_buffer(640)
+    _check(load_library().meteora_describe_plan(ctypes.byref(shape), buf, len(buf)), "meteora_describe_plan")
+    return buf.value.decode()
 
 
 def meteora_set_tuning(name: str, value: int) -> None:

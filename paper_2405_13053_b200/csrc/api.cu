@@ -1,5 +1,6 @@
 // C ABI of the library (declared in include/meteora.h): argument validation, workspace carve-up,
 // dispatch between the tensor-core path and the plain CUDA-core path.
+#include <stdio.h>
 #include <string.h>
 
 #include <vector>
@@ -26,11 +27,17 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     int col_logits = 0;
     ws.ld_u = tc_stacked_pitch(s, &col_logits);
     ws.col_logits = col_logits;
-    ws.status = (int32_t*)take(64 * sizeof(int32_t));
+    ws.status = (int32_t*)take(kHeaderBytes);   // status words [0,64), fused-decode tile counters [64,1024)
+    ws.tile_ctr = ws.status ? ws.status + 64 : nullptr;
     ws.topk_idx = (int32_t*)take(T * s.k * sizeof(int32_t));
     ws.topk_w = (float*)take(T * s.k * sizeof(float));
     ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
     ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (s.T <= 256 ? 32 : 1));   // up to 32 slices for decode batches
+    // fused decode scratch: at most 296 resident CTAs (or 8 per row tile), each one tile of 128 x BN fp32
+    const size_t row_tiles = ((size_t)s.d_out + 127) / 128;
+    const size_t bn = (T + 15) / 16 * 16;
+    const size_t part_tiles = s.T <= 256 ? (row_tiles * 8 < 296 ? row_tiles * 8 : 296) : 0;
+    ws.part_g = (float*)take(part_tiles * bn * 128 * sizeof(float));
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);
     ws.bytes = off;
@@ -67,14 +74,24 @@ static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 static int forward_device(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                           const meteora_shape_t& s, void* y, const Workspace& ws, cudaStream_t st) {
     int rc;
+    Profile& pf = profile();
+    const bool timed = pf.open && 2 * (pf.used + 1) <= (int)pf.ev.size();
+    if (decode_fused_supported(s)) {
+        if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
+        rc = launch_decode_fused(x, W0, A, B, Wg, s, ws, y, st);
+        if (rc != METEORA_ERR_CUDA) {
+            if (timed) cudaEventRecord(pf.ev[2 * pf.used++ + 1], st);
+            return rc;
+        }
+        cudaGetLastError();   // the cooperative launch was refused (not all CTAs can be resident): use the chain
+        tuning().fused_refused += 1;
+    }
     if (tc_path_supported(s)) {
         const bool pdl = tuning().pdl != 0;
         if ((rc = launch_stacked_shrink_tc(x, A, Wg, s, ws, st)) != METEORA_OK) return rc;
-        if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, tc_stacked_zsplits(s), s, ws.topk_idx, ws.topk_w, ws.uw, pdl,
-                                             st)) != METEORA_OK)
+        if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, tc_stacked_zsplits(s), s, ws.topk_idx,
+                                             ws.topk_w, ws.uw, pdl, st)) != METEORA_OK)
             return rc;
-        Profile& pf = profile();
-        const bool timed = pf.open && 2 * (pf.used + 1) <= (int)pf.ev.size();
         if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
         rc = launch_base_lora_tc(x, W0, B, s, ws, y, pdl && !timed, st);
         if (timed) cudaEventRecord(pf.ev[2 * pf.used++ + 1], st);
@@ -183,7 +200,7 @@ int meteora_workspace_routing(const meteora_shape_t* shape, void* workspace, int
 
 int meteora_workspace_init(void* workspace, void* stream) {
     if (!workspace) return METEORA_ERR_INVALID_ARG;
-    return cuda_status(cudaMemsetAsync(workspace, 0, 64 * sizeof(int32_t), (cudaStream_t)stream));
+    return cuda_status(cudaMemsetAsync(workspace, 0, kHeaderBytes, (cudaStream_t)stream));
 }
 
 int meteora_workspace_status(void* workspace, void* stream) {
@@ -194,7 +211,7 @@ int meteora_workspace_status(void* workspace, void* stream) {
         return METEORA_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return METEORA_ERR_CUDA;
     if (word != 0) {
-        if (cudaMemsetAsync(workspace, 0, 64 * sizeof(int32_t), st) != cudaSuccess) return METEORA_ERR_CUDA;
+        if (cudaMemsetAsync(workspace, 0, kHeaderBytes, st) != cudaSuccess) return METEORA_ERR_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return METEORA_ERR_CUDA;
         return METEORA_ERR_TIMEOUT;
     }
@@ -232,6 +249,16 @@ int meteora_profile_end(float* total_ms, int* launches) {
     return METEORA_OK;
 }
 
+int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_bytes) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (!buf || buf_bytes == 0) return METEORA_ERR_INVALID_ARG;
+    char tmp[512];
+    describe_plan(*shape, tmp, sizeof(tmp));
+    snprintf(buf, buf_bytes, "%s fused_refused=%d", tmp, tuning().fused_refused);
+    return METEORA_OK;
+}
+
 int meteora_set_tuning(const char* name, int value) {
     if (!name) return METEORA_ERR_INVALID_ARG;
     Tuning& t = tuning();
@@ -244,6 +271,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "simt_expand")) t.simt_expand = value;
     else if (!strcmp(name, "force_simt")) t.force_simt = value;
     else if (!strcmp(name, "pdl")) t.pdl = value;
+    else if (!strcmp(name, "fused")) t.fused = value;
     else return METEORA_ERR_INVALID_ARG;
     return METEORA_OK;
 }

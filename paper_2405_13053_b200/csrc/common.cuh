@@ -12,6 +12,9 @@ namespace meteora {
 // ---------------------------------------------------------------------------------------------
 // Workspace layout.  Every region starts on a 256-byte boundary.
 // ---------------------------------------------------------------------------------------------
+constexpr size_t kHeaderBytes = 4096;    // zero-initialised head of every workspace
+constexpr int kMaxFusedRowTiles = 960;   // tile counters that fit into the header
+
 struct Workspace {
     int32_t* status;    // [64]  word 0: error flag of bounded device waits; words 1..: where it gave up
     int32_t* topk_idx;  // [T,k]
@@ -21,6 +24,8 @@ struct Workspace {
                         //           copies (slices of the contraction axis) that the selection kernel adds up
     int ld_u;           // row pitch of u_all in floats
     int col_logits;     // first logit column inside a u_all row
+    float* part_g;      // fused decode: fp32 partial accumulator tiles of the base product (T <= 256 only)
+    int32_t* tile_ctr;  // fused decode: one counter per 128-row tile of d_out (inside the header)
     void* x_dev;        // [T,d_in]  staging for the host-buffer entry point
     void* y_dev;        // [T,d_out]
     size_t bytes;       // total
@@ -61,6 +66,12 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
 int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
                         void* y, bool pdl, cudaStream_t st);
 
+// fused decode kernel (wgemm_tcgen05.cu + decode_fused.cuh)
+bool decode_fused_supported(const meteora_shape_t& s);
+int describe_plan(const meteora_shape_t& s, char* buf, size_t n);
+int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                        const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
+
 struct Tuning {
     int splits = 0;
     int stages = 0;
@@ -71,6 +82,8 @@ struct Tuning {
     int simt_expand = 0;   // 1: keep the LoRA expand on CUDA cores even for rank 8
     int force_simt = 0;
     int pdl = 1;
+    int fused = 1;           // 0: never use the single-launch decode kernel
+    int fused_refused = 0;   // cooperative launches the driver refused (the chain ran instead)
 };
 Tuning& tuning();
 

@@ -322,16 +322,29 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             const int o = tile_m * kBM + rit;
             const float* src = S > 1 ? d.part_g + (size_t)tile_m * S * part_stride : part;
             for (int t0 = tg; t0 < ntok; t0 += 4 * TPP) {
-                float2 acc[4];
+                float2 acc[4], v[4][8];
+                // all partial loads of four tokens first (one L2 round trip), then the sums in split order
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int t = min(t0 + u * TPP, ntok - 1);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        v[u][q] = make_float2(0.f, 0.f);
+                        if (q < S) {
+                            const float2* a = reinterpret_cast<const float2*>(src + q * part_stride + t * kBM + rit);
+                            v[u][q] = S > 1 ? __ldcg(a) : *a;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
                     acc[u] = make_float2(0.f, 0.f);
-                    for (int q = 0; q < S; ++q) {
-                        const float2* a = reinterpret_cast<const float2*>(src + q * part_stride + t * kBM + rit);
-                        const float2 v = S > 1 ? __ldcg(a) : *a;
-                        acc[u].x += v.x;
-                        acc[u].y += v.y;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (q < S) {
+                            acc[u].x += v[u][q].x;
+                            acc[u].y += v[u][q].y;
+                        }
                     }
                 }
 #pragma unroll

@@ -18,10 +18,13 @@
 // and drains instead of hanging.
 #include <cuda.h>
 
+#include <stdio.h>
+
 #include <mutex>
 #include <vector>
 
 #include "common.cuh"
+#include "select.cuh"
 
 namespace meteora {
 
@@ -670,6 +673,12 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     }
 }
 
+}  // namespace meteora
+
+#include "decode_fused.cuh"
+
+namespace meteora {
+
 // ------------------------------------------------------------------------------------------------
 // Host side: tensor maps, planning, launches
 // ------------------------------------------------------------------------------------------------
@@ -1001,6 +1010,152 @@ int launch_base_lora_tc(const void* x, const void* W0, const void* B, const mete
     p.pdl_wait = pdl ? 1 : 0;
     p.pdl_trigger = 0;
     return launch_wgemm(mW, mW, mX, p, row_tiles, pl, pdl, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Fused decode launch: base product + stacked shrink + selection in one cooperative kernel.
+// ------------------------------------------------------------------------------------------------
+// How many CTAs of the fused kernel with `smem` bytes of dynamic shared memory fit on the device at once.
+static int max_resident_ctas(size_t smem) {
+    static std::mutex mu;
+    static std::vector<std::pair<size_t, int>> cache;
+    const size_t key = (smem + 1023) / 1024;
+    std::lock_guard<std::mutex> lock(mu);
+    for (auto& e : cache)
+        if (e.first == key) return e.second;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_decode_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess)
+            cudaGetLastError();
+        attr_set = true;
+    }
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_fused, kThreads, smem) != cudaSuccess) {
+        cudaGetLastError();
+        per_sm = 0;
+    }
+    const int n = per_sm * sm_count();
+    cache.push_back({key, n});
+    return n;
+}
+
+struct FusedPlan {
+    bool ok;
+    int why;   // why not: 1 knob/shape, 2 too many row tiles, 3 several token tiles, 4 residency, 5 operand sizes
+    Plan main;
+    int row_tiles, n_main, n_aux, a_tiles, aux_slices, aux_stages;
+};
+
+static FusedPlan make_fused_plan(const meteora_shape_t& s) {
+    FusedPlan fp = {};
+    fp.why = 1;
+    if (!tuning().fused || !tc_path_supported(s) || s.T > 256 || s.r != 8 || tuning().simt_expand) return fp;
+    fp.row_tiles = (s.d_out + kBM - 1) / kBM;
+    fp.why = 2;
+    if (fp.row_tiles > kMaxFusedRowTiles) return fp;
+    fp.main = make_plan(fp.row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
+    fp.why = 3;
+    if (fp.main.n_tiles != 1) return fp;
+    fp.why = 5;
+    if (!fp.main.lora_mma || fp.main.us_in_ring) return fp;
+    fp.why = 4;
+    const int S = fp.main.splits;
+    fp.n_main = fp.row_tiles * S;
+    const int capacity = max_resident_ctas(fp.main.smem);
+    fp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
+    const int aux_tiles = fp.a_tiles + 1;
+    const int n_aux = std::min(capacity - fp.n_main, 24);
+    if (n_aux < aux_tiles) return fp;
+    const int ksteps = (s.d_in + kBK - 1) / kBK;
+    fp.aux_slices = std::min(std::min(n_aux / aux_tiles, ksteps), 32);
+    fp.n_aux = aux_tiles * fp.aux_slices;
+    const size_t chunk = kWTileBytes + (size_t)fp.main.BN * 128;
+    const size_t ring_bytes = (size_t)fp.main.stages * fp.main.kc * chunk;
+    const int nks_aux = (ksteps + fp.aux_slices - 1) / fp.aux_slices;
+    fp.aux_stages = (int)std::min<size_t>(ring_bytes / chunk, (size_t)std::min(fp.main.stages, std::max(nks_aux, 1)));
+    fp.why = 5;
+    if (fp.aux_stages < 1) return fp;
+    fp.why = 0;
+    fp.ok = true;
+    return fp;
+}
+
+bool decode_fused_supported(const meteora_shape_t& s) { return make_fused_plan(s).ok; }
+
+// Human-readable launch plan of meteora_linear_forward for this shape (for logs and benchmark records).
+int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
+    if (!tc_path_supported(s)) return snprintf(buf, n, "path=simt");
+    const FusedPlan fp = make_fused_plan(s);
+    if (fp.ok)
+        return snprintf(buf, n,
+                        "path=fused_decode launches=1 main_ctas=%d splits=%d aux_ctas=%d aux_slices=%d tile_tokens=%d "
+                        "stages=%d kc=%d smem=%zu resident_ctas=%d",
+                        fp.n_main, fp.main.splits, fp.n_aux, fp.aux_slices, fp.main.BN, fp.main.stages, fp.main.kc,
+                        fp.main.smem, max_resident_ctas(fp.main.smem));
+    const int row_tiles = (s.d_out + kBM - 1) / kBM;
+    const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
+    return snprintf(buf, n,
+                    "path=chain(not fused: reason %d) launches=3 base_ctas=%d cluster=%d tile_tokens=%d stages=%d kc=%d "
+                    "smem=%zu expand=%s",
+                    fp.why, row_tiles * pl.splits * pl.n_tiles, pl.splits, pl.BN, pl.stages, pl.kc, pl.smem,
+                    pl.lora_mma ? "mma" : "simt");
+}
+
+int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                        const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st) {
+    const FusedPlan fp = make_fused_plan(s);
+    if (!fp.ok) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    const Plan& pl = fp.main;
+    const int depth = pl.maps3d ? pl.kc : 0, depth1 = pl.maps3d ? 1 : 0;
+    CUtensorMap mW, mX, mA, mG, mX1;
+    int rc;
+    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, depth, &mW)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, depth, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, depth1, &mA)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Wg, s.d_in, s.N, kBM, depth1, &mG)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, depth1, &mX1)) != METEORA_OK) return rc;
+    DecodeParams d = {};
+    fill_common(d.main, pl, s.T, s.d_in, ws.status);
+    d.main.split_tile = 0x7FFFFFFF;
+    d.main.rows0 = s.d_out;
+    d.main.mode = MODE_LORA;
+    d.main.topk_idx = ws.topk_idx;
+    d.main.uw = ws.uw;
+    d.main.B = (const __nv_bfloat16*)B;
+    d.main.y = (__nv_bfloat16*)y;
+    d.main.d_out = s.d_out;
+    d.main.N = s.N;
+    d.main.r = s.r;
+    d.main.k = s.k;
+    d.n_main = fp.n_main;
+    d.a_tiles = fp.a_tiles;
+    d.a_rows = s.N * s.r;
+    d.aux_slices = fp.aux_slices;
+    d.aux_stages = fp.aux_stages;
+    d.u_part = ws.u_all;
+    d.ld_u = ws.ld_u;
+    d.col_logits = ws.col_logits;
+    d.topk_idx = ws.topk_idx;
+    d.topk_w = ws.topk_w;
+    d.uw = ws.uw;
+    d.inv_tau = 1.0f / s.temperature;
+    d.ctr = ws.status + 16;
+    d.part_g = ws.part_g;
+    d.tile_ctr = ws.tile_ctr;
+    d.row_tiles = fp.row_tiles;
+    if (pl.smem > 227 * 1024) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(fp.n_main + fp.n_aux);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mG, mX1, d));
 }
 
 }  // namespace meteora
