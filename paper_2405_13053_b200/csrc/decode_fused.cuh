@@ -75,6 +75,17 @@ __device__ __forceinline__ void stage_us_mma_coherent(const WGemmParams& p, uint
     }
 }
 
+#ifdef METEORA_TRACE
+#define FUSED_STAMP(p, base, slot)                                                  \
+    do {                                                                            \
+        unsigned long long t_;                                                      \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                      \
+        (p).status[(base) + (slot)] = (int)(t_ & 0x7FFFFFFF);                       \
+    } while (0)
+#else
+#define FUSED_STAMP(p, base, slot) do { } while (0)
+#endif
+
 __device__ __forceinline__ void flag_error(const WGemmParams& p, int word, int code) {
     atomicExch(p.status, 1);
     atomicExch(p.status + word, code);
@@ -178,6 +189,9 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int ntok = min(p.BN, p.T);
     const int half = ((p.BN / 16 + 1) / 2) * 16;
     const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
+    const bool tr_main = blockIdx.x == 0, tr_aux = (int)blockIdx.x == d.n_main;
+    if (threadIdx.x == 0 && tr_main) FUSED_STAMP(p, 32, 0);
+    if (threadIdx.x == 0 && tr_aux) FUSED_STAMP(p, 48, 0);
 
     if (is_aux) {
         // ================================================================== aux CTA
@@ -200,6 +214,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             if (lane == 0 && active) {
                 if (!fused_mma(geom, tmem_base, idesc, niter)) flag_error(p, 2, 500);
                 umma_commit(bar_acc);
+                if (tr_aux) FUSED_STAMP(p, 48, 1);
             }
         } else if (active) {
             bool acc_ok = mbar_wait(bar_acc, 0);
@@ -230,9 +245,11 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         __syncthreads();
         if (active) {
             if (threadIdx.x == 0) {
+                if (tr_aux) FUSED_STAMP(p, 48, 2);
                 __threadfence();
                 atomicAdd(d.ctr + 0, 1);
                 if (!wait_counter(d.ctr + 0, n_active)) flag_error(p, 4, 700);   // every slice of every tile is in
+                if (tr_aux) FUSED_STAMP(p, 48, 3);
             }
             __syncthreads();
             const int nwarps = kThreads / 32;                                    // tokens dealt round-robin
@@ -243,6 +260,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             if (threadIdx.x == 0) {
                 __threadfence();
                 atomicAdd(d.ctr + 1, 1);
+                if (tr_aux) FUSED_STAMP(p, 48, 4);
             }
         }
     } else {
@@ -261,12 +279,14 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             if (lane == 0) {
                 // let the stacked shrink get its loads into the memory queues first
                 bool ok = wait_counter(d.ctr + 3, n_active);
+                if (tr_main) FUSED_STAMP(p, 32, 1);
                 ok = fused_producer(geom, &tmW0, &tmX, tile_m * kBM, ks0, niter, nullptr) && ok;
                 if (!ok) flag_error(p, 1, 100);
             }
         } else if (warp == 1) {
             if (lane == 0) {
                 bool ok = fused_mma(geom, tmem_base, idesc, niter);
+                if (tr_main) FUSED_STAMP(p, 32, 2);
                 if (ok) ok = mbar_wait(bar_us, 0);                            // operands of the expand staged
                 if (ok) {
                     tc_fence_after();
@@ -282,7 +302,9 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         } else {
             const int a0 = split * p.na;
             stage_slab_mma(p, epi, a0, tile_m * kBM, etid);                   // B rows: no routing needed
+            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
             if (etid == 0 && !wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);   // routing published
+            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 4);
             epi_barrier();
             stage_us_mma_coherent(p, reinterpret_cast<uint4*>(epi + p.us_off), a0, ntok, etid);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -292,6 +314,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             if (!acc_ok && lane == 0) flag_error(p, 3, 300);
             acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
             tc_fence_after();
+            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 5);
             // Accumulators out of TMEM: to the fp32 scratch when the tile is split over several CTAs (lane =
             // row, a warp writes 128 contiguous bytes per token), else to the idle ring.
             float* part = S > 1 ? my_part : reinterpret_cast<float*>(ring_ptr);
@@ -314,6 +337,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 atomicAdd(d.tile_ctr + tile_m, 1);
                 if (!wait_counter(d.tile_ctr + tile_m, S)) flag_error(p, 4, 900);   // all partials of the tile in
             }
+            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 6);
             epi_barrier();
             // sum the slice of rows this CTA owns over the S partials, in split order, and store y
             const int P = 64 / S, TPP = kEpiThreads / P, NROWS = kBM / S;
@@ -365,6 +389,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0 && tr_main) FUSED_STAMP(p, 32, 7);
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"((uint32_t)p.tmem_cols)
