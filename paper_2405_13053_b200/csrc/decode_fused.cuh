@@ -24,6 +24,7 @@ struct DecodeParams {
     int a_tiles, a_rows;   // row tiles / rows of the stacked A matrix (N * r rows); one more tile holds Wg
     int aux_slices;        // contraction slices per aux row tile; active aux CTAs = (a_tiles + 1) * aux_slices
     int aux_stages;        // ring depth of the aux main loop (one k-step per stage)
+    int bar_stages;        // barriers are laid out for max(main stages, aux stages) ring slots
     float* u_part;         // [aux_slices][T][ld_u] partial stacked shrink
     int ld_u, col_logits;
     int32_t* topk_idx;     // selection results, written by aux CTAs, read by main CTAs
@@ -160,7 +161,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const uint32_t stage_bytes = p.kc * (kWTileBytes + x_tile_bytes);
     const uint32_t ring_bytes = p.stages * stage_bytes;
     const uint32_t bar_base = ring + ring_bytes;
-    const int nbar = 2 * p.stages + 3;               // aux CTAs use a prefix of the same barriers
+    const int nbar = 2 * d.bar_stages + 3;           // sized for the deeper of the two rings
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + nbar * 8);
     uint8_t* epi = ring_ptr + ring_bytes + p.epi_off;
 

@@ -891,7 +891,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     int cols = 32;
     while (cols < bn) cols *= 2;
     pl.tmem_cols = cols;
-    pl.epi_off = (int)align_up((size_t)(2 * stages + 3) * 8 + 16, 128);
+    pl.epi_off = (int)align_up((size_t)(2 * std::max(stages, 16) + 3) * 8 + 16, 128);
     pl.smem = 1024 + (size_t)stages * stage_bytes + pl.epi_off + epi_bytes;
     return pl;
 }
@@ -1073,7 +1073,10 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     const size_t chunk = kWTileBytes + (size_t)fp.main.BN * 128;
     const size_t ring_bytes = (size_t)fp.main.stages * fp.main.kc * chunk;
     const int nks_aux = (ksteps + fp.aux_slices - 1) / fp.aux_slices;
-    fp.aux_stages = (int)std::min<size_t>(ring_bytes / chunk, (size_t)std::min(fp.main.stages, std::max(nks_aux, 1)));
+    fp.aux_stages = (int)std::min<size_t>(ring_bytes / chunk, (size_t)std::max(nks_aux, 1));
+    // the barrier block behind the ring was laid out for the main ring: keep the aux ring within it
+    const int bar_cap = (fp.main.epi_off - 16) / 8 - 3;
+    fp.aux_stages = std::min(fp.aux_stages, std::min(bar_cap / 2, 16));
     fp.why = 5;
     if (fp.aux_stages < 1) return fp;
     fp.why = 0;
@@ -1133,6 +1136,7 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.a_rows = s.N * s.r;
     d.aux_slices = fp.aux_slices;
     d.aux_stages = fp.aux_stages;
+    d.bar_stages = std::max(fp.aux_stages, pl.stages);
     d.u_part = ws.u_all;
     d.ld_u = ws.ld_u;
     d.col_logits = ws.col_logits;
