@@ -54,7 +54,46 @@ __device__ __forceinline__ void select_token(const float* u_all, int ld_u, int c
                                              size_t zstride, int t, int N, int r, int k, float inv_tau, int lane,
                                              int32_t* topk_idx, float* topk_w, float* uw) {
     const float* row = u_all + (size_t)t * ld_u;
-    if (zsplits > 1 && zsplits <= 32 && r == 8 && k <= 4) {
+    if (zsplits <= 8) {
+        // Few partial copies: lane n owns logit n and reads it from every slice, the (at most 8) loads
+        // issued together; the slices are added in slice order.
+        float part0[8], part1[8];
+#pragma unroll
+        for (int z = 0; z < 8; ++z) {
+            const bool on = z < zsplits;
+            part0[z] = (on && lane < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane) : 0.f;
+            part1[z] = (on && lane + 32 < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32) : 0.f;
+        }
+        float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+        for (int z = 0; z < 8; ++z) {
+            v0 += part0[z];
+            v1 += part1[z];
+        }
+        int idx;
+        float w;
+        warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+        if (lane < k) {
+            topk_idx[(size_t)t * k + lane] = idx;
+            topk_w[(size_t)t * k + lane] = w;
+        }
+        for (int c0 = 0; c0 < k * r; c0 += 32) {
+            const int c = c0 + lane;
+            const int j = min(c / r, k - 1), q = c - j * r;
+            const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
+            const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
+            float pu[8];
+#pragma unroll
+            for (int z = 0; z < 8; ++z)
+                pu[z] = (z < zsplits && c < k * r) ? ld_part<kCoherent>(row + z * zstride + ij * r + q) : 0.f;
+            float u = 0.f;
+#pragma unroll
+            for (int z = 0; z < 8; ++z) u += pu[z];
+            if (c < k * r) uw[(size_t)t * k * r + c] = wj * u;
+        }
+        return;
+    }
+    if (zsplits <= 32 && r == 8 && k <= 4) {
         // Many partial copies: lane z reads slice z, so all loads of a phase are in flight at once (one
         // memory round trip instead of one per slice); the slices are then added across lanes by a
         // butterfly, the same order for every token and every run.
