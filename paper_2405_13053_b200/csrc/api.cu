@@ -272,6 +272,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "force_simt")) t.force_simt = value;
     else if (!strcmp(name, "pdl")) t.pdl = value;
     else if (!strcmp(name, "fused")) t.fused = value;
+    else if (!strcmp(name, "coop")) t.coop = value;
     else return METEORA_ERR_INVALID_ARG;
     return METEORA_OK;
 }

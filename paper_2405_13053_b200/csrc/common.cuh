@@ -83,6 +83,7 @@ struct Tuning {
     int force_simt = 0;
     int pdl = 1;
     int fused = 1;           // 0: never use the single-launch decode kernel
+    int coop = 1;            // 0 (measurement only): launch it without the co-residency guarantee
     int fused_refused = 0;   // cooperative launches the driver refused (the chain ran instead)
 };
 Tuning& tuning();

@@ -20,7 +20,8 @@ namespace meteora {
 
 struct DecodeParams {
     WGemmParams main;      // base product (MODE_LORA, lora_mma): ring geometry, staging offsets, outputs
-    int n_main;            // main CTAs = row tiles * S; CTAs from n_main on are aux
+    int n_main;            // main CTAs = row tiles * S
+    int n_aux;             // aux CTAs; they take the lowest block indices so that they are scheduled first
     int a_tiles, a_rows;   // row tiles / rows of the stacked A matrix (N * r rows); one more tile holds Wg
     int aux_slices;        // contraction slices per aux row tile; active aux CTAs = (a_tiles + 1) * aux_slices
     int aux_stages;        // ring depth of the aux main loop (one k-step per stage)
@@ -52,12 +53,10 @@ __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
     return true;
 }
 
-// Token-side operand of the tensor-core expand, as stage_us_mma but reading the routing with loads that
-// bypass L1 (it was written by other CTAs of this same kernel).
-__device__ __forceinline__ void stage_us_mma_coherent(const WGemmParams& p, uint4* us, int a0, int ntok, int etid) {
-    const int total = p.na * p.BN;
-    for (int v = etid; v < total; v += kEpiThreads) us[v] = make_uint4(0u, 0u, 0u, 0u);
-    epi_barrier();
+// Token-side operand of the tensor-core expand: the caller has zeroed it; scatter bf16(w_j * A_e x_t) of the
+// slots whose adapter belongs to this CTA, reading the routing with loads that bypass L1 (it was written
+// by other CTAs of this same kernel).
+__device__ __forceinline__ void scatter_us_mma_coherent(const WGemmParams& p, uint4* us, int a0, int ntok, int etid) {
     const int slots = ntok * p.k;
     const float4* uw4 = reinterpret_cast<const float4*>(p.uw);
     for (int i = etid; i < slots; i += kEpiThreads) {
@@ -166,7 +165,8 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     uint8_t* epi = ring_ptr + ring_bytes + p.epi_off;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool is_aux = (int)blockIdx.x >= d.n_main;
+    const bool is_aux = (int)blockIdx.x < d.n_aux;
+    const int main_id = (int)blockIdx.x - d.n_aux;
     const int n_active = (d.a_tiles + 1) * d.aux_slices;
 
     if (threadIdx.x == 0) {
@@ -190,13 +190,13 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int ntok = min(p.BN, p.T);
     const int half = ((p.BN / 16 + 1) / 2) * 16;
     const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
-    const bool tr_main = blockIdx.x == 0, tr_aux = (int)blockIdx.x == d.n_main;
+    const bool tr_main = main_id == 0, tr_aux = blockIdx.x == 0;
     if (threadIdx.x == 0 && tr_main) FUSED_STAMP(p, 32, 0);
     if (threadIdx.x == 0 && tr_aux) FUSED_STAMP(p, 48, 0);
 
     if (is_aux) {
         // ================================================================== aux CTA
-        const int aux_id = blockIdx.x - d.n_main;
+        const int aux_id = blockIdx.x;
         const bool active = aux_id < n_active;
         const int tile = aux_id % (d.a_tiles + 1), slice = aux_id / (d.a_tiles + 1);
         const int ks0 = active ? (int)(((long long)p.ksteps * slice) / d.aux_slices) : 0;
@@ -267,8 +267,8 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     } else {
         // ================================================================== main CTA
         const int S = p.splits;
-        const int split = blockIdx.x % S;
-        const int tile_m = blockIdx.x / S;
+        const int split = main_id % S;
+        const int tile_m = main_id / S;
         const int ks0 = (int)(((long long)p.ksteps * split) / S);
         const int ks1 = (int)(((long long)p.ksteps * (split + 1)) / S);
         const int niter = (ks1 - ks0) / p.kc;
@@ -303,11 +303,13 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         } else {
             const int a0 = split * p.na;
             stage_slab_mma(p, epi, a0, tile_m * kBM, etid);                   // B rows: no routing needed
+            uint4* us = reinterpret_cast<uint4*>(epi + p.us_off);
+            for (int v = etid; v < p.na * p.BN; v += kEpiThreads) us[v] = make_uint4(0u, 0u, 0u, 0u);
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
             if (etid == 0 && !wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);   // routing published
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 4);
             epi_barrier();
-            stage_us_mma_coherent(p, reinterpret_cast<uint4*>(epi + p.us_off), a0, ntok, etid);
+            scatter_us_mma_coherent(p, us, a0, ntok, etid);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             epi_barrier();
             if (etid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_us) : "memory");

@@ -1132,6 +1132,7 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.main.r = s.r;
     d.main.k = s.k;
     d.n_main = fp.n_main;
+    d.n_aux = fp.n_aux;
     d.a_tiles = fp.a_tiles;
     d.a_rows = s.N * s.r;
     d.aux_slices = fp.aux_slices;
@@ -1158,7 +1159,7 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = tuning().coop ? 1 : 0;
     return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mG, mX1, d));
 }
 
