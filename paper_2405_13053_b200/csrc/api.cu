@@ -266,6 +266,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "stages")) t.stages = value;
     else if (!strcmp(name, "tile_tokens")) t.tile_tokens = value;
     else if (!strcmp(name, "kc")) t.kc = value;
+    else if (!strcmp(name, "no_tma_store")) t.no_tma_store = value;
     else if (!strcmp(name, "zmax")) t.zmax = value;
     else if (!strcmp(name, "stacked_direct")) t.stacked_direct = value;
     else if (!strcmp(name, "simt_expand")) t.simt_expand = value;

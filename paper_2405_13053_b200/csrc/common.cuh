@@ -77,6 +77,7 @@ struct Tuning {
     int stages = 0;
     int tile_tokens = 0;
     int kc = 0;
+    int no_tma_store = 0;  // 1: write y with plain stores even where the TMA store applies
     int zmax = 0;          // cap on the contraction slices of the decode-batch stacked shrink (0: automatic)
     int stacked_direct = 0;  // 1: decode-batch stacked shrink without clusters, slices stored directly
     int simt_expand = 0;   // 1: keep the LoRA expand on CUDA cores even for rank 8

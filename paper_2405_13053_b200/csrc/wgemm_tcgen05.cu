@@ -85,6 +85,7 @@ struct WGemmParams {
     int na;              // adapters per split, even (two 8-wide adapters per K = 16 MMA)
     int us_in_ring;      // the token-side operand is too big for the staging area: build it in the idle ring
     int us_off;          // byte offset of the token-side operand inside the staging area (slab at slab_off)
+    int tma_store;       // 1: the finished tile is rounded to bf16 in shared memory and leaves by one TMA store
     int32_t* status;
     int pdl_wait;        // epilogue waits for the preceding grid before reading its results
     int pdl_trigger;     // let the dependent grid start as soon as this one is resident
@@ -132,6 +133,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
+}
+// Shared memory -> global tensor tile; the calling thread waits until the copy has completed.
+__device__ __forceinline__ void tma_store_2d_and_wait(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"((uint64_t)tm), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
@@ -442,7 +451,7 @@ __device__ __forceinline__ void reduce_and_finish(const WGemmParams& p, uint32_t
 
 __global__ void __launch_bounds__(kThreads)
 k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
-        const __grid_constant__ CUtensorMap tmX, const WGemmParams p) {
+        const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY, const WGemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;                 // 1024-byte aligned for the 128-byte swizzle
@@ -641,16 +650,27 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] = 0.f;
             }
+            if (p.tma_store) {
+                // final values already (the expand ran as MMAs): round once and stage as ystage[t][row]
+                __nv_bfloat16* ystage = reinterpret_cast<__nv_bfloat16*>(ring_ptr);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) part[(c + i) * kBM + row_in_tile] = v[i];
+                for (int i = 0; i < 16; ++i) ystage[(c + i) * kBM + row_in_tile] = __float2bfloat16_rn(v[i]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) part[(c + i) * kBM + row_in_tile] = v[i];
+            }
         }
+        if (p.tma_store) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> TMA read
     }
     if (threadIdx.x == 64) METEORA_STAMP(p, 4);                 // accumulators parked
     __syncwarp();
     if (S > 1) cluster_sync(); else __syncthreads();
     if (threadIdx.x == 64) METEORA_STAMP(p, 5);                 // partials of the cluster visible
 
-    if (warp >= 2 && !(p.mode == MODE_STACKED && S == 1)) {
+    if (p.tma_store) {
+        // one copy moves the whole 128 x BN tile; rows beyond d_out and tokens beyond T are clipped by the map
+        if (threadIdx.x == 64) tma_store_2d_and_wait(&tmY, ring, tile_m * kBM, tok0);
+    } else if (warp >= 2 && !(p.mode == MODE_STACKED && S == 1)) {
         const int etid = threadIdx.x - 64;
         switch (S) {
             case 1: reduce_and_finish<1>(p, ring, epi, tile_m, split, tok0, ntok, etid); break;
@@ -758,6 +778,21 @@ static int get_tensor_map(const void* ptr, int K, int rows, int box_rows, int de
     }
     *out = e.map;
     return METEORA_OK;
+}
+
+// Tensor map of y[T, d_out] (bf16, row-major) for storing a tile of 128 outputs x box_tokens tokens from
+// shared memory laid out [token][128 outputs]; not swizzled.  Needs d_out % 8 == 0 (16-byte row pitch).
+static int get_store_map(const void* y, int d_out, int T, int box_tokens, CUtensorMap* out) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return METEORA_ERR_CUDA;
+    const cuuint64_t gdim[2] = {(cuuint64_t)d_out, (cuuint64_t)T};
+    const cuuint64_t gstride[1] = {(cuuint64_t)d_out * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBM, (cuuint32_t)box_tokens};
+    const cuuint32_t estride[2] = {1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(y), gdim, gstride, box, estride,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? METEORA_OK : METEORA_ERR_CUDA;
 }
 
 static int sm_count() {
@@ -896,7 +931,8 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     return pl;
 }
 
-static int launch_wgemm(const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& mx, WGemmParams& p,
+static int launch_wgemm(const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& mx, const CUtensorMap& my,
+                        WGemmParams& p,
                         int row_tiles, const Plan& pl, bool pdl_attr, cudaStream_t st) {
     if (pl.smem > 227 * 1024) return METEORA_ERR_UNSUPPORTED_SHAPE;
     static int smem_set[64] = {};
@@ -927,7 +963,7 @@ static int launch_wgemm(const CUtensorMap& m0, const CUtensorMap& m1, const CUte
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_wgemm, m0, m1, mx, p));
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_wgemm, m0, m1, mx, my, p));
 }
 
 static int stacked_row_tiles(const meteora_shape_t& s) { return (s.N * s.r + kBM - 1) / kBM + 1; }
@@ -982,7 +1018,7 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     p.col1 = ws.col_logits;
     p.pdl_wait = 0;
     p.pdl_trigger = tuning().pdl ? 1 : 0;
-    return launch_wgemm(mA, mG, mX, p, row_tiles, pl, false, st);
+    return launch_wgemm(mA, mG, mX, mX, p, row_tiles, pl, false, st);
 }
 
 int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
@@ -1009,7 +1045,13 @@ int launch_base_lora_tc(const void* x, const void* W0, const void* B, const mete
     p.k = s.k;
     p.pdl_wait = pdl ? 1 : 0;
     p.pdl_trigger = 0;
-    return launch_wgemm(mW, mW, mX, p, row_tiles, pl, pdl, st);
+    CUtensorMap mY = mX;
+    p.tma_store = 0;
+    if (pl.splits == 1 && pl.lora_mma && s.d_out % 8 == 0 && !tuning().no_tma_store) {
+        if ((rc = get_store_map(y, s.d_out, s.T, pl.BN, &mY)) != METEORA_OK) return rc;
+        p.tma_store = 1;
+    }
+    return launch_wgemm(mW, mW, mX, mY, p, row_tiles, pl, pdl, st);
 }
 
 // ------------------------------------------------------------------------------------------------
