@@ -32,7 +32,7 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     ws.topk_idx = (int32_t*)take(T * s.k * sizeof(int32_t));
     ws.topk_w = (float*)take(T * s.k * sizeof(float));
     ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
-    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (s.T <= 256 ? 32 : 1));   // up to 32 slices for decode batches
+    ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (size_t)stacked_zsplits_bound(s.T));   // one copy per slice of the contraction axis
     // fused decode scratch: at most 296 resident CTAs (or 8 per row tile), each one tile of 128 x BN fp32
     const size_t row_tiles = ((size_t)s.d_out + 127) / 128;
     const size_t bn = (T + 15) / 16 * 16;

@@ -60,6 +60,7 @@ int launch_gemm_simt(const void* x, const void* W0, const void* B, const int32_t
 // wgemm_tcgen05.cu
 bool tc_path_supported(const meteora_shape_t& s);
 int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits);  // row pitch (floats) of u_all
+int stacked_zsplits_bound(int T);                                  // upper bound of those copies, sizes the workspace
 int tc_stacked_zsplits(const meteora_shape_t& s);                 // copies of u_all the stacked shrink writes (<= 4)
 int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const meteora_shape_t& s,
                              const Workspace& ws, cudaStream_t st);

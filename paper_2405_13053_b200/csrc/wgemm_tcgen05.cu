@@ -829,6 +829,14 @@ struct Plan {
 //   - split-K cluster size S in {1,2,4,8}: the largest that keeps one CTA per SM; if that leaves more
 //     than a quarter of the SMs idle, the next one (two CTAs per SM share the shared memory);
 //   - ring depth: whatever the shared memory left after the epilogue staging allows.
+// Upper bound of the contraction slices (copies of u_all) the stacked shrink may use for T tokens: 32 for a
+// decode batch; for larger batches as many as it takes to reach one CTA per SM with 256-token tiles.
+int stacked_zsplits_bound(int T) {
+    if (T <= 256) return kMaxZSplits;
+    const int tiles = 3 * ((T + 255) / 256);
+    return std::min(kMaxZSplits, std::max(1, 148 / tiles));
+}
+
 static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k) {
     const Tuning& tn = tuning();
     Plan pl = {};
@@ -861,6 +869,11 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
         }
         const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits) : (tn.stacked_direct ? kMaxZSplits : 4);
         pl.zsplits = std::min(zcap, std::max(1, ksteps / splits / 2));
+    } else if (!lora && splits == 1) {
+        // Stacked shrink of a prefill batch with too few tiles to fill the device: slices of the contraction
+        // axis over grid z, stored straight to u_all[z] (same bound as the workspace: stacked_zsplits_bound).
+        const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits) : kMaxZSplits;
+        pl.zsplits = std::min(std::min(zcap, stacked_zsplits_bound(T)), std::max(1, ksteps / 4));
     }
     const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
