@@ -869,11 +869,16 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
         }
         const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits) : (tn.stacked_direct ? kMaxZSplits : 4);
         pl.zsplits = std::min(zcap, std::max(1, ksteps / splits / 2));
-    } else if (!lora && splits == 1) {
-        // Stacked shrink of a prefill batch with too few tiles to fill the device: slices of the contraction
-        // axis over grid z, stored straight to u_all[z] (same bound as the workspace: stacked_zsplits_bound).
+    } else if (!lora) {
+        // Stacked shrink of a prefill batch: never a cluster (summing 128 x 256 partial tiles through
+        // distributed shared memory costs more than the product itself); if the tiles leave SMs idle, slices
+        // of the contraction axis over grid z, stored straight to u_all[z] and added by the selection kernel
+        // (same bound as the workspace: stacked_zsplits_bound).
+        splits = 1;
+        pl.splits = 1;
         const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits) : kMaxZSplits;
-        pl.zsplits = std::min(std::min(zcap, stacked_zsplits_bound(T)), std::max(1, ksteps / 4));
+        const int fill = std::max(1, sms / tiles);
+        pl.zsplits = std::min(std::min(zcap, std::min(fill, stacked_zsplits_bound(T))), std::max(1, ksteps / 4));
     }
     const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
