@@ -841,7 +841,11 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     const Tuning& tn = tuning();
     Plan pl = {};
     const int ksteps = (K + kBK - 1) / kBK;
+    // tokens per tile: a decode batch is one tile; a prefill batch uses 256-token tiles unless those leave SMs
+    // idle, then 128 (prefill tiles are never split along the contraction axis: summing 128 x 256 partial
+    // tiles across a cluster costs more than it gains)
     int bn = tn.tile_tokens > 0 ? tn.tile_tokens : (T <= 256 ? (T + 15) / 16 * 16 : 256);
+    if (tn.tile_tokens == 0 && T > 256 && row_tiles * ((T + 255) / 256) < sm_count()) bn = 128;
     bn = std::min(256, std::max(16, (bn + 15) / 16 * 16));
     pl.BN = bn;
     pl.n_tiles = (T + bn - 1) / bn;
@@ -850,7 +854,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     int splits = 1;
     if (tn.splits > 0) {
         splits = tn.splits >= 8 ? 8 : tn.splits >= 4 ? 4 : tn.splits >= 2 ? 2 : 1;
-    } else {
+    } else if (pl.n_tiles == 1) {
         while (splits < 8 && tiles * splits * 2 <= sms) splits *= 2;
         if (splits < 8 && tiles * splits * 4 < sms * 3 && tiles * splits * 2 <= 2 * sms) splits *= 2;
     }
