@@ -65,8 +65,11 @@ def measured_peaks():
 
 
 def kernel_sha():
-    with open(os.path.join(ROOT, "paper_2405_13053_b200", "csrc", "wgemm_tcgen05.cu"), "rb") as fh:
-        return hashlib.sha256(fh.read()).hexdigest()[:16]
+    h = hashlib.sha256()
+    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "select.cuh"):
+        with open(os.path.join(ROOT, "paper_2405_13053_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
 
 
 class ClockSampler:
@@ -287,26 +290,43 @@ def run_ours(args):
     check_status()
     e2e_value = tokens_per_step * K / (ms_e2e * 1e-3)
 
-    # ---- dominant kernel: event pairs around the base-product launch of every call, same launches
-    prof_steps = min(K, 50)
-    step_device()
-    torch.cuda.synchronize()
-    mb.meteora_profile_begin(prof_steps * R)
-    for _ in range(prof_steps):
+    # ---- dominant kernel.  Which kernels a call launches depends on the shape (meteora_describe_plan):
+    #   single-launch decode kernel: one launch is the whole call, so its average duration over the timed region
+    #     is the graph-replayed region itself divided by the launches (idle gaps between launches included);
+    #   three-launch chain: event pairs around the base-product launch of every call, in a second region of the
+    #     same launches issued behind a long blocker kernel so that the host is never the bottleneck.
+    plan = mb.meteora_describe_plan(shape)
+    single_launch = "path=fused_decode" in plan
+    launches_per_call = 1 if single_launch else 3
+    if single_launch:
+        kernel_name = "k_decode_fused (base product + stacked shrink + selection + LoRA expand, one launch per call)"
+        kernel_ms, kernel_launches = ms_total, K * R
+    else:
+        kernel_name = "k_wgemm (base product + LoRA expand epilogue)"
+        prof_steps = min(K, 8)
         step_device()
-    kernel_ms, kernel_launches = mb.meteora_profile_end()
+        torch.cuda.synchronize()
+        blocker = torch.empty((8192, 8192), dtype=dt, device="cuda")
+        for _ in range(6):
+            torch.matmul(blocker, blocker)                      # ~6 ms of queued work ahead of the timed launches
+        mb.meteora_profile_begin(prof_steps * R)
+        for _ in range(prof_steps):
+            step_device()
+        kernel_ms, kernel_launches = mb.meteora_profile_end()
+        del blocker
     check_status()
 
     # ---- algorithmic bytes (adapters actually selected, from the realised routing of module 0)
     idx0, _ = mb.meteora_workspace_routing(shape, mods[0]["ws"])
     touched = int(torch.unique(idx0).numel())
-    bytes_kernel = (D_IN * D_OUT + touched * D_OUT * RANK + T * (D_IN + D_OUT)) * es
-    bytes_path = bytes_kernel + (N_ADAPTERS * D_IN + touched * RANK * D_IN) * es
+    bytes_base = (D_IN * D_OUT + touched * D_OUT * RANK + T * (D_IN + D_OUT)) * es
+    bytes_path = bytes_base + (N_ADAPTERS * D_IN + touched * RANK * D_IN) * es
+    bytes_kernel = bytes_path if single_launch else bytes_base
     peak, peak_kind = measured_peaks()
     per_launch_s = kernel_ms * 1e-3 / max(kernel_launches, 1)
     achieved = bytes_kernel / per_launch_s / 1e9
     traffic = None
-    if NCU_TRAFFIC["kernel_sha"] == kernel_sha():
+    if NCU_TRAFFIC["kernel_sha"] == kernel_sha() and single_launch:
         traffic = NCU_TRAFFIC["bytes_per_launch"].get(str(T))
     per_call_s = ms_total * 1e-3 / (K * R)
 
@@ -319,12 +339,12 @@ def run_ours(args):
                    "tokens_per_module": T, "modules_per_step": R, "launch": mode, "e2e_launch": mode_e2e,
                    "l2": f"weights of the {R} modules total {R * bytes_path / 1e6:.0f} MB > 126 MB L2, "
                          "so no weight is L2-resident between visits",
-                   "parallelism": f"token-sharded replicas x{world}, no collective"},
+                   "parallelism": f"token-sharded replicas x{world}, no collective", "plan": plan},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": R * T * D_IN * es,
                 "d2h_bytes_per_step": R * T * D_OUT * es, "ms_per_step": ms_e2e / K},
-        "gpu_launches": 3 * R * K,
+        "gpu_launches": launches_per_call * R * K,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "k_wgemm (base product + LoRA epilogue)", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved,
                      "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "algorithmic_bytes_per_launch": bytes_kernel,
                      "us_per_launch": per_launch_s * 1e6, "launches_timed": kernel_launches},
