@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--launch", choices=["graph", "stream"], default="graph")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target length of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every (shape, T) of configs 1-3 instead of the headline step; one JSON line each")
     return ap.parse_args()
 
 
@@ -62,6 +64,15 @@ def measured_peaks():
         return float(p["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def measured_tensor_peak():
+    """Sustained dense bf16 TFLOP/s (the kernels here are timed inside long loops)."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1400.0, "fallback"
 
 
 def kernel_sha():
@@ -372,9 +383,100 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------- sweep
+def run_sweep(args):
+    """Per-call time of meteora_linear_forward for every shape of configs 1-3 (device-resident inputs, graph
+    replay over enough independent modules that HBM-bound shapes never find their weights in L2)."""
+    import ctypes
+
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import build as lib_build
+    from paper_2405_13053_b200 import workloads
+
+    lib_build.build_library()
+    lib = mb.load_library()
+    torch.cuda.set_device(0)
+    hbm, _ = measured_peaks()
+    tc, _ = measured_tensor_peak()
+    dt, es = torch.bfloat16, 2
+    cases = [("config1", "q_proj", 4096, 4096, T, "rms") for T in workloads.CONFIG1_T]
+    for name, (di, do) in workloads.CONFIG2_SHAPES.items():
+        cases += [("config2", name, di, do, T, "clusters") for T in workloads.CONFIG2_T]
+    for name, (di, do) in workloads.CONFIG3_SHAPES.items():
+        cases += [("config3", name, di, do, T, "normal") for T in workloads.CONFIG3_T]
+    for cfg, name, d_in, d_out, T, x_kind in cases:
+        w_bytes = d_in * d_out * es
+        R = max(1, min(16, int(600e6 // w_bytes))) if T <= 256 else 1
+        shape = mb.make_shape(T, d_in, d_out, N_ADAPTERS, RANK, TOPK, dt)
+        g = torch.Generator(device="cuda").manual_seed(7)
+        x_np = workloads.make_x(T, d_in, x_kind, 5, "bf16")          # token statistics of the config; weights on device
+        mods = []
+        for i in range(R):
+            m = {"x": torch.from_numpy(x_np).to(dt).cuda(),
+                 "W0": (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt),
+                 "A": ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt),
+                 "B": (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt),
+                 "Wg": (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt),
+                 "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": mb.alloc_workspace(shape)}
+            mods.append(m)
+
+        def step():
+            for m in mods:
+                rc = lib.meteora_linear_forward(m["x"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(),
+                                                m["B"].data_ptr(), m["Wg"].data_ptr(), ctypes.byref(shape),
+                                                m["y"].data_ptr(), m["ws"].data_ptr(), m["ws"].numel(),
+                                                torch.cuda.current_stream().cuda_stream)
+                if rc != 0:
+                    raise mb.MeteoraError(rc, "meteora_linear_forward")
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        iters = 100 if T <= 256 else 20
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        for m in mods:
+            st = mb.meteora_workspace_status(m["ws"])
+            if st != 0:
+                raise mb.MeteoraError(st, "device status")
+        us = e0.elapsed_time(e1) * 1e3 / (iters * R)
+        idx0, _ = mb.meteora_workspace_routing(shape, mods[0]["ws"])
+        touched = int(torch.unique(idx0).numel())
+        counts = torch.bincount(idx0.flatten().long(), minlength=N_ADAPTERS).tolist()
+        nbytes = (d_in * d_out + N_ADAPTERS * d_in + touched * RANK * (d_in + d_out) + T * (d_in + d_out)) * es
+        flops = 2.0 * T * d_in * d_out + 2.0 * T * N_ADAPTERS * d_in + 2.0 * T * TOPK * RANK * (d_in + d_out)
+        t_mem, t_tc = nbytes / hbm / 1e3, flops / tc / 1e6                       # microseconds
+        bound = "hbm" if t_mem >= t_tc else "tensor"
+        print(json.dumps({"config": cfg, "shape": f"{name} {d_in}->{d_out}", "T": T, "us_per_call": round(us, 2),
+                          "tokens_per_s": round(T / us * 1e6), "bound": bound,
+                          "roofline_us": round(max(t_mem, t_tc), 2), "frac_of_roofline": round(max(t_mem, t_tc) / us, 3),
+                          "achieved": round(nbytes / us / 1e3, 1) if bound == "hbm" else round(flops / us / 1e6, 1),
+                          "unit": "GB/s" if bound == "hbm" else "TFLOP/s", "adapters_touched": touched,
+                          "max_share_of_slots": round(max(counts) / max(1, T * TOPK), 3), "modules": R,
+                          "plan": mb.meteora_describe_plan(shape).split(" fused_refused")[0]}), flush=True)
+        del mods, graph
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
