@@ -36,6 +36,7 @@ struct DecodeParams {
     float* part_g;         // [row tile][split][BN][128] fp32 partial accumulator tiles of the base product
     int32_t* tile_ctr;     // [row tiles] partials written per tile
     int row_tiles;
+    int overlap;           // launched with programmatic stream serialization: prefetch weights, then wait
 };
 
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
@@ -191,6 +192,40 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int half = ((p.BN / 16 + 1) / 2) * 16;
     const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
     const bool tr_main = main_id == 0, tr_aux = blockIdx.x == 0;
+
+    if (d.overlap) {
+        // Overlap with the previous kernel of the stream: it may still be running.  Until it has completed
+        // (griddepcontrol.wait) nothing it could have written is read and nothing is written; the weights of
+        // this CTA are only pulled into L2, which changes no value anyone can observe.
+        if (threadIdx.x == 0) {
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            if (is_aux) {
+                if ((int)blockIdx.x < n_active) {
+                    const int tile = blockIdx.x % (d.a_tiles + 1), slice = blockIdx.x / (d.a_tiles + 1);
+                    const int k0 = (int)(((long long)p.ksteps * slice) / d.aux_slices);
+                    const int k1 = (int)(((long long)p.ksteps * (slice + 1)) / d.aux_slices);
+                    const bool is_gate = tile >= d.a_tiles;
+                    for (int ks = k0; ks < k1; ++ks) {
+                        if (p.maps3d) tma_prefetch_3d(is_gate ? &tmG : &tmA, 0, is_gate ? 0 : tile * kBM, ks);
+                        else tma_prefetch_2d(is_gate ? &tmG : &tmA, ks * kBK, is_gate ? 0 : tile * kBM);
+                    }
+                }
+            } else {
+                const int S = p.splits, split = main_id % S, tile_m = main_id / S;
+                const int k0 = (int)(((long long)p.ksteps * split) / S);
+                const int k1 = (int)(((long long)p.ksteps * (split + 1)) / S);
+                for (int ks = k0; ks < k1; ks += p.kc) {
+                    if (p.maps3d) tma_prefetch_3d(&tmW0, 0, tile_m * kBM, ks);
+                    else tma_prefetch_2d(&tmW0, ks * kBK, tile_m * kBM);
+                }
+                // B rows of this split's adapters for the tile's 128 output rows (2 KB per adapter)
+                const int row0 = tile_m * kBM, rows = min(kBM, p.d_out - row0);
+                for (int a = split * p.na; a < min(p.N, (split + 1) * p.na); ++a)
+                    bulk_prefetch_l2(p.B + ((size_t)a * p.d_out + row0) * 8, (uint32_t)rows * 16u);
+            }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
     if (threadIdx.x == 0 && tr_main) FUSED_STAMP(p, 32, 0);
     if (threadIdx.x == 0 && tr_aux) FUSED_STAMP(p, 48, 0);
 

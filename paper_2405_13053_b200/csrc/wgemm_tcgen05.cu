@@ -135,6 +135,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
         : "memory");
 }
 // Shared memory -> global tensor tile; the calling thread waits until the copy has completed.
+// Tile of a tensor map into L2 only (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tm, int c0, int c1) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tm, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(c0), "r"(c1),
+                 "r"(c2)
+                 : "memory");
+}
+// `bytes` (a multiple of 16) from a 16-byte aligned global address into L2 only.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* gptr, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void tma_store_2d_and_wait(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"((uint64_t)tm), "r"(src), "r"(c0), "r"(c1)
@@ -816,7 +830,7 @@ int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits) {
 }
 
 struct Plan;
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k);
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, size_t budget = 0);
 
 struct Plan {
     int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
@@ -837,7 +851,7 @@ int stacked_zsplits_bound(int T) {
     return std::min(kMaxZSplits, std::max(1, 148 / tiles));
 }
 
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k) {
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, size_t budget) {
     const Tuning& tn = tuning();
     Plan pl = {};
     const int ksteps = (K + kBK - 1) / kBK;
@@ -886,7 +900,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     }
     const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
-    const size_t total_budget = two_per_sm ? 112 * 1024 : 226 * 1024;
+    const size_t total_budget = budget ? budget : two_per_sm ? 112 * 1024 : 226 * 1024;
 
     // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
     const int tile_tokens = std::min(T, bn);
@@ -1108,7 +1122,7 @@ struct FusedPlan {
     bool ok;
     int why;   // why not: 1 knob/shape, 2 too many row tiles, 3 several token tiles, 4 residency, 5 operand sizes
     Plan main;
-    int row_tiles, n_main, n_aux, a_tiles, aux_slices, aux_stages;
+    int row_tiles, n_main, n_aux, a_tiles, aux_slices, aux_stages, overlap;
 };
 
 static FusedPlan make_fused_plan(const meteora_shape_t& s) {
@@ -1123,7 +1137,8 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.row_tiles = (s.d_out + kBM - 1) / kBM;
     fp.why = 2;
     if (fp.row_tiles > kMaxFusedRowTiles) return fp;
-    fp.main = make_plan(fp.row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
+    fp.overlap = tuning().overlap ? 1 : 0;
+    fp.main = make_plan(fp.row_tiles, s.T, s.d_in, true, s.N, s.r, s.k, fp.overlap ? 110 * 1024 : 0);
     fp.why = 3;
     if (fp.main.n_tiles != 1) return fp;
     fp.why = 5;
@@ -1131,7 +1146,9 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.why = 4;
     const int S = fp.main.splits;
     fp.n_main = fp.row_tiles * S;
-    const int capacity = max_resident_ctas(fp.main.smem);
+    int capacity = max_resident_ctas(fp.main.smem);
+    // overlapped calls: this call and the next one share the SMs, so aim at one CTA per SM for each
+    if (fp.overlap && capacity >= 2 * sm_count() && fp.n_main + 3 <= sm_count()) capacity = sm_count();
     fp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
     const int aux_tiles = fp.a_tiles + 1;
     const int n_aux = std::min(capacity - fp.n_main, 24);
@@ -1162,9 +1179,9 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     if (fp.ok)
         return snprintf(buf, n,
                         "path=fused_decode launches=1 main_ctas=%d splits=%d aux_ctas=%d aux_slices=%d tile_tokens=%d "
-                        "stages=%d kc=%d smem=%zu resident_ctas=%d",
+                        "stages=%d kc=%d smem=%zu resident_ctas=%d overlap=%d",
                         fp.n_main, fp.main.splits, fp.n_aux, fp.aux_slices, fp.main.BN, fp.main.stages, fp.main.kc,
-                        fp.main.smem, max_resident_ctas(fp.main.smem));
+                        fp.main.smem, max_resident_ctas(fp.main.smem), fp.overlap);
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     return snprintf(buf, n,
@@ -1225,10 +1242,16 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
-    attr[0].val.cooperative = 1;
+    if (fp.overlap) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
+        attr[0].val.cooperative = 1;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = tuning().coop ? 1 : 0;
+    cfg.numAttrs = (fp.overlap || tuning().coop) ? 1 : 0;
+    d.overlap = fp.overlap;
     return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mG, mX1, d));
 }
 
