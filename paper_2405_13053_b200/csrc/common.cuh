@@ -86,8 +86,6 @@ struct Tuning {
     int pdl = 1;
     int fused = 1;           // 0: never use the single-launch decode kernel
     int coop = 1;            // 0 (measurement only): launch it without the co-residency guarantee
-    int overlap = 0;         // 1: the decode kernel takes half an SM and is launched with programmatic stream
-                             // serialization: the next call's CTAs prefetch their weights into L2 meanwhile
     int fused_refused = 0;   // cooperative launches the driver refused (the chain ran instead)
 };
 Tuning& tuning();

@@ -3,16 +3,17 @@
 //
 // The grid holds two kinds of CTAs, all resident at the same time (cooperative launch, no clusters):
 //   - main CTAs, S per 128-row tile of W0 along the contraction axis: stream W0 through TMA + tcgen05 into
-//     TMEM, add the LoRA expand of their share of the adapters as extra MMAs (Eq. 2), write the partial
-//     accumulator tile to an fp32 scratch (it stays in L2) and, once the tile's S partials are in, each sums
-//     its slice of the rows in split order and stores y;
+//     TMEM, write the partial accumulator tile to an fp32 scratch (it stays in L2) and, once the tile's S
+//     partials are in, each sums its slice of the rows in split order, adds the LoRA expand of those rows
+//     (Eq. 2: the B rows of every adapter wait in shared memory, the routing arrives from the aux CTAs) and
+//     stores y;
 //   - a few aux CTAs on the SMs the main CTAs leave free: each computes a slice of the stacked shrink
 //     [A_0..A_{N-1}; Wg] x (every adapter's A_i x and the gate logits, Sec. 3.1) on the same main loop and
 //     writes it as an fp32 partial; once all partials are in, the aux CTAs share the tokens and run the
 //     top-k selection and the softmax over the selected logits (Eq. 3), publishing topk_idx, topk_w, uw.
 // The main CTAs hold their first loads back until the aux CTAs have issued theirs, so the 2 MB of the shrink
-// are ahead of the 33 MB of W0 in the memory queues; they need the routing only for the expand at the end of
-// their main loop.  Every wait is bounded; on expiry the status word is set and the kernel drains.  The
+// are ahead of the 33 MB of W0 in the memory queues; they need the routing only after their main loop and
+// the exchange of the partial tiles.  Every wait is bounded; on expiry the status word is set and the kernel drains.  The
 // counters live in the workspace header and are re-armed by the last CTA to exit.
 #pragma once
 
@@ -36,7 +37,7 @@ struct DecodeParams {
     float* part_g;         // [row tile][split][BN][128] fp32 partial accumulator tiles of the base product
     int32_t* tile_ctr;     // [row tiles] partials written per tile
     int row_tiles;
-    int overlap;           // launched with programmatic stream serialization: prefetch weights, then wait
+    int trace_call;        // trace builds: which record of the trace buffer this launch fills
 };
 
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
@@ -54,34 +55,91 @@ __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
     return true;
 }
 
-// Token-side operand of the tensor-core expand: the caller has zeroed it; scatter bf16(w_j * A_e x_t) of the
-// slots whose adapter belongs to this CTA, reading the routing with loads that bypass L1 (it was written
-// by other CTAs of this same kernel).
-__device__ __forceinline__ void scatter_us_mma_coherent(const WGemmParams& p, uint4* us, int a0, int ntok, int etid) {
-    const int slots = ntok * p.k;
-    const float4* uw4 = reinterpret_cast<const float4*>(p.uw);
-    for (int i = etid; i < slots; i += kEpiThreads) {
-        const int a = __ldcg(p.topk_idx + i) - a0;
-        if (a >= 0 && a < p.na) {
-            const float4 lo = __ldcg(uw4 + 2 * i), hi = __ldcg(uw4 + 2 * i + 1);
-            const __nv_bfloat162 q0 = __floats2bfloat162_rn(lo.x, lo.y), q1 = __floats2bfloat162_rn(lo.z, lo.w);
-            const __nv_bfloat162 q2 = __floats2bfloat162_rn(hi.x, hi.y), q3 = __floats2bfloat162_rn(hi.z, hi.w);
-            uint4 val;
-            val.x = *reinterpret_cast<const uint32_t*>(&q0);
-            val.y = *reinterpret_cast<const uint32_t*>(&q1);
-            val.z = *reinterpret_cast<const uint32_t*>(&q2);
-            val.w = *reinterpret_cast<const uint32_t*>(&q3);
-            us[a * p.BN + i / p.k] = val;
+// B rows [row0, row0 + nrows) of every adapter as slab[e][row][8 bf16]; rows past d_out are zero.
+__device__ __forceinline__ void stage_slab_rows(const WGemmParams& p, uint4* slab, int row0, int nrows, int etid) {
+    const uint4* Bg = reinterpret_cast<const uint4*>(p.B);
+    const int total = p.N * nrows;
+    for (int i = etid; i < total; i += kEpiThreads) {
+        const int e = i / nrows, o = row0 + (i - e * nrows);
+        slab[i] = o < p.d_out ? __ldg(Bg + (size_t)e * p.d_out + o) : make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+// Last step of a main CTA: rows [row_lo, row_lo + 4 * nq) of the tile, all tokens.  Work items are (token,
+// group of 4 rows); a thread keeps U items in flight: the C partial tiles' values first (one round trip to
+// L2), then their sum in split order, the expand of Eq. 2 from the staged B rows and the routing in shared
+// memory, one rounding to bf16 and the store.  `before_compute` runs once, after the first loads are issued.
+template <int C, int U, typename F>
+__device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* part, size_t part_stride, bool from_l2,
+                                            int tile_row0, int row_lo, int nq, int ntok, const uint4* slab,
+                                            int slab_rows, const float* s_uw, const int* s_idx, int etid,
+                                            F before_compute) {
+    const int items = nq * ntok;
+    const float4* s_uw4 = reinterpret_cast<const float4*>(s_uw);
+    for (int base = 0; base < items; base += kEpiThreads * U) {
+        float4 v[U][C];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int it = min(base + etid + u * kEpiThreads, items - 1);
+            const int t = it / nq, ql = it - t * nq;
+            const float* a = part + (size_t)t * kBM + row_lo + ql * 4;
+#pragma unroll
+            for (int q = 0; q < C; ++q) {
+                const float4* src = reinterpret_cast<const float4*>(a + q * part_stride);
+                v[u][q] = from_l2 ? __ldcg(src) : *src;
+            }
+        }
+        if (base == 0) before_compute();
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int it = base + etid + u * kEpiThreads;
+            if (it >= items) break;
+            const int t = it / nq, ql = it - t * nq;
+            float4 acc = v[u][0];
+#pragma unroll
+            for (int q = 1; q < C; ++q) {
+                acc.x += v[u][q].x;
+                acc.y += v[u][q].y;
+                acc.z += v[u][q].z;
+                acc.w += v[u][q].w;
+            }
+            for (int j = 0; j < p.k; ++j) {
+                const int slot = t * p.k + j;
+                const float4 u0 = s_uw4[2 * slot], u1 = s_uw4[2 * slot + 1];
+                const uint4* b = slab + (size_t)s_idx[slot] * slab_rows + ql * 4;
+                fma8(b[0], u0, u1, acc.x);
+                fma8(b[1], u0, u1, acc.y);
+                fma8(b[2], u0, u1, acc.z);
+                fma8(b[3], u0, u1, acc.w);
+            }
+            const int o = tile_row0 + row_lo + ql * 4;
+            __nv_bfloat16* dst = p.y + (size_t)t * p.d_out + o;
+            if ((p.d_out & 3) == 0 && o + 3 < p.d_out) {
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(dst) = pk;
+            } else {
+                const float f[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (o + i < p.d_out) dst[i] = __float2bfloat16_rn(f[i]);
+            }
         }
     }
 }
 
 #ifdef METEORA_TRACE
-#define FUSED_STAMP(p, base, slot)                                                  \
-    do {                                                                            \
-        unsigned long long t_;                                                      \
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                      \
-        (p).status[(base) + (slot)] = (int)(t_ & 0x7FFFFFFF);                       \
+// Trace build only: every CTA stamps the global nanosecond timer at the points of interest.
+constexpr int kTraceCalls = 32, kTraceCtas = 256, kTraceSlots = 16;
+__device__ unsigned long long g_fused_trace[kTraceCalls * kTraceCtas * kTraceSlots];
+#define FUSED_STAMP(p, base, slot)                                                                   \
+    do {                                                                                             \
+        unsigned long long t_;                                                                       \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                       \
+        if (blockIdx.x < kTraceCtas)                                                                 \
+            g_fused_trace[((d.trace_call % kTraceCalls) * kTraceCtas + blockIdx.x) * kTraceSlots + (slot)] = t_; \
     } while (0)
 #else
 #define FUSED_STAMP(p, base, slot) do { } while (0)
@@ -191,41 +249,14 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int ntok = min(p.BN, p.T);
     const int half = ((p.BN / 16 + 1) / 2) * 16;
     const int c_begin = warp < 6 ? 0 : half, c_end = warp < 6 ? half : p.BN;
+#ifdef METEORA_TRACE
+    const bool tr_main = !is_aux, tr_aux = is_aux;
+#else
     const bool tr_main = main_id == 0, tr_aux = blockIdx.x == 0;
+#endif
 
-    if (d.overlap) {
-        // Overlap with the previous kernel of the stream: it may still be running.  Until it has completed
-        // (griddepcontrol.wait) nothing it could have written is read and nothing is written; the weights of
-        // this CTA are only pulled into L2, which changes no value anyone can observe.
-        if (threadIdx.x == 0) {
-            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-            if (is_aux) {
-                if ((int)blockIdx.x < n_active) {
-                    const int tile = blockIdx.x % (d.a_tiles + 1), slice = blockIdx.x / (d.a_tiles + 1);
-                    const int k0 = (int)(((long long)p.ksteps * slice) / d.aux_slices);
-                    const int k1 = (int)(((long long)p.ksteps * (slice + 1)) / d.aux_slices);
-                    const bool is_gate = tile >= d.a_tiles;
-                    for (int ks = k0; ks < k1; ++ks) {
-                        if (p.maps3d) tma_prefetch_3d(is_gate ? &tmG : &tmA, 0, is_gate ? 0 : tile * kBM, ks);
-                        else tma_prefetch_2d(is_gate ? &tmG : &tmA, ks * kBK, is_gate ? 0 : tile * kBM);
-                    }
-                }
-            } else {
-                const int S = p.splits, split = main_id % S, tile_m = main_id / S;
-                const int k0 = (int)(((long long)p.ksteps * split) / S);
-                const int k1 = (int)(((long long)p.ksteps * (split + 1)) / S);
-                for (int ks = k0; ks < k1; ks += p.kc) {
-                    if (p.maps3d) tma_prefetch_3d(&tmW0, 0, tile_m * kBM, ks);
-                    else tma_prefetch_2d(&tmW0, ks * kBK, tile_m * kBM);
-                }
-                // B rows of this split's adapters for the tile's 128 output rows (2 KB per adapter)
-                const int row0 = tile_m * kBM, rows = min(kBM, p.d_out - row0);
-                for (int a = split * p.na; a < min(p.N, (split + 1) * p.na); ++a)
-                    bulk_prefetch_l2(p.B + ((size_t)a * p.d_out + row0) * 8, (uint32_t)rows * 16u);
-            }
-        }
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-    }
+    if (threadIdx.x == 0 && tr_main) FUSED_STAMP(p, 32, 8);
+    if (threadIdx.x == 0 && tr_aux) FUSED_STAMP(p, 48, 5);
     if (threadIdx.x == 0 && tr_main) FUSED_STAMP(p, 32, 0);
     if (threadIdx.x == 0 && tr_aux) FUSED_STAMP(p, 48, 0);
 
@@ -308,7 +339,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         const int ks1 = (int)(((long long)p.ksteps * (split + 1)) / S);
         const int niter = (ks1 - ks0) / p.kc;
         const RingGeom geom = {ring, bar_base, x_tile_bytes, stage_bytes, p.stages, p.kc, p.maps3d};
-        const uint32_t bar_acc = bar_base + 2 * p.stages * 8, bar_us = bar_acc + 16;
+        const uint32_t bar_acc = bar_base + 2 * p.stages * 8;
         const size_t part_stride = (size_t)p.BN * kBM;                       // floats per partial tile
         float* my_part = d.part_g + ((size_t)tile_m * S + split) * part_stride;
         if (warp == 0) {
@@ -323,31 +354,17 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             if (lane == 0) {
                 bool ok = fused_mma(geom, tmem_base, idesc, niter);
                 if (tr_main) FUSED_STAMP(p, 32, 2);
-                if (ok) ok = mbar_wait(bar_us, 0);                            // operands of the expand staged
-                if (ok) {
-                    tc_fence_after();
-                    const uint32_t slab_a = smem_u32(epi + p.slab_off), us_a = smem_u32(epi + p.us_off);
-                    const uint32_t ka = kBM * 16, kb = p.BN * 16;
-                    for (int m = 0; m < p.na / 2; ++m)
-                        umma_bf16(tmem_base, smem_desc_plain(slab_a + 2 * m * ka, ka, 128),
-                                  smem_desc_plain(us_a + 2 * m * kb, kb, 128), idesc, (niter | m) != 0);
-                }
                 umma_commit(bar_acc);
                 if (!ok) flag_error(p, 2, 200);
             }
         } else {
-            const int a0 = split * p.na;
-            stage_slab_mma(p, epi, a0, tile_m * kBM, etid);                   // B rows: no routing needed
-            uint4* us = reinterpret_cast<uint4*>(epi + p.us_off);
-            for (int v = etid; v < p.na * p.BN; v += kEpiThreads) us[v] = make_uint4(0u, 0u, 0u, 0u);
+            // B rows of the slice of the tile this CTA finishes, for every adapter: no routing needed yet
+            const int nrows = kBM / S, row_lo = nrows * split;
+            uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
+            float* s_uw = reinterpret_cast<float*>(epi + p.uw_off);
+            int* s_idx = reinterpret_cast<int*>(epi + p.idx_off);
+            stage_slab_rows(p, slab, tile_m * kBM + row_lo, nrows, etid);
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
-            if (etid == 0 && !wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);   // routing published
-            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 4);
-            epi_barrier();
-            scatter_us_mma_coherent(p, us, a0, ntok, etid);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            epi_barrier();
-            if (etid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_us) : "memory");
             bool acc_ok = mbar_wait(bar_acc, 0);
             if (!acc_ok && lane == 0) flag_error(p, 3, 300);
             acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
@@ -367,60 +384,35 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 }
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    if (S == 1 || c + i < ntok) part[(c + i) * kBM + row_in_tile] = v[i];
+                    if (c + i < ntok) part[(c + i) * kBM + row_in_tile] = v[i];
             }
             epi_barrier();
-            if (S > 1 && etid == 0) {
-                __threadfence();
-                atomicAdd(d.tile_ctr + tile_m, 1);
-                if (!wait_counter(d.tile_ctr + tile_m, S)) flag_error(p, 4, 900);   // all partials of the tile in
+            if (etid == 0) {
+                if (S > 1) {
+                    __threadfence();
+                    atomicAdd(d.tile_ctr + tile_m, 1);
+                }
+                if (!wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);              // routing published
+                if (tr_main) FUSED_STAMP(p, 32, 4);
+                if (S > 1 && !wait_counter(d.tile_ctr + tile_m, S)) flag_error(p, 4, 900);  // all partials of the tile in
+                if (tr_main) FUSED_STAMP(p, 32, 6);
             }
-            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 6);
             epi_barrier();
-            // sum the slice of rows this CTA owns over the S partials, in split order, and store y
-            const int P = 64 / S, TPP = kEpiThreads / P, NROWS = kBM / S;
-            const int pr = etid % P, tg = etid / P;
-            const int rit = NROWS * split + 2 * pr;
-            const int o = tile_m * kBM + rit;
             const float* src = S > 1 ? d.part_g + (size_t)tile_m * S * part_stride : part;
-            for (int t0 = tg; t0 < ntok; t0 += 4 * TPP) {
-                float2 acc[4], v[4][8];
-                // all partial loads of four tokens first (one L2 round trip), then the sums in split order
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int t = min(t0 + u * TPP, ntok - 1);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        v[u][q] = make_float2(0.f, 0.f);
-                        if (q < S) {
-                            const float2* a = reinterpret_cast<const float2*>(src + q * part_stride + t * kBM + rit);
-                            v[u][q] = S > 1 ? __ldcg(a) : *a;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    acc[u] = make_float2(0.f, 0.f);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (q < S) {
-                            acc[u].x += v[u][q].x;
-                            acc[u].y += v[u][q].y;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int t = t0 + u * TPP;
-                    if (t >= ntok) break;
-                    __nv_bfloat16* dst = p.y + (size_t)t * p.d_out + o;
-                    if (o + 1 < p.d_out && (p.d_out & 1) == 0) {
-                        *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(acc[u].x, acc[u].y);
-                    } else {
-                        if (o < p.d_out) dst[0] = __float2bfloat16_rn(acc[u].x);
-                        if (o + 1 < p.d_out) dst[1] = __float2bfloat16_rn(acc[u].y);
-                    }
-                }
+            auto stage_routing = [&]() {
+                // the routing was written by other CTAs of this kernel: loads that bypass L1
+                const int slots = ntok * p.k;
+                for (int i = etid; i < slots; i += kEpiThreads) s_idx[i] = min(max(__ldcg(p.topk_idx + i), 0), p.N - 1);
+                const float4* uw4 = reinterpret_cast<const float4*>(p.uw);
+                for (int i = etid; i < 2 * slots; i += kEpiThreads) reinterpret_cast<float4*>(s_uw)[i] = __ldcg(uw4 + i);
+                epi_barrier();
+            };
+            const int nq = nrows / 4;
+            switch (S) {
+                case 1: finish_rows<1, 4>(p, src, part_stride, false, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
+                case 2: finish_rows<2, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
+                case 4: finish_rows<4, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
+                default: finish_rows<8, 2>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
             }
         }
     }

@@ -85,6 +85,7 @@ struct WGemmParams {
     int na;              // adapters per split, even (two 8-wide adapters per K = 16 MMA)
     int us_in_ring;      // the token-side operand is too big for the staging area: build it in the idle ring
     int us_off;          // byte offset of the token-side operand inside the staging area (slab at slab_off)
+    int idx_off;         // single-launch decode kernel: byte offset of the staged adapter indices (weights at uw_off)
     int tma_store;       // 1: the finished tile is rounded to bf16 in shared memory and leaves by one TMA store
     int32_t* status;
     int pdl_wait;        // epilogue waits for the preceding grid before reading its results
@@ -135,20 +136,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
         : "memory");
 }
 // Shared memory -> global tensor tile; the calling thread waits until the copy has completed.
-// Tile of a tensor map into L2 only (no shared-memory destination, nothing to wait for).
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tm, int c0, int c1) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(c0), "r"(c1)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tm, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tm), "r"(c0), "r"(c1),
-                 "r"(c2)
-                 : "memory");
-}
-// `bytes` (a multiple of 16) from a 16-byte aligned global address into L2 only.
-__device__ __forceinline__ void bulk_prefetch_l2(const void* gptr, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void tma_store_2d_and_wait(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"((uint64_t)tm), "r"(src), "r"(c0), "r"(c1)
@@ -830,11 +817,11 @@ int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits) {
 }
 
 struct Plan;
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, size_t budget = 0);
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi = false);
 
 struct Plan {
     int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
-    int epi_off, uw_off, slab_off, slab_q, per_slot, lora_mma, na, us_in_ring, us_off;
+    int epi_off, uw_off, slab_off, slab_q, per_slot, lora_mma, na, us_in_ring, us_off, idx_off;
     size_t smem;
 };
 
@@ -851,7 +838,7 @@ int stacked_zsplits_bound(int T) {
     return std::min(kMaxZSplits, std::max(1, 148 / tiles));
 }
 
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, size_t budget) {
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi) {
     const Tuning& tn = tuning();
     Plan pl = {};
     const int ksteps = (K + kBK - 1) / kBK;
@@ -900,13 +887,19 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     }
     const int ksteps_cta = std::max(1, ksteps / (splits * pl.zsplits));
     const bool two_per_sm = tiles * splits * pl.zsplits > sms;
-    const size_t total_budget = budget ? budget : two_per_sm ? 112 * 1024 : 226 * 1024;
+    const size_t total_budget = two_per_sm ? 112 * 1024 : 226 * 1024;
 
     // epilogue staging (LoRA mode): s_e, s_uw, B slab of this CTA's 128/S rows
     const int tile_tokens = std::min(T, bn);
     size_t epi_bytes = 0;
     size_t us_bytes = 0;
-    if (lora && r == 8 && !tn.simt_expand) {
+    if (lora && fused_epi) {
+        // single-launch decode kernel: B rows of the CTA's slice of the tile for every adapter, then the routing
+        pl.slab_off = 0;
+        pl.uw_off = (int)align_up((size_t)N * (kBM / splits) * 16, 16);
+        pl.idx_off = pl.uw_off + bn * k * r * 4;
+        epi_bytes = (size_t)pl.idx_off + (size_t)bn * k * 4;
+    } else if (lora && r == 8 && !tn.simt_expand) {
         // expand on the tensor cores: B rows of this split's adapters for all 128 rows, and the masked,
         // gate-weighted shrink outputs of the tile's tokens as the other operand
         pl.lora_mma = 1;
@@ -1028,6 +1021,7 @@ static void fill_common(WGemmParams& p, const Plan& pl, int T, int K, int32_t* s
     p.na = pl.na;
     p.us_in_ring = pl.us_in_ring;
     p.us_off = pl.us_off;
+    p.idx_off = pl.idx_off;
     p.status = status;
 }
 
@@ -1122,7 +1116,7 @@ struct FusedPlan {
     bool ok;
     int why;   // why not: 1 knob/shape, 2 too many row tiles, 3 several token tiles, 4 residency, 5 operand sizes
     Plan main;
-    int row_tiles, n_main, n_aux, a_tiles, aux_slices, aux_stages, overlap;
+    int row_tiles, n_main, n_aux, a_tiles, aux_slices, aux_stages;
 };
 
 static FusedPlan make_fused_plan(const meteora_shape_t& s) {
@@ -1137,18 +1131,13 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.row_tiles = (s.d_out + kBM - 1) / kBM;
     fp.why = 2;
     if (fp.row_tiles > kMaxFusedRowTiles) return fp;
-    fp.overlap = tuning().overlap ? 1 : 0;
-    fp.main = make_plan(fp.row_tiles, s.T, s.d_in, true, s.N, s.r, s.k, fp.overlap ? 110 * 1024 : 0);
+    fp.main = make_plan(fp.row_tiles, s.T, s.d_in, true, s.N, s.r, s.k, true);
     fp.why = 3;
     if (fp.main.n_tiles != 1) return fp;
-    fp.why = 5;
-    if (!fp.main.lora_mma || fp.main.us_in_ring) return fp;
     fp.why = 4;
     const int S = fp.main.splits;
     fp.n_main = fp.row_tiles * S;
-    int capacity = max_resident_ctas(fp.main.smem);
-    // overlapped calls: this call and the next one share the SMs, so aim at one CTA per SM for each
-    if (fp.overlap && capacity >= 2 * sm_count() && fp.n_main + 3 <= sm_count()) capacity = sm_count();
+    const int capacity = max_resident_ctas(fp.main.smem);
     fp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
     const int aux_tiles = fp.a_tiles + 1;
     const int n_aux = std::min(capacity - fp.n_main, 24);
@@ -1179,9 +1168,9 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     if (fp.ok)
         return snprintf(buf, n,
                         "path=fused_decode launches=1 main_ctas=%d splits=%d aux_ctas=%d aux_slices=%d tile_tokens=%d "
-                        "stages=%d kc=%d smem=%zu resident_ctas=%d overlap=%d",
+                        "stages=%d kc=%d smem=%zu resident_ctas=%d",
                         fp.n_main, fp.main.splits, fp.n_aux, fp.aux_slices, fp.main.BN, fp.main.stages, fp.main.kc,
-                        fp.main.smem, max_resident_ctas(fp.main.smem), fp.overlap);
+                        fp.main.smem, max_resident_ctas(fp.main.smem));
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     return snprintf(buf, n,
@@ -1242,17 +1231,24 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
-    if (fp.overlap) {
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-    } else {
-        attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
-        attr[0].val.cooperative = 1;
-    }
+    attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
+    attr[0].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (fp.overlap || tuning().coop) ? 1 : 0;
-    d.overlap = fp.overlap;
+    cfg.numAttrs = tuning().coop ? 1 : 0;
+#ifdef METEORA_TRACE
+    static int trace_calls = 0;
+    d.trace_call = trace_calls++;
+#endif
     return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mG, mX1, d));
 }
 
 }  // namespace meteora
+
+#ifdef METEORA_TRACE
+// Trace build only: copy the device-side time stamps of the decode kernel to the host.
+extern "C" int meteora_trace_read(unsigned long long* host, size_t count) {
+    const size_t total = (size_t)meteora::kTraceCalls * meteora::kTraceCtas * meteora::kTraceSlots;
+    if (count > total) count = total;
+    return cudaMemcpyFromSymbol(host, meteora::g_fused_trace, count * sizeof(unsigned long long)) == cudaSuccess ? 0 : -5;
+}
+#endif
