@@ -23,8 +23,11 @@ struct DecodeParams {
     WGemmParams main;      // base product (MODE_LORA, lora_mma): ring geometry, staging offsets, outputs
     int n_main;            // main CTAs = row tiles * S
     int n_aux;             // aux CTAs; they take the lowest block indices so that they are scheduled first
-    int a_tiles, a_rows;   // row tiles / rows of the stacked A matrix (N * r rows); one more tile holds Wg
-    int aux_slices;        // contraction slices per aux row tile; active aux CTAs = (a_tiles + 1) * aux_slices
+    int a_tiles, a_rows;   // row tiles / rows of the stacked A matrix (N * r rows)
+    int aux_tiles;         // row tiles of the stacked shrink: a_tiles, plus one for Wg unless it fits behind A's last rows
+    int gate_tile;         // the tile that holds the N rows of Wg, from tile row gate_row0 on
+    int gate_row0;
+    int aux_slices;        // contraction slices per aux row tile; active aux CTAs = aux_tiles * aux_slices
     int aux_stages;        // ring depth of the aux main loop (one k-step per stage)
     int bar_stages;        // barriers are laid out for max(main stages, aux stages) ring slots
     float* u_part;         // [aux_slices][T][ld_u] partial stacked shrink
@@ -158,8 +161,11 @@ struct RingGeom {
 
 // Producer side of a main loop (one thread).  `first_batch_done`, if not null, is bumped once the loads
 // that fit into the ring without waiting have been issued.
+// A second weight map `tmW2` (or the only one, when tmW is null) lands `w2_off` bytes into the weight tile: the
+// rows of Wg behind the last rows of A.
 __device__ __forceinline__ bool fused_producer(const RingGeom& g, const CUtensorMap* tmW, const CUtensorMap* tmXp,
-                                               int row0, int ks0, int niter, int32_t* first_batch_done) {
+                                               int row0, int ks0, int niter, int32_t* first_batch_done,
+                                               const CUtensorMap* tmW2 = nullptr, uint32_t w2_off = 0) {
     bool ok = true;
     for (int i = 0; i < niter; ++i) {
         const int s = i % g.stages, round = i / g.stages;
@@ -174,10 +180,12 @@ __device__ __forceinline__ bool fused_producer(const RingGeom& g, const CUtensor
         const int kstep = ks0 + i * g.kc;
         mbar_expect_tx(full, g.stage_bytes);
         if (g.maps3d) {
-            tma_load_3d(dst, tmW, 0, row0, kstep, full);
+            if (tmW) tma_load_3d(dst, tmW, 0, row0, kstep, full);
+            if (tmW2) tma_load_3d(dst + w2_off, tmW2, 0, 0, kstep, full);
             tma_load_3d(dst + g.kc * kWTileBytes, tmXp, 0, 0, kstep, full);
         } else {
-            tma_load_2d(dst, tmW, kstep * kBK, row0, full);
+            if (tmW) tma_load_2d(dst, tmW, kstep * kBK, row0, full);
+            if (tmW2) tma_load_2d(dst + w2_off, tmW2, kstep * kBK, 0, full);
             tma_load_2d(dst + kWTileBytes, tmXp, kstep * kBK, 0, full);
         }
     }
@@ -208,8 +216,9 @@ __device__ __forceinline__ bool fused_mma(const RingGeom& g, uint32_t tmem_base,
 
 __global__ void __launch_bounds__(kThreads)
 k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmX,
-               const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmG,
-               const __grid_constant__ CUtensorMap tmX1, const DecodeParams d) {
+               const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAt,
+               const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmX1,
+               const DecodeParams d) {
     const WGemmParams& p = d.main;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -226,7 +235,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool is_aux = (int)blockIdx.x < d.n_aux;
     const int main_id = (int)blockIdx.x - d.n_aux;
-    const int n_active = (d.a_tiles + 1) * d.aux_slices;
+    const int n_active = d.aux_tiles * d.aux_slices;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < nbar; ++s) mbar_init(bar_base + s * 8, 1);
@@ -264,7 +273,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         // ================================================================== aux CTA
         const int aux_id = blockIdx.x;
         const bool active = aux_id < n_active;
-        const int tile = aux_id % (d.a_tiles + 1), slice = aux_id / (d.a_tiles + 1);
+        const int tile = aux_id % d.aux_tiles, slice = aux_id / d.aux_tiles;
         const int ks0 = active ? (int)(((long long)p.ksteps * slice) / d.aux_slices) : 0;
         const int ks1 = active ? (int)(((long long)p.ksteps * (slice + 1)) / d.aux_slices) : 0;
         const int niter = ks1 - ks0;
@@ -272,9 +281,10 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         const uint32_t bar_acc = bar_base + 2 * d.aux_stages * 8;
         if (warp == 0) {
             if (lane == 0 && active) {
-                const bool is_gate = tile >= d.a_tiles;
-                if (!fused_producer(geom, is_gate ? &tmG : &tmA, &tmX1, is_gate ? 0 : tile * kBM, ks0, niter,
-                                    d.ctr + 3))
+                // A's last tile has its own map (its box stops at A's last row when Wg follows in the same tile)
+                const CUtensorMap* mA = tile >= d.a_tiles ? nullptr : tile == d.a_tiles - 1 ? &tmAt : &tmA;
+                const CUtensorMap* mG = tile == d.gate_tile ? &tmG : nullptr;
+                if (!fused_producer(geom, mA, &tmX1, tile * kBM, ks0, niter, d.ctr + 3, mG, (uint32_t)d.gate_row0 * 128u))
                     flag_error(p, 1, 400);
             }
         } else if (warp == 1) {
@@ -289,10 +299,13 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
             tc_fence_after();
             // accumulators straight to the partial buffer: lane = row, a warp writes 128 contiguous bytes
-            const int row = tile < d.a_tiles ? tile * kBM + quad * 32 + lane : quad * 32 + lane;
-            const int limit = tile < d.a_tiles ? d.a_rows : p.N;
-            const int col = tile < d.a_tiles ? row : d.col_logits + row;
-            float* dst = d.u_part + (size_t)slice * p.T * d.ld_u + col;
+            const int trow = quad * 32 + lane;                                   // row of the tile
+            int col = -1;                                                        // column of u_part, -1: padding row
+            if (tile < d.a_tiles && tile * kBM + trow < d.a_rows && !(tile == d.gate_tile && trow >= d.gate_row0))
+                col = tile * kBM + trow;
+            if (tile == d.gate_tile && trow >= d.gate_row0 && trow < d.gate_row0 + p.N)
+                col = d.col_logits + trow - d.gate_row0;
+            float* dst = d.u_part + (size_t)slice * p.T * d.ld_u + max(col, 0);
             for (int c = c_begin; c < c_end; c += 16) {
                 float v[16];
                 if (acc_ok) {
@@ -301,7 +314,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
 #pragma unroll
                     for (int i = 0; i < 16; ++i) v[i] = 0.f;
                 }
-                if (row < limit) {
+                if (col >= 0) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
                         if (c + i < p.T) dst[(size_t)(c + i) * d.ld_u] = v[i];

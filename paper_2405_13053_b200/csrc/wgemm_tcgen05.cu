@@ -1116,7 +1116,7 @@ struct FusedPlan {
     bool ok;
     int why;   // why not: 1 knob/shape, 2 too many row tiles, 3 several token tiles, 4 residency, 5 operand sizes
     Plan main;
-    int row_tiles, n_main, n_aux, a_tiles, aux_slices, aux_stages;
+    int row_tiles, n_main, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages;
 };
 
 static FusedPlan make_fused_plan(const meteora_shape_t& s) {
@@ -1139,7 +1139,13 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.n_main = fp.row_tiles * S;
     const int capacity = max_resident_ctas(fp.main.smem);
     fp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
-    const int aux_tiles = fp.a_tiles + 1;
+    // Wg rides behind A's last rows when the tile has room for it (N * r = 224, N = 28: rows 96..123 of tile 1)
+    const int tail_rows = s.N * s.r - (fp.a_tiles - 1) * kBM;
+    const bool merged = tail_rows % 8 == 0 && tail_rows + s.N <= kBM;
+    fp.aux_tiles = merged ? fp.a_tiles : fp.a_tiles + 1;
+    fp.gate_tile = fp.aux_tiles - 1;
+    fp.gate_row0 = merged ? tail_rows : 0;
+    const int aux_tiles = fp.aux_tiles;
     const int n_aux = std::min(capacity - fp.n_main, 24);
     if (n_aux < aux_tiles) return fp;
     const int ksteps = (s.d_in + kBK - 1) / kBK;
@@ -1186,12 +1192,14 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     if (!fp.ok) return METEORA_ERR_UNSUPPORTED_SHAPE;
     const Plan& pl = fp.main;
     const int depth = pl.maps3d ? pl.kc : 0, depth1 = pl.maps3d ? 1 : 0;
-    CUtensorMap mW, mX, mA, mG, mX1;
+    CUtensorMap mW, mX, mA, mAt, mG, mX1;
     int rc;
+    const int tail_box = fp.gate_row0 > 0 ? fp.gate_row0 : kBM, gate_box = kBM - fp.gate_row0;
     if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, depth, &mW)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, depth, &mX)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, depth1, &mA)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(Wg, s.d_in, s.N, kBM, depth1, &mG)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, tail_box, depth1, &mAt)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Wg, s.d_in, s.N, gate_box, depth1, &mG)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, depth1, &mX1)) != METEORA_OK) return rc;
     DecodeParams d = {};
     fill_common(d.main, pl, s.T, s.d_in, ws.status);
@@ -1210,6 +1218,9 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.n_aux = fp.n_aux;
     d.a_tiles = fp.a_tiles;
     d.a_rows = s.N * s.r;
+    d.aux_tiles = fp.aux_tiles;
+    d.gate_tile = fp.gate_tile;
+    d.gate_row0 = fp.gate_row0;
     d.aux_slices = fp.aux_slices;
     d.aux_stages = fp.aux_stages;
     d.bar_stages = std::max(fp.aux_stages, pl.stages);
@@ -1239,7 +1250,7 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     static int trace_calls = 0;
     d.trace_call = trace_calls++;
 #endif
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mG, mX1, d));
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mAt, mG, mX1, d));
 }
 
 }  // namespace meteora
