@@ -46,6 +46,48 @@ __device__ __forceinline__ float ld_part(const float* p) { return kCoherent ? __
 template <bool kCoherent>
 __device__ __forceinline__ float4 ld_part4(const float4* p) { return kCoherent ? __ldcg(p) : *p; }
 
+// Selection for one token with at most ZMAX partial copies: lane n owns logit n and reads it from every slice,
+// the loads issued together (one memory round trip); the slices are added in slice order.
+template <bool kCoherent, int ZMAX>
+__device__ __forceinline__ void select_token_few(const float* row, int col_logits, int zsplits, size_t zstride,
+                                                 int t, int N, int r, int k, float inv_tau, int lane,
+                                                 int32_t* topk_idx, float* topk_w, float* uw) {
+    float part0[ZMAX], part1[ZMAX];
+#pragma unroll
+    for (int z = 0; z < ZMAX; ++z) {
+        const bool on = z < zsplits;
+        part0[z] = (on && lane < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane) : 0.f;
+        part1[z] = (on && lane + 32 < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32) : 0.f;
+    }
+    float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+    for (int z = 0; z < ZMAX; ++z) {
+        v0 += part0[z];
+        v1 += part1[z];
+    }
+    int idx;
+    float w;
+    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    if (lane < k) {
+        topk_idx[(size_t)t * k + lane] = idx;
+        topk_w[(size_t)t * k + lane] = w;
+    }
+    for (int c0 = 0; c0 < k * r; c0 += 32) {
+        const int c = c0 + lane;
+        const int j = min(c / r, k - 1), q = c - j * r;
+        const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
+        const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
+        float pu[ZMAX];
+#pragma unroll
+        for (int z = 0; z < ZMAX; ++z)
+            pu[z] = (z < zsplits && c < k * r) ? ld_part<kCoherent>(row + z * zstride + ij * r + q) : 0.f;
+        float u = 0.f;
+#pragma unroll
+        for (int z = 0; z < ZMAX; ++z) u += pu[z];
+        if (c < k * r) uw[(size_t)t * k * r + c] = wj * u;
+    }
+}
+
 // Selection for one token (one warp): row t of u_all holds A_i x for every adapter (N*r values) and, from
 // column col_logits on, the N gate logits; u_all comes as `zsplits` partial copies (slices of the contraction
 // axis, zstride floats apart).  Writes the picks, their weights and uw[t,j,:] = w_j * (A_{i_j} x).
@@ -55,42 +97,11 @@ __device__ __forceinline__ void select_token(const float* u_all, int ld_u, int c
                                              int32_t* topk_idx, float* topk_w, float* uw) {
     const float* row = u_all + (size_t)t * ld_u;
     if (zsplits <= 8) {
-        // Few partial copies: lane n owns logit n and reads it from every slice, the (at most 8) loads
-        // issued together; the slices are added in slice order.
-        float part0[8], part1[8];
-#pragma unroll
-        for (int z = 0; z < 8; ++z) {
-            const bool on = z < zsplits;
-            part0[z] = (on && lane < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane) : 0.f;
-            part1[z] = (on && lane + 32 < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32) : 0.f;
-        }
-        float v0 = 0.f, v1 = 0.f;
-#pragma unroll
-        for (int z = 0; z < 8; ++z) {
-            v0 += part0[z];
-            v1 += part1[z];
-        }
-        int idx;
-        float w;
-        warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
-        if (lane < k) {
-            topk_idx[(size_t)t * k + lane] = idx;
-            topk_w[(size_t)t * k + lane] = w;
-        }
-        for (int c0 = 0; c0 < k * r; c0 += 32) {
-            const int c = c0 + lane;
-            const int j = min(c / r, k - 1), q = c - j * r;
-            const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
-            const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
-            float pu[8];
-#pragma unroll
-            for (int z = 0; z < 8; ++z)
-                pu[z] = (z < zsplits && c < k * r) ? ld_part<kCoherent>(row + z * zstride + ij * r + q) : 0.f;
-            float u = 0.f;
-#pragma unroll
-            for (int z = 0; z < 8; ++z) u += pu[z];
-            if (c < k * r) uw[(size_t)t * k * r + c] = wj * u;
-        }
+        select_token_few<kCoherent, 8>(row, col_logits, zsplits, zstride, t, N, r, k, inv_tau, lane, topk_idx, topk_w, uw);
+        return;
+    }
+    if (zsplits <= 16) {
+        select_token_few<kCoherent, 16>(row, col_logits, zsplits, zstride, t, N, r, k, inv_tau, lane, topk_idx, topk_w, uw);
         return;
     }
     if (zsplits <= 32 && r == 8 && k <= 4) {

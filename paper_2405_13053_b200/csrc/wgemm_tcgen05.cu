@@ -1149,7 +1149,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     const int n_aux = std::min(capacity - fp.n_main, 24);
     if (n_aux < aux_tiles) return fp;
     const int ksteps = (s.d_in + kBK - 1) / kBK;
-    fp.aux_slices = std::min(std::min(n_aux / aux_tiles, ksteps), 32);
+    fp.aux_slices = std::min(std::min(n_aux / aux_tiles, ksteps), 16);   // 16: the selection reads all slices at once
     fp.n_aux = aux_tiles * fp.aux_slices;
     const size_t chunk = kWTileBytes + (size_t)fp.main.BN * 128;
     const size_t ring_bytes = (size_t)fp.main.stages * fp.main.kc * chunk;
