@@ -58,25 +58,27 @@ __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
     return true;
 }
 
-// B rows [row0, row0 + nrows) of every adapter as slab[e][row][8 bf16]; rows past d_out are zero.
+// B rows [row0, row0 + nrows) of every adapter (8 bf16 = 16 bytes each) as slab[e][row % 4][row / 4], so that
+// threads owning consecutive groups of 4 rows read consecutive 16-byte words; rows past d_out are zero.
 __device__ __forceinline__ void stage_slab_rows(const WGemmParams& p, uint4* slab, int row0, int nrows, int etid) {
     const uint4* Bg = reinterpret_cast<const uint4*>(p.B);
-    const int total = p.N * nrows;
+    const int total = p.N * nrows, nq = nrows / 4;
     for (int i = etid; i < total; i += kEpiThreads) {
-        const int e = i / nrows, o = row0 + (i - e * nrows);
-        slab[i] = o < p.d_out ? __ldg(Bg + (size_t)e * p.d_out + o) : make_uint4(0u, 0u, 0u, 0u);
+        const int e = i / nrows, rl = i - e * nrows, o = row0 + rl;
+        slab[e * nrows + (rl & 3) * nq + (rl >> 2)] =
+            o < p.d_out ? __ldg(Bg + (size_t)e * p.d_out + o) : make_uint4(0u, 0u, 0u, 0u);
     }
 }
 
 // Last step of a main CTA: rows [row_lo, row_lo + 4 * nq) of the tile, all tokens.  Work items are (token,
 // group of 4 rows); a thread keeps U items in flight: the C partial tiles' values first (one round trip to
 // L2), then their sum in split order, the expand of Eq. 2 from the staged B rows and the routing in shared
-// memory, one rounding to bf16 and the store.  `before_compute` runs once, after the first loads are issued.
-template <int C, int U, typename F>
+// memory, one rounding to bf16 and the store.  The routing is staged by warp 0, which arrives on named
+// barrier 2 when it is in shared memory; the threads here join that barrier after issuing their first loads.
+template <int C, int U>
 __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* part, size_t part_stride, bool from_l2,
                                             int tile_row0, int row_lo, int nq, int ntok, const uint4* slab,
-                                            int slab_rows, const float* s_uw, const int* s_idx, int etid,
-                                            F before_compute) {
+                                            int slab_rows, const float* s_uw, const int* s_idx, int etid) {
     const int items = nq * ntok;
     const float4* s_uw4 = reinterpret_cast<const float4*>(s_uw);
     for (int base = 0; base < items; base += kEpiThreads * U) {
@@ -92,7 +94,7 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* p
                 v[u][q] = from_l2 ? __ldcg(src) : *src;
             }
         }
-        if (base == 0) before_compute();
+        if (base == 0) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int it = base + etid + u * kEpiThreads;
@@ -109,11 +111,11 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* p
             for (int j = 0; j < p.k; ++j) {
                 const int slot = t * p.k + j;
                 const float4 u0 = s_uw4[2 * slot], u1 = s_uw4[2 * slot + 1];
-                const uint4* b = slab + (size_t)s_idx[slot] * slab_rows + ql * 4;
+                const uint4* b = slab + (size_t)s_idx[slot] * slab_rows + ql;
                 fma8(b[0], u0, u1, acc.x);
-                fma8(b[1], u0, u1, acc.y);
-                fma8(b[2], u0, u1, acc.z);
-                fma8(b[3], u0, u1, acc.w);
+                fma8(b[nq], u0, u1, acc.y);
+                fma8(b[2 * nq], u0, u1, acc.z);
+                fma8(b[3 * nq], u0, u1, acc.w);
             }
             const int o = tile_row0 + row_lo + ql * 4;
             __nv_bfloat16* dst = p.y + (size_t)t * p.d_out + o;
@@ -362,6 +364,24 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 if (tr_main) FUSED_STAMP(p, 32, 1);
                 ok = fused_producer(geom, &tmW0, &tmX, tile_m * kBM, ks0, niter, nullptr) && ok;
                 if (!ok) flag_error(p, 1, 100);
+                if (!wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);              // routing published
+                if (tr_main) FUSED_STAMP(p, 32, 4);
+            }
+            __syncwarp();
+            // The routing into shared memory for the epilogue warps (it was written by other CTAs of this kernel:
+            // loads that bypass L1), then named barrier 2.
+            {
+                int* s_idx = reinterpret_cast<int*>(epi + p.idx_off);
+                float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off);
+                const int slots = ntok * p.k;
+                const float4* uw4 = reinterpret_cast<const float4*>(p.uw);
+#pragma unroll 8
+                for (int i = lane; i < slots; i += 32) s_idx[i] = min(max(__ldcg(p.topk_idx + i), 0), p.N - 1);
+#pragma unroll 8
+                for (int i = lane; i < 2 * slots; i += 32) s_uw4[i] = __ldcg(uw4 + i);
+                __syncwarp();
+                asm volatile("bar.arrive 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
+                if (lane == 0 && tr_main) FUSED_STAMP(p, 32, 9);
             }
         } else if (warp == 1) {
             if (lane == 0) {
@@ -405,28 +425,19 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     __threadfence();
                     atomicAdd(d.tile_ctr + tile_m, 1);
                 }
-                if (!wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);              // routing published
-                if (tr_main) FUSED_STAMP(p, 32, 4);
                 if (S > 1 && !wait_counter(d.tile_ctr + tile_m, S)) flag_error(p, 4, 900);  // all partials of the tile in
                 if (tr_main) FUSED_STAMP(p, 32, 6);
             }
             epi_barrier();
             const float* src = S > 1 ? d.part_g + (size_t)tile_m * S * part_stride : part;
-            auto stage_routing = [&]() {
-                // the routing was written by other CTAs of this kernel: loads that bypass L1
-                const int slots = ntok * p.k;
-                for (int i = etid; i < slots; i += kEpiThreads) s_idx[i] = min(max(__ldcg(p.topk_idx + i), 0), p.N - 1);
-                const float4* uw4 = reinterpret_cast<const float4*>(p.uw);
-                for (int i = etid; i < 2 * slots; i += kEpiThreads) reinterpret_cast<float4*>(s_uw)[i] = __ldcg(uw4 + i);
-                epi_barrier();
-            };
             const int nq = nrows / 4;
             switch (S) {
-                case 1: finish_rows<1, 4>(p, src, part_stride, false, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
-                case 2: finish_rows<2, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
-                case 4: finish_rows<4, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
-                default: finish_rows<8, 2>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid, stage_routing); break;
+                case 1: finish_rows<1, 4>(p, src, part_stride, false, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
+                case 2: finish_rows<2, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
+                case 4: finish_rows<4, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
+                default: finish_rows<8, 2>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
             }
+            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);
         }
     }
 
