@@ -36,6 +36,7 @@ struct DecodeParams {
     float* topk_w;
     float* uw;
     float inv_tau;
+    int hold;              // main CTAs start loading only after the aux CTAs have issued their first loads
     int32_t* ctr;          // [0] aux partials written, [1] selections published, [2] CTAs exited, [3] aux loads issued
     float* part_g;         // [row tile][split][BN][128] fp32 partial accumulator tiles of the base product
     int32_t* tile_ctr;     // [row tiles] partials written per tile
@@ -56,6 +57,64 @@ __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
         __nanosleep(32);
     }
     return true;
+}
+
+// Selection for one token by one warp, every partial copy of the token's row read in ONE round trip: the
+// N*r shrink values and the N logits are summed over the `zsplits` copies in slice order (two 16-byte columns
+// per lane, all loads in flight together) into `wbuf` (shared memory, ld_u floats), then top-k, softmax over
+// the picks (Eq. 3) and uw[t,j,:] = w_j * (A_{i_j} x) come from there.  Rank 8 only; N * 8 + N <= 256 floats
+// per 32 lanes and pass, further passes for larger N.
+__device__ __forceinline__ void select_token_wide(const float* u_part, int ld_u, int col_logits, int zsplits,
+                                                  size_t zstride, int t, int N, int k, float inv_tau, int lane,
+                                                  float* wbuf, int32_t* topk_idx, float* topk_w, float* uw) {
+    constexpr int ZMAX = 16;
+    const int n_a4 = N * 2, n_c4 = n_a4 + (N + 3) / 4;             // 16-byte chunks: shrink values, then logits
+    const float* row = u_part + (size_t)t * ld_u;
+    for (int c0 = 0; c0 < n_c4; c0 += 64) {
+        float4 acc[2];
+        float4 v[2][ZMAX];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c4 = c0 + h * 32 + lane;
+            const int col = c4 < n_a4 ? 4 * c4 : col_logits + 4 * (c4 - n_a4);
+#pragma unroll
+            for (int z = 0; z < ZMAX; ++z)
+                v[h][z] = (c4 < n_c4 && z < zsplits) ? __ldcg(reinterpret_cast<const float4*>(row + z * zstride + col))
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int z = 0; z < ZMAX; ++z) {
+                acc[h].x += v[h][z].x;
+                acc[h].y += v[h][z].y;
+                acc[h].z += v[h][z].z;
+                acc[h].w += v[h][z].w;
+            }
+            const int c4 = c0 + h * 32 + lane;
+            const int col = c4 < n_a4 ? 4 * c4 : col_logits + 4 * (c4 - n_a4);
+            if (c4 < n_c4) *reinterpret_cast<float4*>(wbuf + col) = acc[h];
+        }
+    }
+    __syncwarp();
+    const float v0 = lane < N ? wbuf[col_logits + lane] : 0.f;
+    const float v1 = lane + 32 < N ? wbuf[col_logits + lane + 32] : 0.f;
+    int idx;
+    float w;
+    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    if (lane < k) {
+        topk_idx[(size_t)t * k + lane] = idx;
+        topk_w[(size_t)t * k + lane] = w;
+    }
+    for (int c0 = 0; c0 < k * 8; c0 += 32) {
+        const int c = c0 + lane;
+        const int j = min(c / 8, k - 1), q = c - j * 8;
+        const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
+        const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
+        if (c < k * 8) uw[(size_t)t * k * 8 + c] = wj * wbuf[ij * 8 + q];
+    }
+    __syncwarp();
 }
 
 // B rows [row0, row0 + nrows) of every adapter (8 bf16 = 16 bytes each) as slab[e][row % 4][row / 4], so that
@@ -335,9 +394,10 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             }
             __syncthreads();
             const int nwarps = kThreads / 32;                                    // tokens dealt round-robin
+            float* wbuf = reinterpret_cast<float*>(ring_ptr) + warp * d.ld_u;     // the ring is idle by now
             for (int t = aux_id * nwarps + warp; t < p.T; t += n_active * nwarps)
-                select_token<true>(d.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.r,
-                                   p.k, d.inv_tau, lane, d.topk_idx, d.topk_w, d.uw);
+                select_token_wide(d.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.k,
+                                  d.inv_tau, lane, wbuf, d.topk_idx, d.topk_w, d.uw);
             __syncthreads();
             if (threadIdx.x == 0) {
                 __threadfence();
@@ -360,7 +420,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         if (warp == 0) {
             if (lane == 0) {
                 // let the stacked shrink get its loads into the memory queues first
-                bool ok = wait_counter(d.ctr + 3, n_active);
+                bool ok = d.hold ? wait_counter(d.ctr + 3, n_active) : true;
                 if (tr_main) FUSED_STAMP(p, 32, 1);
                 ok = fused_producer(geom, &tmW0, &tmX, tile_m * kBM, ks0, niter, nullptr) && ok;
                 if (!ok) flag_error(p, 1, 100);

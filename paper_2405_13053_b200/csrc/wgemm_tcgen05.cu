@@ -1160,6 +1160,9 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.aux_stages = std::min(fp.aux_stages, std::min(bar_cap / 2, 16));
     fp.why = 5;
     if (fp.aux_stages < 1) return fp;
+    // the aux CTAs' selection keeps one summed row of the stacked shrink per warp in the idle ring
+    int col_logits = 0;
+    if (ring_bytes < (size_t)(kThreads / 32) * tc_stacked_pitch(s, &col_logits) * sizeof(float)) return fp;
     fp.why = 0;
     fp.ok = true;
     return fp;
@@ -1231,6 +1234,7 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.topk_w = ws.topk_w;
     d.uw = ws.uw;
     d.inv_tau = 1.0f / s.temperature;
+    d.hold = tuning().no_hold ? 0 : 1;
     d.ctr = ws.status + 16;
     d.part_g = ws.part_g;
     d.tile_ctr = ws.tile_ctr;
