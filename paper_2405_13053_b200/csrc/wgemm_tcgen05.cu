@@ -1122,11 +1122,9 @@ struct FusedPlan {
 static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     FusedPlan fp = {};
     fp.why = 1;
-    // Measured on B200 (4096 -> 4096): the single launch wins from about 64 tokens up (23 vs 25 us at T = 128);
-    // below that the three-launch chain is ahead (16.7 vs 18.3 us at T = 1), because the routing sits on the
-    // critical path of the one kernel while the chain's first two launches are cheap.  fused = 2 forces it.
-    const int fused = tuning().fused;
-    if (!fused || (fused == 1 && s.T < 64)) return fp;
+    // Measured on B200 (4096 -> 4096): the single launch is ahead of the three-launch chain at every decode
+    // batch size (15.7 vs 16.5 us at T = 1, 19.5 vs 25 us at T = 128).
+    if (!tuning().fused) return fp;
     if (!tc_path_supported(s) || s.T > 256 || s.r != 8 || tuning().simt_expand) return fp;
     fp.row_tiles = (s.d_out + kBM - 1) / kBM;
     fp.why = 2;
