@@ -33,10 +33,11 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     ws.topk_w = (float*)take(T * s.k * sizeof(float));
     ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
     ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (size_t)stacked_zsplits_bound(s.T));   // one copy per slice of the contraction axis
-    // fused decode scratch: at most 296 resident CTAs (or 8 per row tile), each one tile of 128 x BN fp32
+    // decode kernel scratch: two partial tiles of 128 x BN fp32 per main CTA, at most 148 main CTAs, at most
+    // 14 per row tile
     const size_t row_tiles = ((size_t)s.d_out + 127) / 128;
     const size_t bn = (T + 15) / 16 * 16;
-    const size_t part_tiles = s.T <= 256 ? (row_tiles * 8 < 296 ? row_tiles * 8 : 296) : 0;
+    const size_t part_tiles = s.T <= 256 ? (row_tiles * 28 < 296 ? row_tiles * 28 : 296) : 0;
     ws.part_g = (float*)take(part_tiles * bn * 128 * sizeof(float));
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);

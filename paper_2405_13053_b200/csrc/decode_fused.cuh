@@ -2,26 +2,31 @@
 // Included by wgemm_tcgen05.cu after the device helpers it uses.
 //
 // The grid holds two kinds of CTAs, all resident at the same time (cooperative launch, no clusters):
-//   - main CTAs, S per 128-row tile of W0 along the contraction axis: stream W0 through TMA + tcgen05 into
-//     TMEM, write the partial accumulator tile to an fp32 scratch (it stays in L2) and, once the tile's S
-//     partials are in, each sums its slice of the rows in split order, adds the LoRA expand of those rows
-//     (Eq. 2: the B rows of every adapter wait in shared memory, the routing arrives from the aux CTAs) and
-//     stores y;
+//   - main CTAs.  The base product W0 x is cut into units of one 128-row tile of W0 times kc k-steps, numbered
+//     tile by tile, and main CTA i takes the units [U*i/M, U*(i+1)/M): every SM streams the same number of
+//     bytes whatever the shape, and a CTA's range covers the tail of one tile and the head of the next (at most
+//     two segments; the host launches this kernel only when M >= row tiles).  Each segment runs through
+//     TMA + tcgen05 into its own TMEM accumulator and goes to an fp32 scratch (it stays in L2).  When all the
+//     CTAs that share a tile have delivered, each of them sums its slice of the tile's rows in CTA order, adds
+//     the LoRA expand of those rows (Eq. 2: the B rows of every adapter wait in shared memory, the routing
+//     arrives from the aux CTAs) and stores y;
 //   - a few aux CTAs on the SMs the main CTAs leave free: each computes a slice of the stacked shrink
 //     [A_0..A_{N-1}; Wg] x (every adapter's A_i x and the gate logits, Sec. 3.1) on the same main loop and
 //     writes it as an fp32 partial; once all partials are in, the aux CTAs share the tokens and run the
 //     top-k selection and the softmax over the selected logits (Eq. 3), publishing topk_idx, topk_w, uw.
 // The main CTAs hold their first loads back until the aux CTAs have issued theirs, so the 2 MB of the shrink
-// are ahead of the 33 MB of W0 in the memory queues; they need the routing only after their main loop and
-// the exchange of the partial tiles.  Every wait is bounded; on expiry the status word is set and the kernel drains.  The
+// are ahead of W0 in the memory queues; they need the routing only after their main loop and the exchange
+// of the partial tiles.  Every wait is bounded; on expiry the status word is set and the kernel drains.  The
 // counters live in the workspace header and are re-armed by the last CTA to exit.
 #pragma once
 
 namespace meteora {
 
 struct DecodeParams {
-    WGemmParams main;      // base product (MODE_LORA, lora_mma): ring geometry, staging offsets, outputs
-    int n_main;            // main CTAs = row tiles * S
+    WGemmParams main;      // base product: ring geometry, staging offsets, outputs
+    int n_main;            // main CTAs (M)
+    int upt;               // units per row tile = k-steps / kc
+    long long units;       // row tiles * upt (U)
     int n_aux;             // aux CTAs; they take the lowest block indices so that they are scheduled first
     int a_tiles, a_rows;   // row tiles / rows of the stacked A matrix (N * r rows)
     int aux_tiles;         // row tiles of the stacked shrink: a_tiles, plus one for Wg unless it fits behind A's last rows
@@ -38,8 +43,8 @@ struct DecodeParams {
     float inv_tau;
     int hold;              // main CTAs start loading only after the aux CTAs have issued their first loads
     int32_t* ctr;          // [0] aux partials written, [1] selections published, [2] CTAs exited, [3] aux loads issued
-    float* part_g;         // [row tile][split][BN][128] fp32 partial accumulator tiles of the base product
-    int32_t* tile_ctr;     // [row tiles] partials written per tile
+    float* part_g;         // [main CTA][segment 0/1][BN][128] fp32 partial accumulator tiles of the base product
+    int32_t* tile_ctr;     // [row tiles] partials delivered per tile
     int row_tiles;
     int trace_call;        // trace builds: which record of the trace buffer this launch fills
 };
@@ -129,16 +134,17 @@ __device__ __forceinline__ void stage_slab_rows(const WGemmParams& p, uint4* sla
     }
 }
 
-// Last step of a main CTA: rows [row_lo, row_lo + 4 * nq) of the tile, all tokens.  Work items are (token,
-// group of 4 rows); a thread keeps U items in flight: the C partial tiles' values first (one round trip to
-// L2), then their sum in split order, the expand of Eq. 2 from the staged B rows and the routing in shared
-// memory, one rounding to bf16 and the store.  The routing is staged by warp 0, which arrives on named
-// barrier 2 when it is in shared memory; the threads here join that barrier after issuing their first loads.
+// Last step of a main CTA for one tile: rows [4*q0, 4*(q0+nq)) of the tile, all tokens.  Work items are
+// (token, group of 4 rows); a thread keeps U items in flight: the values of the C partial tiles first (one round
+// trip to L2; `parts` in CTA order, the first `c` are real), then their sum in that order, the expand of Eq. 2
+// from the staged B rows and the routing in shared memory, one rounding to bf16 and the store.  The routing is
+// staged by warp 0, which arrives on named barrier 2 when it is in shared memory; the threads here join that
+// barrier once (`routing_pending`), after issuing their first loads.
 template <int C, int U>
-__device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* part, size_t part_stride, bool from_l2,
-                                            int tile_row0, int row_lo, int nq, int ntok, const uint4* slab,
-                                            int slab_rows, const float* s_uw, const int* s_idx, int etid) {
-    const int items = nq * ntok;
+__device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* const (&parts)[C], int c,
+                                            int tile_row0, int q0, int nq, int ntok, const uint4* slab,
+                                            const float* s_uw, const int* s_idx, int etid, bool& routing_pending) {
+    const int items = nq * ntok, slab_rows = 4 * nq;
     const float4* s_uw4 = reinterpret_cast<const float4*>(s_uw);
     for (int base = 0; base < items; base += kEpiThreads * U) {
         float4 v[U][C];
@@ -146,14 +152,15 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* p
         for (int u = 0; u < U; ++u) {
             const int it = min(base + etid + u * kEpiThreads, items - 1);
             const int t = it / nq, ql = it - t * nq;
-            const float* a = part + (size_t)t * kBM + row_lo + ql * 4;
+            const size_t off = (size_t)t * kBM + (q0 + ql) * 4;
 #pragma unroll
-            for (int q = 0; q < C; ++q) {
-                const float4* src = reinterpret_cast<const float4*>(a + q * part_stride);
-                v[u][q] = from_l2 ? __ldcg(src) : *src;
-            }
+            for (int q = 0; q < C; ++q)
+                v[u][q] = q < c ? __ldcg(reinterpret_cast<const float4*>(parts[q] + off)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (base == 0) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
+        if (routing_pending) {
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
+            routing_pending = false;
+        }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int it = base + etid + u * kEpiThreads;
@@ -176,7 +183,7 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* p
                 fma8(b[2 * nq], u0, u1, acc.z);
                 fma8(b[3 * nq], u0, u1, acc.w);
             }
-            const int o = tile_row0 + row_lo + ql * 4;
+            const int o = tile_row0 + (q0 + ql) * 4;
             __nv_bfloat16* dst = p.y + (size_t)t * p.d_out + o;
             if ((p.d_out & 3) == 0 && o + 3 < p.d_out) {
                 const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
@@ -192,6 +199,22 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* p
             }
         }
     }
+}
+
+template <int C, int U>
+__device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* part_g, size_t part_stride,
+                                            long long units, int M, int upt, int tile, int first_cta, int c,
+                                            int q0, int nq, int ntok, const uint4* slab, const float* s_uw,
+                                            const int* s_idx, int etid, bool& routing_pending) {
+    // partial of contributor q: CTA first_cta + q, its segment 0 if its range starts in this tile, else 1
+    const float* parts[C];
+#pragma unroll
+    for (int q = 0; q < C; ++q) {
+        const int cta = first_cta + min(q, c - 1);
+        const int seg = (int)(units * cta / M) / upt == tile ? 0 : 1;
+        parts[q] = part_g + ((size_t)cta * 2 + seg) * part_stride;
+    }
+    finish_rows<C, U>(p, parts, c, tile * kBM, q0, nq, ntok, slab, s_uw, s_idx, etid, routing_pending);
 }
 
 #ifdef METEORA_TRACE
@@ -407,22 +430,36 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         }
     } else {
         // ================================================================== main CTA
-        const int S = p.splits;
-        const int split = main_id % S;
-        const int tile_m = main_id / S;
-        const int ks0 = (int)(((long long)p.ksteps * split) / S);
-        const int ks1 = (int)(((long long)p.ksteps * (split + 1)) / S);
-        const int niter = (ks1 - ks0) / p.kc;
+        const int M = d.n_main, upt = d.upt;
+        const long long U = d.units;
+        const int u0 = (int)(U * main_id / M), u1 = (int)(U * (main_id + 1) / M);    // M <= U: never empty
+        const int n_it = u1 - u0;
+        const int tile_a = u0 / upt, tile_b = (u1 - 1) / upt;
+        const int nseg = tile_b - tile_a + 1;                                        // 1 or 2
+        const int it_switch = nseg > 1 ? (tile_a + 1) * upt - u0 : n_it;             // iterations of segment 0
         const RingGeom geom = {ring, bar_base, x_tile_bytes, stage_bytes, p.stages, p.kc, p.maps3d};
-        const uint32_t bar_acc = bar_base + 2 * p.stages * 8;
-        const size_t part_stride = (size_t)p.BN * kBM;                       // floats per partial tile
-        float* my_part = d.part_g + ((size_t)tile_m * S + split) * part_stride;
+        const uint32_t bar_acc = bar_base + 2 * p.stages * 8;                        // [0], [1]: one per segment
+        const size_t part_stride = (size_t)p.BN * kBM;                               // floats per partial tile
         if (warp == 0) {
             if (lane == 0) {
                 // let the stacked shrink get its loads into the memory queues first
                 bool ok = d.hold ? wait_counter(d.ctr + 3, n_active) : true;
                 if (tr_main) FUSED_STAMP(p, 32, 1);
-                ok = fused_producer(geom, &tmW0, &tmX, tile_m * kBM, ks0, niter, nullptr) && ok;
+                for (int it = 0; it < n_it && ok; ++it) {
+                    const int st = it % geom.stages, round = it / geom.stages;
+                    if (round > 0) ok = mbar_wait(bar_base + (geom.stages + st) * 8, (round & 1) ^ 1);
+                    if (!ok) break;
+                    const uint32_t full = bar_base + st * 8, dst = ring + st * stage_bytes;
+                    const int unit = u0 + it, tile = unit / upt, kstep = (unit - tile * upt) * p.kc;
+                    mbar_expect_tx(full, stage_bytes);
+                    if (p.maps3d) {
+                        tma_load_3d(dst, &tmW0, 0, tile * kBM, kstep, full);
+                        tma_load_3d(dst + p.kc * kWTileBytes, &tmX, 0, 0, kstep, full);
+                    } else {
+                        tma_load_2d(dst, &tmW0, kstep * kBK, tile * kBM, full);
+                        tma_load_2d(dst + kWTileBytes, &tmX, kstep * kBK, 0, full);
+                    }
+                }
                 if (!ok) flag_error(p, 1, 100);
                 if (!wait_counter(d.ctr + 1, n_active)) flag_error(p, 4, 800);              // routing published
                 if (tr_main) FUSED_STAMP(p, 32, 4);
@@ -445,58 +482,107 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             }
         } else if (warp == 1) {
             if (lane == 0) {
-                bool ok = fused_mma(geom, tmem_base, idesc, niter);
+                bool ok = true, seg0_done = false;
+                for (int it = 0; it < n_it; ++it) {
+                    const int st = it % geom.stages, round = it / geom.stages;
+                    ok = mbar_wait(bar_base + st * 8, round & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const bool second = it >= it_switch;
+                    const bool fresh = it == 0 || it == it_switch;                  // first MMA of a segment overwrites
+                    const uint32_t acc = tmem_base + (second ? (uint32_t)p.BN : 0u);
+                    const uint32_t wa = ring + st * stage_bytes, xa = wa + p.kc * kWTileBytes;
+                    for (int c = 0; c < p.kc; ++c) {
+                        const uint64_t da = smem_desc_sw128(wa + c * kWTileBytes);
+                        const uint64_t db = smem_desc_sw128(xa + c * x_tile_bytes);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / kUmmaK; ++kk)
+                            umma_bf16(acc, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, !fresh || (c | kk) != 0);
+                    }
+                    umma_commit(bar_base + (geom.stages + st) * 8);
+                    if (it == it_switch - 1) {                                      // segment 0 complete
+                        umma_commit(bar_acc);
+                        seg0_done = true;
+                    }
+                }
                 if (tr_main) FUSED_STAMP(p, 32, 2);
-                umma_commit(bar_acc);
+                if (!seg0_done) umma_commit(bar_acc);                               // only after a failed wait
+                if (nseg > 1) umma_commit(bar_acc + 8);
                 if (!ok) flag_error(p, 2, 200);
             }
         } else {
-            // B rows of the slice of the tile this CTA finishes, for every adapter: no routing needed yet
-            const int nrows = kBM / S, row_lo = nrows * split;
+            // Which rows of which tile this CTA finishes: tile `t` is shared by the CTAs owner(first unit) ..
+            // owner(last unit), in that order; contributor j of c takes the groups of 4 rows [32j/c, 32(j+1)/c).
+            int d_tile[2], d_first[2], d_c[2], d_q0[2], d_nq[2];
             uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
+            uint4* d_slab[2];
+            int slab_words = 0;
+            for (int sg = 0; sg < nseg; ++sg) {
+                const int tile = tile_a + sg;
+                const long long x0 = (long long)tile * upt, x1 = x0 + upt - 1;
+                const int first = (int)(((x0 + 1) * M + U - 1) / U) - 1, last = (int)(((x1 + 1) * M + U - 1) / U) - 1;
+                const int c = last - first + 1, j = main_id - first;
+                d_tile[sg] = tile;
+                d_first[sg] = first;
+                d_c[sg] = c;
+                d_q0[sg] = 32 * j / c;
+                d_nq[sg] = 32 * (j + 1) / c - d_q0[sg];
+                d_slab[sg] = slab + slab_words;
+                // B rows of that slice for every adapter: no routing needed yet
+                stage_slab_rows(p, d_slab[sg], tile * kBM + 4 * d_q0[sg], 4 * d_nq[sg], etid);
+                slab_words += p.N * 4 * d_nq[sg];
+            }
             float* s_uw = reinterpret_cast<float*>(epi + p.uw_off);
             int* s_idx = reinterpret_cast<int*>(epi + p.idx_off);
-            stage_slab_rows(p, slab, tile_m * kBM + row_lo, nrows, etid);
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
-            bool acc_ok = mbar_wait(bar_acc, 0);
-            if (!acc_ok && lane == 0) flag_error(p, 3, 300);
-            acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
-            tc_fence_after();
-            if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 5);
-            // Accumulators out of TMEM: to the fp32 scratch when the tile is split over several CTAs (lane =
-            // row, a warp writes 128 contiguous bytes per token), else to the idle ring.
-            float* part = S > 1 ? my_part : reinterpret_cast<float*>(ring_ptr);
+            // Accumulators out of TMEM to the fp32 scratch, segment by segment (lane = row, a warp writes 128
+            // contiguous bytes per token); each delivery bumps the tile's counter.
             const int row_in_tile = quad * 32 + lane;
-            for (int c = c_begin; c < c_end; c += 16) {
-                float v[16];
-                if (acc_ok) {
-                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
-                } else {
+            for (int sg = 0; sg < nseg; ++sg) {
+                bool acc_ok = mbar_wait(bar_acc + 8 * sg, 0);
+                if (!acc_ok && lane == 0) flag_error(p, 3, 300);
+                acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+                tc_fence_after();
+                if (etid == 0 && tr_main && sg == nseg - 1) FUSED_STAMP(p, 32, 5);
+                float* part = d.part_g + ((size_t)main_id * 2 + sg) * part_stride;
+                for (int c = c_begin; c < c_end; c += 16) {
+                    float v[16];
+                    if (acc_ok) {
+                        tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(sg * p.BN + c), v);
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c + i < ntok) part[(c + i) * kBM + row_in_tile] = v[i];
                 }
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (c + i < ntok) part[(c + i) * kBM + row_in_tile] = v[i];
-            }
-            epi_barrier();
-            if (etid == 0) {
-                if (S > 1) {
+                epi_barrier();
+                if (etid == 0) {
                     __threadfence();
-                    atomicAdd(d.tile_ctr + tile_m, 1);
+                    atomicAdd(d.tile_ctr + d_tile[sg], 1);
                 }
-                if (S > 1 && !wait_counter(d.tile_ctr + tile_m, S)) flag_error(p, 4, 900);  // all partials of the tile in
-                if (tr_main) FUSED_STAMP(p, 32, 6);
             }
-            epi_barrier();
-            const float* src = S > 1 ? d.part_g + (size_t)tile_m * S * part_stride : part;
-            const int nq = nrows / 4;
-            switch (S) {
-                case 1: finish_rows<1, 4>(p, src, part_stride, false, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
-                case 2: finish_rows<2, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
-                case 4: finish_rows<4, 4>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
-                default: finish_rows<8, 2>(p, src, part_stride, true, tile_m * kBM, row_lo, nq, ntok, slab, nrows, s_uw, s_idx, etid); break;
+            bool routing_pending = true;
+            for (int sg = 0; sg < nseg; ++sg) {
+                if (etid == 0) {
+                    if (!wait_counter(d.tile_ctr + d_tile[sg], d_c[sg])) flag_error(p, 4, 900);   // all partials of the tile in
+                    if (tr_main && sg == nseg - 1) FUSED_STAMP(p, 32, 6);
+                }
+                epi_barrier();
+                const int c = d_c[sg];
+                if (c <= 1)
+                    finish_tile<1, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                else if (c <= 2)
+                    finish_tile<2, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                else if (c <= 4)
+                    finish_tile<4, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                else if (c <= 8)
+                    finish_tile<8, 2>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                else
+                    finish_tile<16, 1>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
             }
+            if (routing_pending) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);
         }
     }

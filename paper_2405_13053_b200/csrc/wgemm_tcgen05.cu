@@ -1114,28 +1114,37 @@ static int max_resident_ctas(size_t smem) {
 
 struct FusedPlan {
     bool ok;
-    int why;   // why not: 1 knob/shape, 2 too many row tiles, 3 several token tiles, 4 residency, 5 operand sizes
-    Plan main;
-    int row_tiles, n_main, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages;
+    int why;   // why not: 1 knob/shape, 2 more row tiles than main CTAs, 4 residency, 5 shared memory
+    Plan main; // BN, stages, kc, maps3d, tmem_cols, staging offsets, smem of the decode kernel
+    int row_tiles, n_main, upt, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages;
 };
 
+// Launch plan of the single-launch decode kernel.  Main CTAs: as many as the SMs the aux CTAs leave, at most 14
+// per row tile (16 partial tiles is the most the last step sums) and at least one per row tile (a CTA's unit
+// range then spans at most two tiles).  Aux CTAs: about 20, the row tiles of the stacked shrink times up to 16
+// slices of the contraction axis.
 static FusedPlan make_fused_plan(const meteora_shape_t& s) {
+    const Tuning& tn = tuning();
     FusedPlan fp = {};
     fp.why = 1;
     // Measured on B200 (4096 -> 4096): the single launch is ahead of the three-launch chain at every decode
     // batch size (15.7 vs 16.5 us at T = 1, 19.5 vs 25 us at T = 128).
-    if (!tuning().fused) return fp;
-    if (!tc_path_supported(s) || s.T > 256 || s.r != 8 || tuning().simt_expand) return fp;
+    if (!tn.fused) return fp;
+    if (!tc_path_supported(s) || s.T > 256 || s.r != 8 || tn.simt_expand) return fp;
     fp.row_tiles = (s.d_out + kBM - 1) / kBM;
-    fp.why = 2;
     if (fp.row_tiles > kMaxFusedRowTiles) return fp;
-    fp.main = make_plan(fp.row_tiles, s.T, s.d_in, true, s.N, s.r, s.k, true);
-    fp.why = 3;
-    if (fp.main.n_tiles != 1) return fp;
-    fp.why = 4;
-    const int S = fp.main.splits;
-    fp.n_main = fp.row_tiles * S;
-    const int capacity = max_resident_ctas(fp.main.smem);
+    Plan& pl = fp.main;
+    const int sms = std::min(sm_count(), 148);                   // the workspace holds partial tiles for 148 CTAs
+    const int ksteps = (s.d_in + kBK - 1) / kBK;
+    pl.BN = std::min(256, (s.T + 15) / 16 * 16);
+    pl.n_tiles = 1;
+    pl.splits = 1;
+    pl.zsplits = 1;
+    pl.maps3d = (s.d_in % kBK) == 0 ? 1 : 0;
+    pl.kc = (pl.maps3d && ksteps % 2 == 0) ? 2 : 1;
+    if (tn.kc > 0 && pl.maps3d && ksteps % tn.kc == 0 && tn.kc <= 4) pl.kc = tn.kc;
+    fp.upt = ksteps / pl.kc;
+    // aux CTAs
     fp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
     // Wg rides behind A's last rows when the tile has room for it (N * r = 224, N = 28: rows 96..123 of tile 1)
     const int tail_rows = s.N * s.r - (fp.a_tiles - 1) * kBM;
@@ -1143,24 +1152,46 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.aux_tiles = merged ? fp.a_tiles : fp.a_tiles + 1;
     fp.gate_tile = fp.aux_tiles - 1;
     fp.gate_row0 = merged ? tail_rows : 0;
-    const int aux_tiles = fp.aux_tiles;
-    const int n_aux = std::min(capacity - fp.n_main, 24);
-    if (n_aux < aux_tiles) return fp;
-    const int ksteps = (s.d_in + kBK - 1) / kBK;
-    fp.aux_slices = std::min(std::min(n_aux / aux_tiles, ksteps), 16);   // 16: the selection reads all slices at once
-    fp.n_aux = aux_tiles * fp.aux_slices;
-    const size_t chunk = kWTileBytes + (size_t)fp.main.BN * 128;
-    const size_t ring_bytes = (size_t)fp.main.stages * fp.main.kc * chunk;
-    const int nks_aux = (ksteps + fp.aux_slices - 1) / fp.aux_slices;
-    fp.aux_stages = (int)std::min<size_t>(ring_bytes / chunk, (size_t)std::max(nks_aux, 1));
-    // the barrier block behind the ring was laid out for the main ring: keep the aux ring within it
-    const int bar_cap = (fp.main.epi_off - 16) / 8 - 3;
-    fp.aux_stages = std::min(fp.aux_stages, std::min(bar_cap / 2, 16));
+    fp.why = 2;
+    if (fp.aux_tiles + fp.row_tiles > sms) return fp;
+    const int aux_budget = std::min(std::max(20, fp.aux_tiles), sms - fp.row_tiles);
+    fp.aux_slices = std::min(std::min(aux_budget / fp.aux_tiles, ksteps), 16);   // 16: the selection reads all slices at once
+    if (fp.aux_slices < 1) return fp;
+    fp.n_aux = fp.aux_tiles * fp.aux_slices;
+    const long long units = (long long)fp.row_tiles * fp.upt;
+    int n_main = std::min(sms - fp.n_aux, 14 * fp.row_tiles);
+    if (tn.splits > 0) n_main = std::min(n_main, tn.splits * fp.row_tiles);
+    n_main = (int)std::min<long long>(n_main, units);
+    if (n_main < fp.row_tiles) return fp;
+    fp.n_main = n_main;
+    // shared memory: staged B rows (at most 128 rows of every adapter), routing, barriers, ring
     fp.why = 5;
-    if (fp.aux_stages < 1) return fp;
+    pl.slab_off = 0;
+    pl.uw_off = (int)align_up((size_t)s.N * kBM * 16, 16);
+    pl.idx_off = pl.uw_off + pl.BN * s.k * s.r * 4;
+    const size_t epi_bytes = (size_t)pl.idx_off + (size_t)pl.BN * s.k * 4;
+    pl.epi_off = (int)align_up((size_t)(2 * 16 + 3) * 8 + 16, 128);
+    const size_t fixed = 1024 + pl.epi_off + epi_bytes;
+    if (fixed + 48 * 1024 > 226 * 1024) return fp;
+    const size_t chunk = kWTileBytes + (size_t)pl.BN * 128;      // one k-step of both operands
+    const size_t stage_bytes = pl.kc * chunk;
+    const size_t avail = 226 * 1024 - fixed;
+    int stages = tn.stages > 0 ? tn.stages : (int)std::min<size_t>(avail / stage_bytes, 4);
+    stages = std::min(stages, 16);
+    if (stages < 2 || (size_t)stages * stage_bytes > avail) return fp;
+    pl.stages = stages;
+    const size_t ring_bytes = (size_t)stages * stage_bytes;
     // the aux CTAs' selection keeps one summed row of the stacked shrink per warp in the idle ring
     int col_logits = 0;
     if (ring_bytes < (size_t)(kThreads / 32) * tc_stacked_pitch(s, &col_logits) * sizeof(float)) return fp;
+    int cols = 32;
+    while (cols < 2 * pl.BN) cols *= 2;                           // two accumulators: one per segment of a unit range
+    pl.tmem_cols = cols;
+    pl.smem = 1024 + ring_bytes + pl.epi_off + epi_bytes;
+    const int nks_aux = (ksteps + fp.aux_slices - 1) / fp.aux_slices;
+    fp.aux_stages = (int)std::min<size_t>(std::min<size_t>(ring_bytes / chunk, 16), (size_t)std::max(nks_aux, 1));
+    fp.why = 4;
+    if (max_resident_ctas(pl.smem) < fp.n_main + fp.n_aux) return fp;
     fp.why = 0;
     fp.ok = true;
     return fp;
@@ -1174,10 +1205,10 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     const FusedPlan fp = make_fused_plan(s);
     if (fp.ok)
         return snprintf(buf, n,
-                        "path=fused_decode launches=1 main_ctas=%d splits=%d aux_ctas=%d aux_slices=%d tile_tokens=%d "
-                        "stages=%d kc=%d smem=%zu resident_ctas=%d",
-                        fp.n_main, fp.main.splits, fp.n_aux, fp.aux_slices, fp.main.BN, fp.main.stages, fp.main.kc,
-                        fp.main.smem, max_resident_ctas(fp.main.smem));
+                        "path=fused_decode launches=1 main_ctas=%d row_tiles=%d units_per_cta=%.1f aux_ctas=%d "
+                        "aux_slices=%d tile_tokens=%d stages=%d kc=%d smem=%zu resident_ctas=%d",
+                        fp.n_main, fp.row_tiles, (double)fp.row_tiles * fp.upt / fp.n_main, fp.n_aux, fp.aux_slices,
+                        fp.main.BN, fp.main.stages, fp.main.kc, fp.main.smem, max_resident_ctas(fp.main.smem));
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     return snprintf(buf, n,
@@ -1216,6 +1247,8 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.main.r = s.r;
     d.main.k = s.k;
     d.n_main = fp.n_main;
+    d.upt = fp.upt;
+    d.units = (long long)fp.row_tiles * fp.upt;
     d.n_aux = fp.n_aux;
     d.a_tiles = fp.a_tiles;
     d.a_rows = s.N * s.r;

@@ -246,11 +246,20 @@ def test_split_k_cluster_sizes_agree_with_oracle(splits, stages):
         mb.meteora_set_tuning("stages", 0)
 
 
-@pytest.mark.parametrize("T", [1, 8, 100, 256])
-def test_single_launch_decode_kernel_matches_oracle(T):
-    # fused = 2 forces the one-kernel decode path (base product + stacked shrink + selection) at every T <= 256
-    w = workloads.make_workload("fused", T=T, d_in=1024, d_out=640, dtype="bf16", x_kind="rms", seed=50 + T, b_std=0.3)
-    mb.meteora_set_tuning("fused", 2)
+# (d_in, d_out) chosen so that the unit ranges of the main CTAs fall every way they can: many CTAs per row tile
+# (640), a ragged last tile (1000), a contraction length that is no multiple of 64 (1096: plain 2-D tensor
+# maps, one k-step per stage), ranges that straddle two tiles (4224 = 33 tiles over 128 CTAs), more tiles than
+# half the CTAs (9000 = 71 tiles) and, with the "splits" knob capping the CTAs per tile, one CTA per tile.
+@pytest.mark.parametrize("d_in,d_out,T,per_tile", [
+    (1024, 640, 1, 0), (1024, 640, 8, 0), (1024, 640, 100, 0), (1024, 640, 256, 0),
+    (1536, 1000, 37, 0), (1096, 768, 16, 0), (2048, 4224, 5, 0), (2048, 4224, 128, 0),
+    (512, 9000, 24, 0), (1024, 1280, 64, 1), (1024, 1280, 200, 3),
+])
+def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
+    # one kernel per call: base product + stacked shrink + selection + LoRA expand
+    w = workloads.make_workload("fused", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="rms",
+                                seed=50 + T + d_out, b_std=0.3)
+    mb.meteora_set_tuning("splits", per_tile)
     try:
         shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
         assert "fused_decode" in mb.meteora_describe_plan(shape)
@@ -260,7 +269,18 @@ def test_single_launch_decode_kernel_matches_oracle(T):
         np.testing.assert_array_equal(y1, y2)                        # counters re-armed, result reproducible
         np.testing.assert_array_equal(i1, i2)
     finally:
-        mb.meteora_set_tuning("fused", 1)
+        mb.meteora_set_tuning("splits", 0)
+
+
+# Adapter counts that change the layout of the stacked shrink: Wg behind A's only tile (N = 4), Wg in a tile of
+# its own (N = 16: A fills its tile), three A tiles with Wg behind 8 rows (N = 33, logits beyond one warp).
+@pytest.mark.parametrize("N,k,T", [(4, 2, 9), (16, 4, 40), (33, 3, 130), (2, 1, 3)])
+def test_single_launch_decode_kernel_adapter_counts(N, k, T):
+    w = workloads.make_workload("fused_n", T=T, d_in=768, d_out=896, N=N, k=k, dtype="bf16", x_kind="normal",
+                                seed=900 + N, b_std=0.3)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    assert "fused_decode" in mb.meteora_describe_plan(shape)
+    check_forward(w, y_tol=1e-2)
 
 
 def test_chain_and_single_launch_paths_agree():
