@@ -1143,6 +1143,13 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     pl.maps3d = (s.d_in % kBK) == 0 ? 1 : 0;
     pl.kc = (pl.maps3d && ksteps % 2 == 0) ? 2 : 1;
     if (tn.kc > 0 && pl.maps3d && ksteps % tn.kc == 0 && tn.kc <= 4) pl.kc = tn.kc;
+    {
+        // staging of the last step (B rows, routing) comes first; with 256-token tiles two k-steps per stage
+        // would leave room for one stage only
+        const size_t staged = (size_t)s.N * kBM * 16 + (size_t)pl.BN * s.k * (s.r * 4 + 4) + 2048;
+        const size_t one = kWTileBytes + (size_t)pl.BN * 128;
+        while (pl.kc > 1 && staged + 2 * pl.kc * one > 226 * 1024) pl.kc /= 2;
+    }
     fp.upt = ksteps / pl.kc;
     // aux CTAs
     fp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
