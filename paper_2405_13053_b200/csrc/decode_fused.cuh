@@ -139,18 +139,20 @@ __device__ __forceinline__ void stage_slab_rows(const WGemmParams& p, uint4* sla
 // trip to L2; `parts` in CTA order, the first `c` are real), then their sum in that order, the expand of Eq. 2
 // from the staged B rows and the routing in shared memory, one rounding to bf16 and the store.  The routing is
 // staged by warp 0, which arrives on named barrier 2 when it is in shared memory; the threads here join that
-// barrier once (`routing_pending`), after issuing their first loads.
+// barrier once (`routing_pending`), after issuing their first loads.  `nthr` threads (etid = 0 .. nthr-1) share
+// the tile: all 256 epilogue threads, or half of them when the CTA finishes rows of two tiles at once.
 template <int C, int U>
 __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* const (&parts)[C], int c,
                                             int tile_row0, int q0, int nq, int ntok, const uint4* slab,
-                                            const float* s_uw, const int* s_idx, int etid, bool& routing_pending) {
+                                            const float* s_uw, const int* s_idx, int etid, int nthr,
+                                            bool& routing_pending) {
     const int items = nq * ntok, slab_rows = 4 * nq;
     const float4* s_uw4 = reinterpret_cast<const float4*>(s_uw);
-    for (int base = 0; base < items; base += kEpiThreads * U) {
+    for (int base = 0; base < items; base += nthr * U) {
         float4 v[U][C];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int it = min(base + etid + u * kEpiThreads, items - 1);
+            const int it = min(base + etid + u * nthr, items - 1);
             const int t = it / nq, ql = it - t * nq;
             const size_t off = (size_t)t * kBM + (q0 + ql) * 4;
 #pragma unroll
@@ -163,7 +165,7 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* c
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int it = base + etid + u * kEpiThreads;
+            const int it = base + etid + u * nthr;
             if (it >= items) break;
             const int t = it / nq, ql = it - t * nq;
             float4 acc = v[u][0];
@@ -205,7 +207,7 @@ template <int C, int U>
 __device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* part_g, size_t part_stride,
                                             long long units, int M, int upt, int tile, int first_cta, int c,
                                             int q0, int nq, int ntok, const uint4* slab, const float* s_uw,
-                                            const int* s_idx, int etid, bool& routing_pending) {
+                                            const int* s_idx, int etid, int nthr, bool& routing_pending) {
     // partial of contributor q: CTA first_cta + q, its segment 0 if its range starts in this tile, else 1
     const float* parts[C];
 #pragma unroll
@@ -214,7 +216,7 @@ __device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* p
         const int seg = (int)(units * cta / M) / upt == tile ? 0 : 1;
         parts[q] = part_g + ((size_t)cta * 2 + seg) * part_stride;
     }
-    finish_rows<C, U>(p, parts, c, tile * kBM, q0, nq, ntok, slab, s_uw, s_idx, etid, routing_pending);
+    finish_rows<C, U>(p, parts, c, tile * kBM, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
 }
 
 #ifdef METEORA_TRACE
@@ -563,24 +565,27 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                     atomicAdd(d.tile_ctr + d_tile[sg], 1);
                 }
             }
+            // Two tiles to finish: half of the epilogue threads each, side by side (one round trip to L2 for both).
             bool routing_pending = true;
-            for (int sg = 0; sg < nseg; ++sg) {
-                if (etid == 0) {
+            {
+                const int nthr = nseg > 1 ? kEpiThreads / 2 : kEpiThreads;
+                const int sg = nseg > 1 ? etid / nthr : 0, gtid = etid - sg * nthr;
+                if (gtid == 0) {
                     if (!wait_counter(d.tile_ctr + d_tile[sg], d_c[sg])) flag_error(p, 4, 900);   // all partials of the tile in
                     if (tr_main && sg == nseg - 1) FUSED_STAMP(p, 32, 6);
                 }
-                epi_barrier();
+                asm volatile("bar.sync %0, %1;" ::"r"(3 + sg), "r"(nthr) : "memory");
                 const int c = d_c[sg];
                 if (c <= 1)
-                    finish_tile<1, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                    finish_tile<1, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 2)
-                    finish_tile<2, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                    finish_tile<2, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 4)
-                    finish_tile<4, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                    finish_tile<4, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 8)
-                    finish_tile<8, 2>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                    finish_tile<8, 2>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else
-                    finish_tile<16, 1>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, etid, routing_pending);
+                    finish_tile<16, 1>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
             }
             if (routing_pending) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);

@@ -1272,7 +1272,9 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.topk_w = ws.topk_w;
     d.uw = ws.uw;
     d.inv_tau = 1.0f / s.temperature;
-    d.hold = tuning().no_hold ? 0 : 1;
+    // Holding the main CTAs back until the aux CTAs have issued their loads pays only while the base product is
+    // short: from about 64 MB of W0 on the routing is ready long before it is needed either way.
+    d.hold = (tuning().no_hold || (size_t)s.d_in * s.d_out * 2 > ((size_t)64 << 20)) ? 0 : 1;
     d.ctr = ws.status + 16;
     d.part_g = ws.part_g;
     d.tile_ctr = ws.tile_ctr;
