@@ -26,7 +26,7 @@ struct DecodeParams {
     WGemmParams main;      // base product: ring geometry, staging offsets, outputs
     int n_main;            // main CTAs (M)
     int upt;               // units per row tile = k-steps / kc
-    long long units;       // row tiles * upt (U)
+    int units;             // row tiles * upt (U); U * M stays below 2^31 (checked by the host)
     int n_aux;             // aux CTAs; they take the lowest block indices so that they are scheduled first
     int a_tiles, a_rows;   // row tiles / rows of the stacked A matrix (N * r rows)
     int aux_tiles;         // row tiles of the stacked shrink: a_tiles, plus one for Wg unless it fits behind A's last rows
@@ -205,7 +205,7 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* c
 
 template <int C, int U>
 __device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* part_g, size_t part_stride,
-                                            long long units, int M, int upt, int tile, int first_cta, int c,
+                                            int units, int M, int upt, int tile, int first_cta, int c,
                                             int q0, int nq, int ntok, const uint4* slab, const float* s_uw,
                                             const int* s_idx, int etid, int nthr, bool& routing_pending) {
     // partial of contributor q: CTA first_cta + q, its segment 0 if its range starts in this tile, else 1
@@ -213,7 +213,7 @@ __device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* p
 #pragma unroll
     for (int q = 0; q < C; ++q) {
         const int cta = first_cta + min(q, c - 1);
-        const int seg = (int)(units * cta / M) / upt == tile ? 0 : 1;
+        const int seg = (int)((unsigned)units * (unsigned)cta / (unsigned)M) / upt == tile ? 0 : 1;
         parts[q] = part_g + ((size_t)cta * 2 + seg) * part_stride;
     }
     finish_rows<C, U>(p, parts, c, tile * kBM, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
@@ -433,8 +433,9 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     } else {
         // ================================================================== main CTA
         const int M = d.n_main, upt = d.upt;
-        const long long U = d.units;
-        const int u0 = (int)(U * main_id / M), u1 = (int)(U * (main_id + 1) / M);    // M <= U: never empty
+        const unsigned U = (unsigned)d.units;
+        const int u0 = (int)(U * (unsigned)main_id / (unsigned)M);                   // M <= U: never empty
+        const int u1 = (int)(U * (unsigned)(main_id + 1) / (unsigned)M);
         const int n_it = u1 - u0;
         const int tile_a = u0 / upt, tile_b = (u1 - 1) / upt;
         const int nseg = tile_b - tile_a + 1;                                        // 1 or 2
@@ -521,8 +522,9 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
             int slab_words = 0;
             for (int sg = 0; sg < nseg; ++sg) {
                 const int tile = tile_a + sg;
-                const long long x0 = (long long)tile * upt, x1 = x0 + upt - 1;
-                const int first = (int)(((x0 + 1) * M + U - 1) / U) - 1, last = (int)(((x1 + 1) * M + U - 1) / U) - 1;
+                const unsigned x0 = (unsigned)(tile * upt), x1 = x0 + (unsigned)upt - 1u;
+                const int first = (int)(((x0 + 1u) * (unsigned)M + U - 1u) / U) - 1;
+                const int last = (int)(((x1 + 1u) * (unsigned)M + U - 1u) / U) - 1;
                 const int c = last - first + 1, j = main_id - first;
                 d_tile[sg] = tile;
                 d_first[sg] = first;
@@ -577,15 +579,15 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 asm volatile("bar.sync %0, %1;" ::"r"(3 + sg), "r"(nthr) : "memory");
                 const int c = d_c[sg];
                 if (c <= 1)
-                    finish_tile<1, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<1, 4>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 2)
-                    finish_tile<2, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<2, 4>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 4)
-                    finish_tile<4, 4>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<4, 4>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 8)
-                    finish_tile<8, 2>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<8, 2>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else
-                    finish_tile<16, 1>(p, d.part_g, part_stride, U, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<16, 1>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
             }
             if (routing_pending) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);

@@ -1169,7 +1169,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     int n_main = std::min(sms - fp.n_aux, 14 * fp.row_tiles);
     if (tn.splits > 0) n_main = std::min(n_main, tn.splits * fp.row_tiles);
     n_main = (int)std::min<long long>(n_main, units);
-    if (n_main < fp.row_tiles) return fp;
+    if (n_main < fp.row_tiles || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
     fp.n_main = n_main;
     // shared memory: staged B rows (at most 128 rows of every adapter), routing, barriers, ring
     fp.why = 5;
@@ -1255,7 +1255,7 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.main.k = s.k;
     d.n_main = fp.n_main;
     d.upt = fp.upt;
-    d.units = (long long)fp.row_tiles * fp.upt;
+    d.units = fp.row_tiles * fp.upt;
     d.n_aux = fp.n_aux;
     d.a_tiles = fp.a_tiles;
     d.a_rows = s.N * s.r;
