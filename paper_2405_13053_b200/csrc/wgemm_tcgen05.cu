@@ -1166,15 +1166,24 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     if (fp.aux_slices < 1) return fp;
     fp.n_aux = fp.aux_tiles * fp.aux_slices;
     const long long units = (long long)fp.row_tiles * fp.upt;
-    int n_main = std::min(sms - fp.n_aux, 14 * fp.row_tiles);
-    if (tn.splits > 0) n_main = std::min(n_main, tn.splits * fp.row_tiles);
+    // Main CTAs: at most 8 per row tile share a tile's rows in the last step.  A multiple of the row tiles keeps
+    // every CTA inside one tile (one accumulator, one finishing duty); it is taken unless it idles more than a
+    // tenth of the CTAs an uneven split would use (6 per tile keep any tile within 8 unit ranges).
+    const int m_max = sms - fp.n_aux;
+    const int m_even = fp.row_tiles * std::min(8, m_max / fp.row_tiles);
+    int n_main = std::min(m_max, 6 * fp.row_tiles);
+    if (m_even > 0 && m_even * 10 >= n_main * 9) n_main = m_even;
+    if (tn.splits > 0 && tn.splits * fp.row_tiles <= m_max) n_main = std::min(tn.splits, 8) * fp.row_tiles;
     n_main = (int)std::min<long long>(n_main, units);
     if (n_main < fp.row_tiles || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
     fp.n_main = n_main;
     // shared memory: staged B rows (at most 128 rows of every adapter), routing, barriers, ring
     fp.why = 5;
     pl.slab_off = 0;
-    pl.uw_off = (int)align_up((size_t)s.N * kBM * 16, 16);
+    // rows a CTA finishes: 128 / c when every tile belongs to exactly c CTAs, up to 128 (two tiles) otherwise
+    const bool whole = n_main % fp.row_tiles == 0;
+    const int own_rows = whole ? 4 * ((32 + n_main / fp.row_tiles - 1) / (n_main / fp.row_tiles)) : kBM;
+    pl.uw_off = (int)align_up((size_t)s.N * own_rows * 16, 16);
     pl.idx_off = pl.uw_off + pl.BN * s.k * s.r * 4;
     const size_t epi_bytes = (size_t)pl.idx_off + (size_t)pl.BN * s.k * 4;
     pl.epi_off = (int)align_up((size_t)(2 * 16 + 3) * 8 + 16, 128);
