@@ -1172,7 +1172,8 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     const int m_max = sms - fp.n_aux;
     const int m_even = fp.row_tiles * std::min(8, m_max / fp.row_tiles);
     int n_main = std::min(m_max, 6 * fp.row_tiles);
-    if (m_even > 0 && m_even * 10 >= n_main * 9) n_main = m_even;
+    // (large batches exchange 64 KB and more per partial tile: there even 80 % of the CTAs are the better deal)
+    if (m_even > 0 && m_even * 10 >= n_main * (s.T >= 96 ? 8 : 9)) n_main = m_even;
     if (tn.splits > 0 && tn.splits * fp.row_tiles <= m_max) n_main = std::min(tn.splits, 8) * fp.row_tiles;
     n_main = (int)std::min<long long>(n_main, units);
     if (n_main < fp.row_tiles || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
