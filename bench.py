@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "6d6996887df8804f", "bytes_per_launch": {"128": 38622464 + 44000}}
+NCU_TRAFFIC = {"kernel_sha": "be581c2719a90abe", "bytes_per_launch": {"128": 38643627 + 143019}}
 
 
 def parse_args():
