@@ -161,6 +161,34 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------------------------------------- rank plumbing
+def rank_info():
+    """(world size, rank, local rank) of this process as torchrun exports them; (1, 0, 0) when launched alone."""
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def module_seed(i, rank):
+    """Seed of module i on a rank: every rank works on modules of its own (token / module shards, no exchange)."""
+    return 1000 + 100 * i + 17 * rank
+
+
+def max_over_ranks(ms, world, device):
+    """The slowest rank's elapsed time: the job is as fast as its slowest shard."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(modules, tokens, world, steps, ms_total):
+    """Tokens through a MeteoRA linear per second, summed over all ranks."""
+    return modules * tokens * world * steps / (ms_total * 1e-3)
+
+
 # --------------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -170,9 +198,7 @@ def run_ours(args):
     from paper_2405_13053_b200 import build as lib_build
     from paper_2405_13053_b200 import workloads
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = rank_info()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
     torch.cuda.set_device(local)
@@ -195,7 +221,7 @@ def run_ours(args):
     host_w0 = None
     for i in range(R):
         w = workloads.make_workload(f"config1/T{T}/module{i}", T=T, d_in=D_IN, d_out=D_OUT, N=N_ADAPTERS, r=RANK,
-                                    k=TOPK, dtype="bf16", x_kind="rms", seed=1000 + 100 * i + 17 * rank)
+                                    k=TOPK, dtype="bf16", x_kind="rms", seed=module_seed(i, rank))
         if i == 0:
             host_w0 = w
         m = {n: torch.from_numpy(w[n]).to(dt).cuda() for n in ("x", "W0", "A", "B", "Wg")}
@@ -263,10 +289,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), world, "cuda")
 
     def check_status():
         for m in mods:
@@ -287,8 +310,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     clocks = sampler.stop()
     check_status()
-    tokens_per_step = R * T * world
-    value = tokens_per_step * K / (ms_total * 1e-3)
+    value = whole_job_value(R, T, world, K, ms_total)
 
     # ---- end to end: x from pinned host memory, y back to host, every step, through the host entry point
     run_e2e, mode_e2e = make_runner(step_host)
@@ -299,7 +321,7 @@ def run_ours(args):
 
     ms_e2e = timed(e2e_step, K, W)
     check_status()
-    e2e_value = tokens_per_step * K / (ms_e2e * 1e-3)
+    e2e_value = whole_job_value(R, T, world, K, ms_e2e)
 
     # ---- dominant kernel.  Which kernels a call launches depends on the shape (meteora_describe_plan):
     #   single-launch decode kernel: one launch is the whole call, so its average duration over the timed region
