@@ -135,8 +135,13 @@ int meteora_lora_delta_static(const void* x, const void* A, const void* B, const
  *   y[T,d_out] in shape->dtype.  workspace: device scratch of at least
  *   meteora_workspace_bytes(shape); calls that share a workspace must not overlap in time.
  * After the call the workspace holds the routing that was used (meteora_workspace_routing).
- * bf16 shapes with d_in % 8 == 0 and r % 8 == 0 run on the tensor-core path (TMA + tcgen05);
- * every other shape runs on a plain CUDA-core path with the same results up to rounding order.
+ * bf16 shapes with d_in % 8 == 0 and r % 8 == 0 run on the tensor-core paths (TMA + tcgen05):
+ * decode batches (T <= 256, rank 8, d_out <= 16384) as ONE cooperative kernel launch in which
+ * the CTAs exchange partial results through the workspace, everything else as three launches
+ * (stacked shrink [A; Wg] x, selection, base product with the LoRA expand).  Every other shape
+ * runs on a plain CUDA-core path with the same results up to rounding order.  The workspace header
+ * must have been zeroed once (meteora_workspace_init) before its first use; the kernels leave it
+ * ready for the next call.  meteora_describe_plan tells which path a shape takes.
  */
 int meteora_linear_forward(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                            const meteora_shape_t* shape, void* y, void* workspace, size_t workspace_bytes,
@@ -171,13 +176,16 @@ int meteora_workspace_init(void* workspace, void* stream);
 /*
  * Reads the workspace's device status word (SYNCHRONISES `stream`): METEORA_OK, or
  * METEORA_ERR_TIMEOUT if a bounded wait inside a kernel (an mbarrier of the TMA/tensor-core
- * pipeline) gave up, in which case the outputs of that call are invalid.  The word is cleared.
+ * pipeline, or a counter another CTA of the decode kernel bumps) gave up, in which case the
+ * outputs of that call are invalid.  The word is cleared; after a timeout call
+ * meteora_workspace_init again before the workspace's next use (the counters may be mid-count).
  */
 int meteora_workspace_status(void* workspace, void* stream);
 
 /*
- * Timing of the dominant kernel (the base product with its LoRA epilogue) for roofline reports.
- * Between meteora_profile_begin and meteora_profile_end every tensor-core meteora_linear_forward
+ * Timing of the base-product launch (the dominant kernel of the three-launch path) for roofline
+ * reports.  Between meteora_profile_begin and meteora_profile_end every meteora_linear_forward
+ * that takes the three-launch tensor-core path
  * records a CUDA event pair around that one launch on the caller's stream (up to max_launches
  * pairs; the launch is not overlapped with its predecessor while timed).  meteora_profile_end
  * SYNCHRONISES on the recorded events and returns the summed kernel time and the launch count.
@@ -195,11 +203,22 @@ int meteora_profile_end(float* total_ms, int* launches);
 int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_bytes);
 
 /*
- * Tuning knobs for measurements (process-wide, not thread-safe): "splits" (split-K cluster size,
- * 0 = automatic), "stages" (TMA ring depth, 0 = automatic), "tile_tokens" (tokens per tile, 0 =
- * automatic), "kc" (64-element k-chunks fetched per TMA copy: 1, 2 or 4; 0 = automatic), "force_simt" (1 = never take the tensor-core path), "pdl" (1 = overlap the chained
- * kernels of a call by programmatic dependent launch).  Unknown names return
- * METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
+ * Tuning knobs for measurements (process-wide, not thread-safe; 0 = automatic unless stated):
+ *   "splits"         split-K cluster size of the three-launch base product (1, 2, 4, 8); main CTAs
+ *                    per 128-row tile of the decode kernel
+ *   "stages"         TMA ring depth
+ *   "tile_tokens"    tokens per tile of the three-launch path
+ *   "kc"             64-element k-chunks fetched per TMA copy: 1, 2 or 4
+ *   "zmax"           cap on the contraction slices of the stacked shrink
+ *   "stacked_direct" 1 = decode-batch stacked shrink without clusters
+ *   "simt_expand"    1 = LoRA expand of the three-launch path on CUDA cores even for rank 8
+ *   "no_tma_store"   1 = plain stores of y where the TMA store would apply
+ *   "force_simt"     1 = never take a tensor-core path
+ *   "pdl"            default 1 = the three launches of a call overlap by programmatic dependent launch
+ *   "fused"          default 1; 0 = never use the single-launch decode kernel
+ *   "coop"           default 1; 0 = launch the decode kernel without the co-residency guarantee
+ *   "no_hold"        1 = the decode kernel's main CTAs do not wait for the aux CTAs' first loads
+ * Unknown names return METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
  */
 int meteora_set_tuning(const char* name, int value);
 
