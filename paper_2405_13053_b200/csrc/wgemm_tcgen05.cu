@@ -697,6 +697,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
 }  // namespace meteora
 
 #include "decode_fused.cuh"
+#include "wgemm_pair.cuh"
 
 namespace meteora {
 
@@ -1051,8 +1052,85 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     return launch_wgemm(mA, mG, mX, mX, p, row_tiles, pl, false, st);
 }
 
+// Prefill batches on pairs of SMs (wgemm_pair.cuh): 256 x 256 tiles, rank 8, y stored by TMA.
+struct PairPlan {
+    bool ok;
+    int stages, na, epi_off;
+    size_t smem;
+};
+static PairPlan make_pair_plan(const meteora_shape_t& s) {
+    PairPlan pp = {};
+    if (!tuning().pair || tuning().simt_expand || tuning().no_tma_store || tuning().tile_tokens || tuning().splits > 1)
+        return pp;
+    if (!tc_path_supported(s) || s.r != 8 || s.T <= 256 || s.d_out % 8 != 0) return pp;
+    pp.na = (s.N + 1) / 2 * 2;
+    const size_t slab = (size_t)pp.na * kBM * 16, us = (size_t)pp.na * kPairHalf * 16;
+    const size_t ystage = (size_t)kPairTokens * kBM * 2, stage = kWTileBytes + kPairHalf * 128;
+    for (int stages = 6; stages >= 2; --stages) {
+        const size_t epi_off = align_up((size_t)(2 * stages + 3) * 8 + 16, 128);
+        const size_t smem = 1024 + stages * stage + epi_off + slab;
+        if (smem <= 226 * 1024 && stages * stage >= std::max(us, ystage)) {
+            pp.stages = tuning().stages > 1 && tuning().stages < stages ? tuning().stages : stages;
+            pp.epi_off = (int)align_up((size_t)(2 * pp.stages + 3) * 8 + 16, 128);
+            pp.smem = 1024 + pp.stages * stage + pp.epi_off + slab;
+            pp.ok = pp.stages * stage >= std::max(us, ystage);
+            return pp;
+        }
+    }
+    return pp;
+}
+
+static int launch_base_lora_pair(const void* x, const void* W0, const void* B, const meteora_shape_t& s,
+                                 const Workspace& ws, void* y, const PairPlan& pp, bool pdl, cudaStream_t st) {
+    const int row_tiles = (s.d_out + kBM - 1) / kBM;
+    CUtensorMap mW, mX, mY;
+    int rc;
+    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, 0, &mW)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, kPairHalf, 0, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_store_map(y, s.d_out, s.T, kPairTokens, &mY)) != METEORA_OK) return rc;
+    PairParams p = {};
+    p.T = s.T;
+    p.K = s.d_in;
+    p.ksteps = (s.d_in + kBK - 1) / kBK;
+    p.stages = pp.stages;
+    p.d_out = s.d_out;
+    p.N = s.N;
+    p.k = s.k;
+    p.na = pp.na;
+    p.row_tiles = row_tiles;
+    p.epi_off = pp.epi_off;
+    p.slab_off = 0;
+    p.topk_idx = ws.topk_idx;
+    p.uw = ws.uw;
+    p.B = (const __nv_bfloat16*)B;
+    p.status = ws.status;
+    p.pdl_wait = pdl ? 1 : 0;
+    static int smem_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (!smem_set[dev]) {
+        if (cudaFuncSetAttribute(k_wgemm_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            return METEORA_ERR_CUDA;
+        smem_set[dev] = 1;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * ((row_tiles + 1) / 2), (s.T + kPairTokens - 1) / kPairTokens, 1);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = pp.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_wgemm_pair, mW, mX, mY, p));
+}
+
 int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
                         void* y, bool pdl, cudaStream_t st) {
+    const PairPlan pp = make_pair_plan(s);
+    if (pp.ok) return launch_base_lora_pair(x, W0, B, s, ws, y, pp, pdl, st);
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     CUtensorMap mW, mX;
@@ -1227,6 +1305,12 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
                         fp.n_main, fp.row_tiles, (double)fp.row_tiles * fp.upt / fp.n_main, fp.n_aux, fp.aux_slices,
                         fp.main.BN, fp.main.stages, fp.main.kc, fp.main.smem, max_resident_ctas(fp.main.smem));
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
+    const PairPlan pp = make_pair_plan(s);
+    if (pp.ok)
+        return snprintf(buf, n,
+                        "path=chain(not fused: reason %d) launches=3 base=pairs_of_ctas pairs=%d tile=256x256 stages=%d "
+                        "smem=%zu expand=mma",
+                        fp.why, (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens), pp.stages, pp.smem);
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     return snprintf(buf, n,
                     "path=chain(not fused: reason %d) launches=3 base_ctas=%d cluster=%d tile_tokens=%d stages=%d kc=%d "

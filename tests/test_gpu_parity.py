@@ -283,6 +283,27 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T):
     check_forward(w, y_tol=1e-2)
 
 
+# Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
+# one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
+# (257), a contraction length that is no multiple of 64, and adapters up to an odd count.
+@pytest.mark.parametrize("d_in,d_out,T,N,k", [
+    (1024, 640, 600, 28, 2), (512, 256, 257, 28, 2), (1096, 512, 300, 28, 2), (768, 1024, 1024, 7, 3),
+])
+def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
+    w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, dtype="bf16", x_kind="normal",
+                                seed=700 + T, b_std=0.3)
+    mb.meteora_set_tuning("pair", 1)
+    try:
+        shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+        assert "pairs_of_ctas" in mb.meteora_describe_plan(shape)
+        check_forward(w, y_tol=1e-2)
+        y1, i1, _ = run_forward(w)
+        y2, i2, _ = run_forward(w)
+        np.testing.assert_array_equal(y1, y2)
+    finally:
+        mb.meteora_set_tuning("pair", 0)
+
+
 def test_chain_and_single_launch_paths_agree():
     w = workloads.config1(128)
     y_f, i_f, _ = run_forward(w)                                     # T = 128 takes the single launch by default
