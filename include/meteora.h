@@ -218,6 +218,8 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "fused"          default 1; 0 = never use the single-launch decode kernel
  *   "coop"           default 1; 0 = launch the decode kernel without the co-residency guarantee
  *   "no_hold"        1 = the decode kernel's main CTAs do not wait for the aux CTAs' first loads
+ *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)
+ *                    where the pairs cover a quarter of the SMs; 0 = never; 2 = wherever the shape allows
  * Unknown names return METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
  */
 int meteora_set_tuning(const char* name, int value);

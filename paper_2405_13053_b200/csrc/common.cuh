@@ -86,7 +86,8 @@ struct Tuning {
     int pdl = 1;
     int fused = 1;           // 0: never use the single-launch decode kernel
     int coop = 1;            // 0 (measurement only): launch it without the co-residency guarantee
-    int pair = 0;            // 1: prefill base product on pairs of SMs (256 x 256 tiles, two-CTA MMA)
+    int pair = 1;            // prefill base product on pairs of SMs (256 x 256 tiles, two-CTA MMA): 0 never, 1 where
+                             // the pairs cover enough SMs, 2 wherever the shape allows
     int no_hold = 0;         // 1 (measurement only): main CTAs of the decode kernel do not wait for the aux CTAs' first loads
     int fused_refused = 0;   // cooperative launches the driver refused (the chain ran instead)
 };

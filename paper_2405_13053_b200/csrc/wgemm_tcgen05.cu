@@ -1063,6 +1063,10 @@ static PairPlan make_pair_plan(const meteora_shape_t& s) {
     if (!tuning().pair || tuning().simt_expand || tuning().no_tma_store || tuning().tile_tokens || tuning().splits > 1)
         return pp;
     if (!tc_path_supported(s) || s.r != 8 || s.T <= 256 || s.d_out % 8 != 0) return pp;
+    // Measured on B200: ahead of the one-CTA tiles (by 8 - 17 %, and by more where those fall back to 128-token
+    // tiles) as soon as the pairs cover a quarter of the SMs; below that too few SMs work at all.
+    const int pairs = ((s.d_out + 2 * kBM - 1) / (2 * kBM)) * ((s.T + kPairTokens - 1) / kPairTokens);
+    if (tuning().pair == 1 && pairs * 4 < sm_count()) return pp;
     pp.na = (s.N + 1) / 2 * 2;
     const size_t slab = (size_t)pp.na * kBM * 16, us = (size_t)pp.na * kPairHalf * 16;
     const size_t ystage = (size_t)kPairTokens * kBM * 2, stage = kWTileBytes + kPairHalf * 128;

@@ -292,7 +292,7 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T):
 def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
     w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, dtype="bf16", x_kind="normal",
                                 seed=700 + T, b_std=0.3)
-    mb.meteora_set_tuning("pair", 1)
+    mb.meteora_set_tuning("pair", 2)                                 # 2: also where only a few pairs result
     try:
         shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
         assert "pairs_of_ctas" in mb.meteora_describe_plan(shape)
@@ -301,7 +301,21 @@ def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
         y2, i2, _ = run_forward(w)
         np.testing.assert_array_equal(y1, y2)
     finally:
-        mb.meteora_set_tuning("pair", 0)
+        mb.meteora_set_tuning("pair", 1)
+
+
+@pytest.mark.parametrize("d_in,d_out,T", [(1024, 640, 600), (1096, 512, 300)])
+def test_prefill_on_single_sms_matches_oracle(d_in, d_out, T):
+    # the 128 x 256 tiles of one CTA each, which small prefill problems still take by default
+    w = workloads.make_workload("single", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="normal",
+                                seed=800 + T, b_std=0.3)
+    mb.meteora_set_tuning("pair", 0)
+    try:
+        shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+        assert "pairs_of_ctas" not in mb.meteora_describe_plan(shape)
+        check_forward(w, y_tol=1e-2)
+    finally:
+        mb.meteora_set_tuning("pair", 1)
 
 
 def test_chain_and_single_launch_paths_agree():
