@@ -296,4 +296,162 @@ k_wgemm_pair(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CU
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Stacked shrink [A_0..A_{N-1}; Wg] x for prefill batches on pairs of SMs: the 256 rows of a pair tile are two
+// 128-row tiles of the stacked matrix (for N = 28, rank 8 that is all of it: A's rows 0..127 in the leader,
+// A's rows 128..223 followed by the 28 rows of Wg in its peer), the 256 tokens are split as above.  Slices of
+// the contraction axis go over grid z; each writes its fp32 partial straight from TMEM to u_all[z].
+// ------------------------------------------------------------------------------------------------
+struct StackedPairParams {
+    int T, ksteps, stages, zsplits;
+    int a_tiles, a_rows, aux_tiles, gate_tile, gate_row0, N;
+    float* u_all;
+    size_t zstride;
+    int ld_u, col_logits;
+    int32_t* status;
+    int pdl_trigger;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads)
+k_stacked_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAt,
+               const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmX,
+               const StackedPairParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;
+    uint8_t* ring_ptr = smem_raw + (ring - raw);
+    constexpr uint32_t kXHalfBytes = kPairHalf * 128;
+    constexpr uint32_t kStageBytes = kWTileBytes + kXHalfBytes;
+    const uint32_t ring_bytes = p.stages * kStageBytes;
+    const uint32_t bar_base = ring + ring_bytes;                  // full[stages], empty[stages], acc
+    const uint32_t bar_acc = bar_base + 2 * p.stages * 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + (2 * p.stages + 1) * 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const bool leader = rank == 0;
+    const int tile = (blockIdx.x >> 1) * 2 + (int)rank;           // own 128 rows of the stacked matrix
+    const int tok0 = blockIdx.y * kPairTokens;
+    const int tokh = tok0 + (int)rank * kPairHalf;
+    const int ks0 = (int)(((long long)p.ksteps * blockIdx.z) / p.zsplits);
+    const int ks1 = (int)(((long long)p.ksteps * (blockIdx.z + 1)) / p.zsplits);
+    const int niter = ks1 - ks0;
+
+    if (p.pdl_trigger && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(bar_base + s * 8, 1);
+            mbar_init(bar_base + (p.stages + s) * 8, 1);
+        }
+        mbar_init(bar_acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"((uint32_t)kPairTokens)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // Own tile of the stacked matrix: rows of A (the last A tile through the map whose box stops at A's
+            // last row when Wg follows in the same tile), rows of Wg, or nothing but zero fill (a tile past
+            // the end reads A out of range).  Every stage is 16 KB of weights + 16 KB of tokens whatever the tile.
+            const bool has_a = tile < p.a_tiles || tile != p.gate_tile;
+            const bool merged_tail = tile == p.a_tiles - 1 && tile == p.gate_tile;
+            const CUtensorMap* mA = merged_tail ? &tmAt : &tmA;
+            bool ok = true;
+            int issued = 0;
+            for (int i = 0; i < niter; ++i) {
+                const int s = i % p.stages, round = i / p.stages;
+                if (round > 0) ok = mbar_wait(bar_base + (p.stages + s) * 8, (round & 1) ^ 1);
+                if (!ok) break;
+                const uint32_t full = bar_base + s * 8;
+                const uint32_t full_leader = map_to_cta(full, 0);
+                const uint32_t dst = ring + s * kStageBytes;
+                const int c0 = (ks0 + i) * kBK;
+                if (leader) mbar_expect_tx(full, 2 * kStageBytes);
+                if (has_a) tma_load_2d_pair(dst, mA, c0, tile * kBM, full_leader);
+                if (tile == p.gate_tile) tma_load_2d_pair(dst + (uint32_t)p.gate_row0 * 128u, &tmG, c0, 0, full_leader);
+                tma_load_2d_pair(dst + kWTileBytes, &tmX, c0, tokh, full_leader);
+                issued = i + 1;
+            }
+            if (!ok) {
+                atomicExch(p.status, 1);
+                atomicExch(p.status + 1, 2100 + issued);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && leader) {
+            const uint32_t idesc = instr_desc_bf16_pair();
+            bool ok = true;
+            for (int i = 0; i < niter; ++i) {
+                const int s = i % p.stages, round = i / p.stages;
+                ok = mbar_wait(bar_base + s * 8, round & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t wa = ring + s * kStageBytes, xa = wa + kWTileBytes;
+                const uint64_t da = smem_desc_sw128(wa), db = smem_desc_sw128(xa);
+#pragma unroll
+                for (int kk = 0; kk < kBK / kUmmaK; ++kk)
+                    umma_bf16_pair(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (i | kk) != 0);
+                umma_commit_pair(bar_base + (p.stages + s) * 8);
+            }
+            umma_commit_pair(bar_acc);
+            if (!ok) {
+                atomicExch(p.status, 1);
+                atomicExch(p.status + 2, 2200);
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        bool acc_ok = mbar_wait(bar_acc, 0);
+        if (!acc_ok && lane == 0) {
+            atomicExch(p.status, 1);
+            atomicExch(p.status + 3, 2300);
+        }
+        acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+        tc_fence_after();
+        // accumulators straight to u_all[z]: lane = row of the tile = column of u_all, 128 contiguous bytes per warp
+        const int trow = quad * 32 + lane;
+        int col = -1;                                                        // -1: padding row
+        if (tile < p.a_tiles && tile * kBM + trow < p.a_rows && !(tile == p.gate_tile && trow >= p.gate_row0))
+            col = tile * kBM + trow;
+        if (tile == p.gate_tile && trow >= p.gate_row0 && trow < p.gate_row0 + p.N)
+            col = p.col_logits + trow - p.gate_row0;
+        float* dst = p.u_all + (size_t)blockIdx.z * p.zstride + (size_t)tok0 * p.ld_u + max(col, 0);
+        const int ntok = min(kPairTokens, p.T - tok0);
+        const int c_begin = warp < 6 ? 0 : kPairTokens / 2, c_end = warp < 6 ? kPairTokens / 2 : kPairTokens;
+        for (int c = c_begin; c < c_end; c += 16) {
+            float v[16];
+            if (acc_ok && niter > 0) {
+                tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = 0.f;
+            }
+            if (col >= 0) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (c + i < ntok) dst[(size_t)(c + i) * p.ld_u] = v[i];
+            }
+        }
+    }
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"((uint32_t)kPairTokens)
+                     : "memory");
+    }
+}
+
 }  // namespace meteora

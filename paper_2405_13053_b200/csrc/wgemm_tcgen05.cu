@@ -835,7 +835,8 @@ struct Plan {
 // decode batch; for larger batches as many as it takes to reach one CTA per SM with 256-token tiles.
 int stacked_zsplits_bound(int T) {
     if (T <= 256) return kMaxZSplits;
-    const int tiles = 3 * ((T + 255) / 256);
+    // prefill: one pair of CTAs (or three single CTAs) per 256 tokens; slices until about one CTA per SM
+    const int tiles = 2 * ((T + 255) / 256);
     return std::min(kMaxZSplits, std::max(1, 148 / tiles));
 }
 
@@ -998,7 +999,78 @@ static int launch_wgemm(const CUtensorMap& m0, const CUtensorMap& m1, const CUte
 
 static int stacked_row_tiles(const meteora_shape_t& s) { return (s.N * s.r + kBM - 1) / kBM + 1; }
 
+// Stacked shrink of a prefill batch on pairs of SMs (k_stacked_pair).
+struct StackedPairPlan {
+    bool ok;
+    int a_tiles, aux_tiles, gate_tile, gate_row0, zsplits, stages;
+    size_t smem;
+};
+static StackedPairPlan make_stacked_pair_plan(const meteora_shape_t& s) {
+    StackedPairPlan sp = {};
+    if (!tuning().pair || tuning().stacked_direct || !tc_path_supported(s) || s.r != 8 || s.T <= 256) return sp;
+    sp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
+    const int tail_rows = s.N * s.r - (sp.a_tiles - 1) * kBM;
+    const bool merged = tail_rows % 8 == 0 && tail_rows + s.N <= kBM;
+    sp.aux_tiles = merged ? sp.a_tiles : sp.a_tiles + 1;
+    sp.gate_tile = sp.aux_tiles - 1;
+    sp.gate_row0 = merged ? tail_rows : 0;
+    const int ksteps = (s.d_in + kBK - 1) / kBK;
+    const int pairs = ((sp.aux_tiles + 1) / 2) * ((s.T + kPairTokens - 1) / kPairTokens);
+    const int zcap = tuning().zmax > 0 ? std::min(tuning().zmax, kMaxZSplits) : kMaxZSplits;
+    const int fill = std::max(1, sm_count() / (2 * pairs));
+    sp.zsplits = std::min(std::min(zcap, std::min(fill, stacked_zsplits_bound(s.T))), std::max(1, ksteps / 4));
+    sp.stages = std::min(6, std::max(2, (ksteps + sp.zsplits - 1) / sp.zsplits));
+    sp.smem = 1024 + (size_t)sp.stages * (kWTileBytes + kPairHalf * 128) + 256;
+    sp.ok = true;
+    return sp;
+}
+
+static int launch_stacked_shrink_pair(const void* x, const void* A, const void* Wg, const meteora_shape_t& s,
+                                      const Workspace& ws, const StackedPairPlan& sp, cudaStream_t st) {
+    CUtensorMap mA, mAt, mG, mX;
+    int rc;
+    const int tail_box = sp.gate_row0 > 0 ? sp.gate_row0 : kBM, gate_box = kBM - sp.gate_row0;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, 0, &mA)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, tail_box, 0, &mAt)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Wg, s.d_in, s.N, gate_box, 0, &mG)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, kPairHalf, 0, &mX)) != METEORA_OK) return rc;
+    StackedPairParams p = {};
+    p.T = s.T;
+    p.ksteps = (s.d_in + kBK - 1) / kBK;
+    p.stages = sp.stages;
+    p.zsplits = sp.zsplits;
+    p.a_tiles = sp.a_tiles;
+    p.a_rows = s.N * s.r;
+    p.aux_tiles = sp.aux_tiles;
+    p.gate_tile = sp.gate_tile;
+    p.gate_row0 = sp.gate_row0;
+    p.N = s.N;
+    p.u_all = ws.u_all;
+    p.zstride = (size_t)s.T * ws.ld_u;
+    p.ld_u = ws.ld_u;
+    p.col_logits = ws.col_logits;
+    p.status = ws.status;
+    p.pdl_trigger = tuning().pdl ? 1 : 0;
+    static int smem_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (!smem_set[dev]) {
+        if (cudaFuncSetAttribute(k_stacked_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            return METEORA_ERR_CUDA;
+        smem_set[dev] = 1;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * ((sp.aux_tiles + 1) / 2), (s.T + kPairTokens - 1) / kPairTokens, sp.zsplits);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = sp.smem;
+    cfg.stream = st;
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_stacked_pair, mA, mAt, mG, mX, p));
+}
+
 int tc_stacked_zsplits(const meteora_shape_t& s) {
+    const StackedPairPlan sp = make_stacked_pair_plan(s);
+    if (sp.ok) return sp.zsplits;
     return make_plan(stacked_row_tiles(s), s.T, s.d_in, false, s.N, s.r, s.k).zsplits;
 }
 
@@ -1028,6 +1100,8 @@ static void fill_common(WGemmParams& p, const Plan& pl, int T, int K, int32_t* s
 
 int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const meteora_shape_t& s,
                              const Workspace& ws, cudaStream_t st) {
+    const StackedPairPlan sp = make_stacked_pair_plan(s);
+    if (sp.ok) return launch_stacked_shrink_pair(x, A, Wg, s, ws, sp, st);
     const int a_rows = s.N * s.r;
     const int a_tiles = (a_rows + kBM - 1) / kBM;
     const int row_tiles = a_tiles + 1;

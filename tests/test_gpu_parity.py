@@ -285,9 +285,11 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T):
 
 # Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
 # one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
-# (257), a contraction length that is no multiple of 64, and adapters up to an odd count.
+# (257), a contraction length that is no multiple of 64, and adapters up to an odd count.  The stacked shrink of
+# these calls runs on pairs as well: its rows are [A; Wg] packed into 128-row tiles, two tiles per pair.
 @pytest.mark.parametrize("d_in,d_out,T,N,k", [
     (1024, 640, 600, 28, 2), (512, 256, 257, 28, 2), (1096, 512, 300, 28, 2), (768, 1024, 1024, 7, 3),
+    (512, 512, 520, 16, 4), (512, 384, 300, 33, 3),      # Wg in a tile of its own; three tiles of stacked rows
 ])
 def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
     w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, dtype="bf16", x_kind="normal",
