@@ -1008,6 +1008,9 @@ struct StackedPairPlan {
 static StackedPairPlan make_stacked_pair_plan(const meteora_shape_t& s) {
     StackedPairPlan sp = {};
     if (!tuning().pair || tuning().stacked_direct || !tc_path_supported(s) || s.r != 8 || s.T <= 256) return sp;
+    // measured: below about a thousand tokens the pairs' set-up (cluster launch, two cluster barriers) costs
+    // 2 - 3 us more than it saves
+    if (tuning().pair == 1 && s.T < 1024) return sp;
     sp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
     const int tail_rows = s.N * s.r - (sp.a_tiles - 1) * kBM;
     const bool merged = tail_rows % 8 == 0 && tail_rows + s.N <= kBM;
