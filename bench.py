@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "be581c2719a90abe", "bytes_per_launch": {"128": 38643627 + 143019}}
+NCU_TRAFFIC = {"kernel_sha": "d04cced59db3560b", "bytes_per_launch": {"128": 38644224 + 52736}}
 
 
 def parse_args():
@@ -77,7 +77,7 @@ def measured_tensor_peak():
 
 def kernel_sha():
     h = hashlib.sha256()
-    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "select.cuh"):
+    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "wgemm_pair.cuh", "select.cuh"):
         with open(os.path.join(ROOT, "paper_2405_13053_b200", "csrc", name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -335,7 +335,8 @@ def run_ours(args):
         kernel_name = "k_decode_fused (base product + stacked shrink + selection + LoRA expand, one launch per call)"
         kernel_ms, kernel_launches = ms_total, K * R
     else:
-        kernel_name = "k_wgemm (base product + LoRA expand epilogue)"
+        kernel_name = ("k_wgemm_pair (base product + LoRA expand on pairs of SMs)" if "pairs_of_ctas" in plan
+                       else "k_wgemm (base product + LoRA expand)")
         prof_steps = min(K, 8)
         step_device()
         torch.cuda.synchronize()
@@ -356,7 +357,13 @@ def run_ours(args):
     bytes_path = bytes_base + (N_ADAPTERS * D_IN + touched * RANK * D_IN) * es
     bytes_kernel = bytes_path if single_launch else bytes_base
     peak, peak_kind = measured_peaks()
+    tc_peak, tc_kind = measured_tensor_peak()
     per_launch_s = kernel_ms * 1e-3 / max(kernel_launches, 1)
+    flops_base = 2.0 * T * D_IN * D_OUT + 2.0 * T * TOPK * RANK * D_OUT
+    flops_path = flops_base + 2.0 * T * N_ADAPTERS * D_IN + 2.0 * T * TOPK * RANK * D_IN
+    flops_kernel = flops_path if single_launch else flops_base
+    # the bound of the kernel: whichever of its algorithmic bytes / HBM and flops / tensor peak takes longer
+    tensor_bound = flops_kernel / (tc_peak * 1e12) > bytes_kernel / (peak * 1e9)
     achieved = bytes_kernel / per_launch_s / 1e9
     traffic = None
     if NCU_TRAFFIC["kernel_sha"] == kernel_sha() and single_launch:
@@ -368,7 +375,7 @@ def run_ours(args):
         "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"config1: LLaMA3-8B q_proj MeteoRA linear 4096->4096, N=28 r=8 k=2, bf16, "
-                               f"decode batch T={T}; step = {R} independent modules",
+                               f"{'decode' if T <= 256 else 'prefill'} batch T={T}; step = {R} independent modules",
                    "tokens_per_module": T, "modules_per_step": R, "launch": mode, "e2e_launch": mode_e2e,
                    "l2": f"weights of the {R} modules total {R * bytes_path / 1e6:.0f} MB > 126 MB L2, "
                          "so no weight is L2-resident between visits",
@@ -377,13 +384,22 @@ def run_ours(args):
                 "d2h_bytes_per_step": R * T * D_OUT * es, "ms_per_step": ms_e2e / K},
         "gpu_launches": launches_per_call * R * K,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved,
-                     "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "algorithmic_bytes_per_launch": bytes_kernel,
-                     "us_per_launch": per_launch_s * 1e6, "launches_timed": kernel_launches},
-        "path_roofline": {"bound": "hbm", "algorithmic_bytes_per_call": bytes_path, "us_per_call": per_call_s * 1e6,
-                          "achieved": bytes_path / per_call_s / 1e9, "peak": peak, "unit": "GB/s",
-                          "frac": bytes_path / per_call_s / 1e9 / peak, "adapters_touched": touched},
+        "roofline": ({"bound": "tensor", "kernel": kernel_name, "achieved": flops_kernel / per_launch_s / 1e12,
+                      "peak": tc_peak, "peak_kind": f"of {tc_kind} (sustained dense bf16)", "unit": "TFLOP/s",
+                      "frac": flops_kernel / per_launch_s / 1e12 / tc_peak, "traffic": None,
+                      "algorithmic_flops_per_launch": flops_kernel, "us_per_launch": per_launch_s * 1e6,
+                      "launches_timed": kernel_launches} if tensor_bound else
+                     {"bound": "hbm", "kernel": kernel_name, "achieved": achieved,
+                      "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                      "traffic": traffic, "algorithmic_bytes_per_launch": bytes_kernel,
+                      "us_per_launch": per_launch_s * 1e6, "launches_timed": kernel_launches}),
+        "path_roofline": ({"bound": "tensor", "algorithmic_flops_per_call": flops_path, "us_per_call": per_call_s * 1e6,
+                           "achieved": flops_path / per_call_s / 1e12, "peak": tc_peak, "unit": "TFLOP/s",
+                           "frac": flops_path / per_call_s / 1e12 / tc_peak, "adapters_touched": touched}
+                          if flops_path / (tc_peak * 1e12) > bytes_path / (peak * 1e9) else
+                          {"bound": "hbm", "algorithmic_bytes_per_call": bytes_path, "us_per_call": per_call_s * 1e6,
+                           "achieved": bytes_path / per_call_s / 1e9, "peak": peak, "unit": "GB/s",
+                           "frac": bytes_path / per_call_s / 1e9 / peak, "adapters_touched": touched}),
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
