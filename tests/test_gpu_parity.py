@@ -309,23 +309,6 @@ def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k, persist):
         mb.meteora_set_tuning("persist", 1)
 
 
-def test_pairs_walk_over_several_tiles_each():
-    # 10 row pairs x 19 token tiles = 190 tiles on 74 pairs of SMs: every pair takes two or three tiles, so both
-    # accumulators in tensor memory and the staging buffer of y are reused; the last token tile is ragged.
-    # y is compared on sampled tokens of every token tile (the oracle takes the GPU's own routing there).
-    w = workloads.make_workload("pairs_loop", T=4700, d_in=512, d_out=2560, dtype="bf16", x_kind="normal",
-                                seed=4700, b_std=0.3)
-    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
-    assert "pairs_of_ctas(persistent)" in mb.meteora_describe_plan(shape)
-    rng = np.random.default_rng(5)
-    tokens = np.unique(np.concatenate([np.arange(0, w.T, 256), np.arange(127, w.T, 256), np.arange(128, w.T, 256),
-                                       np.array([w.T - 1]), rng.integers(0, w.T, 200)]))
-    check_forward(w, y_tol=1e-2, tokens=tokens)
-    y1, i1, _ = run_forward(w)
-    y2, i2, _ = run_forward(w)
-    np.testing.assert_array_equal(y1, y2)
-
-
 @pytest.mark.parametrize("d_in,d_out,T", [(1024, 640, 600), (1096, 512, 300)])
 def test_prefill_on_single_sms_matches_oracle(d_in, d_out, T):
     # the 128 x 256 tiles of one CTA each, which small prefill problems still take by default
