@@ -39,8 +39,6 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     const size_t bn = (T + 15) / 16 * 16;
     const size_t part_tiles = s.T <= 256 ? (row_tiles * 28 < 296 ? row_tiles * 28 : 296) : 0;
     ws.part_g = (float*)take(part_tiles * bn * 128 * sizeof(float));
-    // prefill, rank 8: masked bf16 copy of uw, one 16-byte row per (adapter up to a multiple of 8, token)
-    ws.us_g = (__nv_bfloat16*)take(s.T > 256 && s.r == 8 ? (size_t)((s.N + 7) / 8 * 8) * T * 16 : 0);
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);
     ws.bytes = off;
@@ -93,8 +91,7 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
         const bool pdl = tuning().pdl != 0;
         if ((rc = launch_stacked_shrink_tc(x, A, Wg, s, ws, st)) != METEORA_OK) return rc;
         if ((rc = launch_select_from_stacked(ws.u_all, ws.ld_u, ws.col_logits, tc_stacked_zsplits(s), s, ws.topk_idx,
-                                             ws.topk_w, ws.uw, tc_wants_us_g(s) ? ws.us_g : nullptr, pdl, st)) !=
-            METEORA_OK)
+                                             ws.topk_w, ws.uw, pdl, st)) != METEORA_OK)
             return rc;
         if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
         rc = launch_base_lora_tc(x, W0, B, s, ws, y, pdl && !timed, st);
@@ -280,7 +277,6 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "coop")) t.coop = value;
     else if (!strcmp(name, "no_hold")) t.no_hold = value;
     else if (!strcmp(name, "pair")) t.pair = value;
-    else if (!strcmp(name, "persist")) t.persist = value;
     else return METEORA_ERR_INVALID_ARG;
     return METEORA_OK;
 }

@@ -24,8 +24,6 @@ struct Workspace {
                         //           copies (slices of the contraction axis) that the selection kernel adds up
     int ld_u;           // row pitch of u_all in floats
     int col_logits;     // first logit column inside a u_all row
-    __nv_bfloat16* us_g;  // [ceil(N/8)*8][T][8]  prefill (T > 256, rank 8): bf16(uw) per adapter, zero where a token did
-                          //           not pick the adapter: the token-side operand of the expand on the tensor cores
     float* part_g;      // fused decode: fp32 partial accumulator tiles of the base product (T <= 256 only)
     int32_t* tile_ctr;  // fused decode: one counter per 128-row tile of d_out (inside the header)
     void* x_dev;        // [T,d_in]  staging for the host-buffer entry point
@@ -44,10 +42,8 @@ inline size_t elem_size(meteora_dtype_t t) { return t == METEORA_BF16 ? 2 : 4; }
 // gate_topk.cu
 int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, int32_t* topk_idx, float* topk_w,
                      float* logits, cudaStream_t st);
-bool tc_wants_us_g(const meteora_shape_t& s);                     // the base product will read Workspace::us_g
 int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int zsplits, const meteora_shape_t& s,
-                               int32_t* topk_idx, float* topk_w, float* uw, __nv_bfloat16* us_g, bool pdl,
-                               cudaStream_t st);
+                               int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st);
 // route.cu
 int launch_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets, int32_t* perm,
                  cudaStream_t st);
@@ -90,7 +86,6 @@ struct Tuning {
     int pdl = 1;
     int fused = 1;           // 0: never use the single-launch decode kernel
     int coop = 1;            // 0 (measurement only): launch it without the co-residency guarantee
-    int persist = 1;         // 0: the pairs' base product as one CTA pair per tile instead of the persistent kernel
     int pair = 1;            // prefill base product on pairs of SMs (256 x 256 tiles, two-CTA MMA): 0 never, 1 where
                              // the pairs cover enough SMs, 2 wherever the shape allows
     int no_hold = 0;         // 1 (measurement only): main CTAs of the decode kernel do not wait for the aux CTAs' first loads

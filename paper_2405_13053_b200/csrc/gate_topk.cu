@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(kGateWarps * 32)
 k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits, int zsplits, size_t zstride, int T,
                       int N, int r, int k,
                       float inv_tau, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
-                      float* __restrict__ uw, __nv_bfloat16* __restrict__ us_g, int pdl) {
+                      float* __restrict__ uw, int pdl) {
     if (pdl) {
         // Let the dependent launch (the base product) start streaming weights now; wait for the
         // stacked shrink, which produced u_all, before reading it.
@@ -59,29 +59,6 @@ k_select_from_stacked(const float* __restrict__ u_all, int ld_u, int col_logits,
     const int t = blockIdx.x * kGateWarps + (threadIdx.x >> 5);
     if (t >= T) return;
     select_token<false>(u_all, ld_u, col_logits, zsplits, zstride, t, N, r, k, inv_tau, lane, topk_idx, topk_w, uw);
-    if (us_g) {
-        // Rank 8 only.  us_g[a][t][0..8) = bf16(uw[t,j,:]) if adapter a is the token's pick j, else zero, for every
-        // a up to the next multiple of 8: with it the expand of Eq. 2 is a plain product over (adapter, rank
-        // entry) that the prefill kernel streams through its tensor-core pipeline.
-        __syncwarp();                                            // this warp's own writes of topk_idx and uw
-        const int n_pad = (N + 7) / 8 * 8;
-        for (int a = lane; a < n_pad; a += 32) {
-            uint4 val = make_uint4(0u, 0u, 0u, 0u);
-            for (int j = 0; j < k; ++j) {
-                if (topk_idx[(size_t)t * k + j] == a) {
-                    const float4* src = reinterpret_cast<const float4*>(uw + ((size_t)t * k + j) * 8);
-                    const float4 lo = src[0], hi = src[1];
-                    const __nv_bfloat162 q0 = __floats2bfloat162_rn(lo.x, lo.y), q1 = __floats2bfloat162_rn(lo.z, lo.w);
-                    const __nv_bfloat162 q2 = __floats2bfloat162_rn(hi.x, hi.y), q3 = __floats2bfloat162_rn(hi.z, hi.w);
-                    val.x = *reinterpret_cast<const uint32_t*>(&q0);
-                    val.y = *reinterpret_cast<const uint32_t*>(&q1);
-                    val.z = *reinterpret_cast<const uint32_t*>(&q2);
-                    val.w = *reinterpret_cast<const uint32_t*>(&q3);
-                }
-            }
-            reinterpret_cast<uint4*>(us_g)[(size_t)a * T + t] = val;
-        }
-    }
 }
 
 int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, int32_t* topk_idx, float* topk_w,
@@ -99,8 +76,7 @@ int launch_gate_topk(const void* x, const void* Wg, const meteora_shape_t& s, in
 }
 
 int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int zsplits, const meteora_shape_t& s,
-                               int32_t* topk_idx, float* topk_w, float* uw, __nv_bfloat16* us_g, bool pdl,
-                               cudaStream_t st) {
+                               int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st) {
     if (s.T == 0) return METEORA_OK;
     const int blocks = (s.T + kGateWarps - 1) / kGateWarps;
     cudaLaunchConfig_t cfg = {};
@@ -115,7 +91,7 @@ int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int
     const float inv_tau = 1.0f / s.temperature;
     cudaError_t e = cudaLaunchKernelEx(&cfg, k_select_from_stacked, u_all, ld_u, col_logits, zsplits,
                                        (size_t)s.T * ld_u, s.T, s.N, s.r, s.k,
-                                       inv_tau, topk_idx, topk_w, uw, us_g, pdl ? 1 : 0);
+                                       inv_tau, topk_idx, topk_w, uw, pdl ? 1 : 0);
     return cuda_status(e);
 }
 

@@ -454,217 +454,4 @@ k_stacked_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
-// ------------------------------------------------------------------------------------------------
-// The same product as k_wgemm_pair as a PERSISTENT kernel: one pair of CTAs per pair of SMs walks over the
-// 256 x 256 tiles (row pairs fastest, so the pairs running at the same time share a token tile in L2), with two
-// accumulators in TMEM, so that a tile's epilogue (TMEM -> bf16 -> shared memory -> TMA store) runs while the
-// tensor cores already work on the next tile.
-//
-// The LoRA expand needs no staging by the epilogue warps here.  The selection kernel has written the masked,
-// gate-weighted shrink outputs as a dense bf16 array us_g[adapter][token][8] (zero where a token did not pick
-// the adapter), so Eq. 2's sum over the picks is a plain product over the N * 8 "columns" (adapter, rank entry)
-// of B, and the producer streams it through the ring as ceil(N / 8) more k-steps: 8 adapters of B's rows of
-// the tile (a 3-D tensor map over B[N, d_out, 8], landing as un-swizzled K-major core matrices) and 8 adapters of
-// us_g for the CTA's 128 tokens, 16 KB each like any other stage.
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2,
-                                                 uint32_t cluster_bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(cluster_bar)
-        : "memory");
-}
-
-struct PairLoopParams {
-    int T, ksteps, ext_steps, stages;     // ext_steps = ceil(N / 8)
-    int row_pairs, tok_tiles, row_tiles;  // tiles: row_pairs x tok_tiles
-    int32_t* status;
-    int pdl_wait;
-};
-
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads)
-k_wgemm_pair_loop(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                  const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmU,
-                  const __grid_constant__ CUtensorMap tmY, const PairLoopParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t ring = (raw + 1023u) & ~1023u;
-    uint8_t* ring_ptr = smem_raw + (ring - raw);
-    constexpr uint32_t kXHalfBytes = kPairHalf * 128;
-    constexpr uint32_t kStageBytes = kWTileBytes + kXHalfBytes;
-    constexpr uint32_t kYStageBytes = kPairTokens * kBM * 2;      // 256 tokens x 128 rows of bf16
-    const uint32_t ring_bytes = p.stages * kStageBytes;
-    const uint32_t ystage_a = ring + ring_bytes;
-    __nv_bfloat16* ystage = reinterpret_cast<__nv_bfloat16*>(ring_ptr + ring_bytes);
-    const uint32_t bar_base = ystage_a + kYStageBytes;            // full[stages], empty[stages], acc_full[2], acc_empty[2]
-    const uint32_t bar_acc_full = bar_base + 2 * p.stages * 8;
-    const uint32_t bar_acc_empty = bar_acc_full + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + kYStageBytes + (2 * p.stages + 4) * 8);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_rank();
-    const bool leader = rank == 0;
-    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int n_tiles = p.row_pairs * p.tok_tiles;
-    const int per_tile = p.ksteps + p.ext_steps;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) {
-            mbar_init(bar_base + s * 8, 1);                       // the leader's expect-tx arrival
-            mbar_init(bar_base + (p.stages + s) * 8, 1);          // one multicast commit
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_acc_full + b * 8, 1);                   // one multicast commit
-            mbar_init(bar_acc_empty + b * 8, 2);                  // both CTAs' epilogue warps have drained it
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(512u)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncwarp();
-    cluster_sync();
-    tc_fence_after();
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
-
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer (both CTAs)
-        if (lane == 0) {
-            bool ok = true;
-            int it = 0;                                           // stage counter across tiles
-            bool waited = !p.pdl_wait;
-            for (int t = pair_id; t < n_tiles && ok; t += n_pairs) {
-                const int rp = t % p.row_pairs, tt = t / p.row_pairs;
-                const int row0 = (rp * 2 + (int)rank) * kBM;      // own 128 rows of W0 / B
-                const int tokh = tt * kPairTokens + (int)rank * kPairHalf;   // own 128 tokens
-                for (int i = 0; i < per_tile; ++i, ++it) {
-                    const int s = it % p.stages, round = it / p.stages;
-                    if (round > 0) ok = mbar_wait(bar_base + (p.stages + s) * 8, (round & 1) ^ 1);
-                    if (!ok) break;
-                    const uint32_t full = bar_base + s * 8;
-                    const uint32_t full_leader = map_to_cta(full, 0);
-                    const uint32_t dst = ring + s * kStageBytes;
-                    if (leader) mbar_expect_tx(full, 2 * kStageBytes);
-                    if (i < p.ksteps) {
-                        tma_load_2d_pair(dst, &tmW, i * kBK, row0, full_leader);
-                        tma_load_2d_pair(dst + kWTileBytes, &tmX, i * kBK, tokh, full_leader);
-                    } else {
-                        if (!waited) {                            // us_g comes from the previous kernel of the stream
-                            asm volatile("griddepcontrol.wait;" ::: "memory");
-                            waited = true;
-                        }
-                        const int a0 = (i - p.ksteps) * 8;
-                        tma_load_3d_pair(dst, &tmB, 0, row0, a0, full_leader);
-                        tma_load_3d_pair(dst + kWTileBytes, &tmU, 0, tokh, a0, full_leader);
-                    }
-                }
-            }
-            if (!ok) {
-                atomicExch(p.status, 1);
-                atomicExch(p.status + 1, 3100);
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (leader only)
-        if (lane == 0 && leader) {
-            const uint32_t idesc = instr_desc_bf16_pair();
-            bool ok = true;
-            int it = 0, local = 0;
-            for (int t = pair_id; t < n_tiles && ok; t += n_pairs, ++local) {
-                const int b = local & 1, use = local >> 1;
-                if (use > 0) ok = mbar_wait_cluster(bar_acc_empty + b * 8, (use & 1) ^ 1);   // drained by both CTAs
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t acc = tmem_base + (uint32_t)(b * kPairTokens);
-                for (int i = 0; i < per_tile; ++i, ++it) {
-                    const int s = it % p.stages, round = it / p.stages;
-                    ok = mbar_wait(bar_base + s * 8, round & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t wa = ring + s * kStageBytes, xa = wa + kWTileBytes;
-                    if (i < p.ksteps) {
-                        const uint64_t da = smem_desc_sw128(wa), db = smem_desc_sw128(xa);
-#pragma unroll
-                        for (int kk = 0; kk < kBK / kUmmaK; ++kk)
-                            umma_bf16_pair(acc, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (i | kk) != 0);
-                    } else {
-                        // 8 adapters of rank 8: four MMAs of K = 16 over un-swizzled core matrices, 2 KB per adapter
-                        constexpr uint32_t ka = kBM * 16, kb = kPairHalf * 16;
-#pragma unroll
-                        for (int m = 0; m < 4; ++m)
-                            umma_bf16_pair(acc, smem_desc_plain(wa + 2 * m * ka, ka, 128),
-                                           smem_desc_plain(xa + 2 * m * kb, kb, 128), idesc, 1u);
-                    }
-                    umma_commit_pair(bar_base + (p.stages + s) * 8);
-                }
-                umma_commit_pair(bar_acc_full + b * 8);            // this tile's accumulators complete (or abandoned)
-            }
-            if (!ok) {
-                atomicExch(p.status, 1);
-                atomicExch(p.status + 2, 3200);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ epilogue warps (both CTAs)
-        const int quad = warp & 3;
-        const int etid = threadIdx.x - 64;
-        const int row_in_tile = quad * 32 + lane;
-        const int c_begin = warp < 6 ? 0 : kPairTokens / 2, c_end = warp < 6 ? kPairTokens / 2 : kPairTokens;
-        int local = 0;
-        bool alive = true;
-        for (int t = pair_id; t < n_tiles; t += n_pairs, ++local) {
-            const int rp = t % p.row_pairs, tt = t / p.row_pairs;
-            const int tile_m = rp * 2 + (int)rank;
-            const int b = local & 1, use = local >> 1;
-            bool acc_ok = alive && mbar_wait(bar_acc_full + b * 8, use & 1);
-            if (!acc_ok && alive && lane == 0) {
-                atomicExch(p.status, 1);
-                atomicExch(p.status + 3, 3300);
-            }
-            acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
-            alive = acc_ok;
-            tc_fence_after();
-            // the previous tile's store has finished reading the staging buffer
-            if (etid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            epi_barrier();
-            for (int c = c_begin; c < c_end; c += 16) {
-                float v[16];
-                if (acc_ok) {
-                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kPairTokens + c), v);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                }
-#pragma unroll
-                for (int i = 0; i < 16; ++i) ystage[(c + i) * kBM + row_in_tile] = __float2bfloat16_rn(v[i]);
-            }
-            tc_fence_before();
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> TMA read
-            epi_barrier();
-            if (etid == 0) {
-                // the accumulator may be overwritten now; the store runs behind the next tile's work
-                mbar_arrive_cluster(map_to_cta(bar_acc_empty + b * 8, 0));
-                if (tile_m < p.row_tiles && acc_ok) {
-                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                                 ::"l"((uint64_t)&tmY), "r"(ystage_a), "r"(tile_m * kBM), "r"(tt * kPairTokens)
-                                 : "memory");
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                }
-            }
-        }
-        if (etid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // y written before the kernel ends
-    }
-    tc_fence_before();
-    __syncwarp();
-    cluster_sync();
-    if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
-    }
-}
-
 }  // namespace meteora

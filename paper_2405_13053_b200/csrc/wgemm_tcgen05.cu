@@ -1161,71 +1161,6 @@ static PairPlan make_pair_plan(const meteora_shape_t& s) {
     return pp;
 }
 
-// 3-D tensor map over rows of 8 bf16 (16 bytes): [planes][rows][8], box = 8 x box_rows x 8 planes, not swizzled,
-// out-of-range rows and planes read as zero.  A box lands as [plane][row][16 B]: un-swizzled K-major core matrices.
-static int get_rank8_map(const void* ptr, int rows, int planes, int box_rows, CUtensorMap* out) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return METEORA_ERR_CUDA;
-    const cuuint64_t gdim[3] = {8, (cuuint64_t)rows, (cuuint64_t)planes};
-    const cuuint64_t gstride[2] = {16, (cuuint64_t)rows * 16};
-    const cuuint32_t box[3] = {8, (cuuint32_t)box_rows, 8};
-    const cuuint32_t estride[3] = {1, 1, 1};
-    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estride,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? METEORA_OK : METEORA_ERR_CUDA;
-}
-
-// Persistent form of the pairs' base product (k_wgemm_pair_loop): 5 ring stages + 64 KB of y staging.
-static bool pair_loop_wanted(const meteora_shape_t& s) { return tuning().persist != 0 && make_pair_plan(s).ok; }
-
-bool tc_wants_us_g(const meteora_shape_t& s) { return pair_loop_wanted(s); }
-
-static int launch_base_lora_pair_loop(const void* x, const void* W0, const void* B, const meteora_shape_t& s,
-                                      const Workspace& ws, void* y, bool pdl, cudaStream_t st) {
-    const int row_tiles = (s.d_out + kBM - 1) / kBM;
-    CUtensorMap mW, mX, mB, mU, mY;
-    int rc;
-    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, 0, &mW)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(x, s.d_in, s.T, kPairHalf, 0, &mX)) != METEORA_OK) return rc;
-    if ((rc = get_rank8_map(B, s.d_out, s.N, kBM, &mB)) != METEORA_OK) return rc;
-    if ((rc = get_rank8_map(ws.us_g, s.T, (s.N + 7) / 8 * 8, kPairHalf, &mU)) != METEORA_OK) return rc;
-    if ((rc = get_store_map(y, s.d_out, s.T, kPairTokens, &mY)) != METEORA_OK) return rc;
-    PairLoopParams p = {};
-    p.T = s.T;
-    p.ksteps = (s.d_in + kBK - 1) / kBK;
-    p.ext_steps = (s.N + 7) / 8;
-    p.stages = tuning().stages > 1 && tuning().stages < 5 ? tuning().stages : 5;
-    p.row_pairs = (row_tiles + 1) / 2;
-    p.tok_tiles = (s.T + kPairTokens - 1) / kPairTokens;
-    p.row_tiles = row_tiles;
-    p.status = ws.status;
-    p.pdl_wait = pdl ? 1 : 0;
-    const size_t smem = 1024 + (size_t)p.stages * (kWTileBytes + kPairHalf * 128) + (size_t)kPairTokens * kBM * 2 + 256;
-    static int smem_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
-    if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
-    if (!smem_set[dev]) {
-        if (cudaFuncSetAttribute(k_wgemm_pair_loop, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-            cudaSuccess)
-            return METEORA_ERR_CUDA;
-        smem_set[dev] = 1;
-    }
-    const int pairs = std::min(p.row_pairs * p.tok_tiles, sm_count() / 2);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * pairs, 1, 1);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_wgemm_pair_loop, mW, mX, mB, mU, mY, p));
-}
-
 static int launch_base_lora_pair(const void* x, const void* W0, const void* B, const meteora_shape_t& s,
                                  const Workspace& ws, void* y, const PairPlan& pp, bool pdl, cudaStream_t st) {
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
@@ -1276,7 +1211,6 @@ static int launch_base_lora_pair(const void* x, const void* W0, const void* B, c
 int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
                         void* y, bool pdl, cudaStream_t st) {
     const PairPlan pp = make_pair_plan(s);
-    if (pp.ok && pair_loop_wanted(s)) return launch_base_lora_pair_loop(x, W0, B, s, ws, y, pdl, st);
     if (pp.ok) return launch_base_lora_pair(x, W0, B, s, ws, y, pp, pdl, st);
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
@@ -1455,10 +1389,9 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     const PairPlan pp = make_pair_plan(s);
     if (pp.ok)
         return snprintf(buf, n,
-                        "path=chain(not fused: reason %d) launches=3 base=pairs_of_ctas%s tiles=%d tile=256x256 stages=%d "
-                        "expand=mma",
-                        fp.why, pair_loop_wanted(s) ? "(persistent)" : "",
-                        (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens), pair_loop_wanted(s) ? 5 : pp.stages);
+                        "path=chain(not fused: reason %d) launches=3 base=pairs_of_ctas pairs=%d tile=256x256 stages=%d "
+                        "smem=%zu expand=mma",
+                        fp.why, (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens), pp.stages, pp.smem);
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     return snprintf(buf, n,
                     "path=chain(not fused: reason %d) launches=3 base_ctas=%d cluster=%d tile_tokens=%d stages=%d kc=%d "

@@ -291,12 +291,10 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T):
     (1024, 640, 600, 28, 2), (512, 256, 257, 28, 2), (1096, 512, 300, 28, 2), (768, 1024, 1024, 7, 3),
     (512, 512, 520, 16, 4), (512, 384, 300, 33, 3),      # Wg in a tile of its own; three tiles of stacked rows
 ])
-@pytest.mark.parametrize("persist", [1, 0])    # 1: pairs walk over the tiles (default); 0: one pair per tile
-def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k, persist):
+def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
     w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, dtype="bf16", x_kind="normal",
                                 seed=700 + T, b_std=0.3)
     mb.meteora_set_tuning("pair", 2)                                 # 2: also where only a few pairs result
-    mb.meteora_set_tuning("persist", persist)
     try:
         shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
         assert "pairs_of_ctas" in mb.meteora_describe_plan(shape)
@@ -306,7 +304,6 @@ def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k, persist):
         np.testing.assert_array_equal(y1, y2)
     finally:
         mb.meteora_set_tuning("pair", 1)
-        mb.meteora_set_tuning("persist", 1)
 
 
 @pytest.mark.parametrize("d_in,d_out,T", [(1024, 640, 600), (1096, 512, 300)])
