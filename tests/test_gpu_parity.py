@@ -306,6 +306,19 @@ def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
         mb.meteora_set_tuning("pair", 1)
 
 
+def test_pairs_of_sms_over_several_waves():
+    # 10 row pairs x 19 token tiles = 190 pair tiles on 74 pairs of SMs: three waves, the last token tile ragged.
+    # y is compared on sampled tokens of every token tile (the oracle takes the GPU's own routing there).
+    w = workloads.make_workload("pairs_waves", T=4700, d_in=512, d_out=2560, dtype="bf16", x_kind="normal",
+                                seed=4700, b_std=0.3)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    assert "pairs_of_ctas" in mb.meteora_describe_plan(shape)
+    rng = np.random.default_rng(5)
+    tokens = np.unique(np.concatenate([np.arange(0, w.T, 256), np.arange(127, w.T, 256), np.arange(128, w.T, 256),
+                                       np.array([w.T - 1]), rng.integers(0, w.T, 200)]))
+    check_forward(w, y_tol=1e-2, tokens=tokens)
+
+
 @pytest.mark.parametrize("d_in,d_out,T", [(1024, 640, 600), (1096, 512, 300)])
 def test_prefill_on_single_sms_matches_oracle(d_in, d_out, T):
     # the 128 x 256 tiles of one CTA each, which small prefill problems still take by default
