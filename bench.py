@@ -510,10 +510,87 @@ def run_sweep(args):
         del mods, graph
 
 
+def run_layer_sweep():
+    """Config 4: the 7 MeteoRA linears of a LLaMA3-8B decoder layer (each with its own gate and adapters), one
+    call each, back to back in one CUDA graph; time per layer against the sum of the linears' rooflines."""
+    import ctypes
+
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import workloads
+
+    lib = mb.load_library()
+    hbm, _ = measured_peaks()
+    tc, _ = measured_tensor_peak()
+    dt, es = torch.bfloat16, 2
+    for T in workloads.CONFIG4_T:
+        g = torch.Generator(device="cuda").manual_seed(11)
+        mods, nbytes, flops = [], 0.0, 0.0
+        for name, (d_in, d_out) in workloads.CONFIG4_LINEARS.items():
+            shape = mb.make_shape(T, d_in, d_out, N_ADAPTERS, RANK, TOPK, dt)
+            x_np = workloads.make_x(T, d_in, "rms", 40 + len(mods), "bf16")
+            mods.append({"name": name, "shape": shape, "x": torch.from_numpy(x_np).to(dt).cuda(),
+                         "W0": (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt),
+                         "A": ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt),
+                         "B": (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt),
+                         "Wg": (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt),
+                         "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": mb.alloc_workspace(shape)})
+            touched = min(N_ADAPTERS, T * TOPK)
+            nbytes += (d_in * d_out + N_ADAPTERS * d_in + touched * RANK * (d_in + d_out) + T * (d_in + d_out)) * es
+            flops += 2.0 * T * d_in * d_out + 2.0 * T * N_ADAPTERS * d_in + 2.0 * T * TOPK * RANK * (d_in + d_out)
+
+        def step():
+            for m in mods:
+                rc = lib.meteora_linear_forward(m["x"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(),
+                                                m["B"].data_ptr(), m["Wg"].data_ptr(), ctypes.byref(m["shape"]),
+                                                m["y"].data_ptr(), m["ws"].data_ptr(), m["ws"].numel(),
+                                                torch.cuda.current_stream().cuda_stream)
+                if rc != 0:
+                    raise mb.MeteoraError(rc, "meteora_linear_forward")
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        iters = 100 if T <= 256 else 10
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        for m in mods:
+            st = mb.meteora_workspace_status(m["ws"])
+            if st != 0:
+                raise mb.MeteoraError(st, "device status")
+        us = e0.elapsed_time(e1) * 1e3 / iters
+        t_mem, t_tc = nbytes / hbm / 1e3, flops / tc / 1e6
+        bound = "hbm" if t_mem >= t_tc else "tensor"
+        print(json.dumps({"config": "config4", "shape": "LLaMA3-8B layer: q k v o gate up down, 7 calls", "T": T,
+                          "us_per_layer": round(us, 2), "tokens_per_s": round(T / us * 1e6), "bound": bound,
+                          "roofline_us": round(max(t_mem, t_tc), 2),
+                          "frac_of_roofline": round(max(t_mem, t_tc) / us, 3),
+                          "achieved": round(nbytes / us / 1e3, 1) if bound == "hbm" else round(flops / us / 1e6, 1),
+                          "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
+                          "l2": "436 MB of W0 per layer: no weight survives in the 126 MB L2 until its next visit"}),
+              flush=True)
+        del mods, graph
+
+
 def main():
     args = parse_args()
     if args.sweep:
         run_sweep(args)
+        run_layer_sweep()
     elif args.impl == "reference":
         run_reference(args)
     else:
