@@ -149,6 +149,27 @@ int meteora_linear_forward(const void* x, const void* W0, const void* A, const v
                            void* stream);
 
 /*
+ * Several MeteoRA linears that read the SAME x (Sec. 3.2: every linear of a decoder block carries its own gate
+ * and adapters; q/k/v share their input, gate/up share theirs), Eq. 2 with Eq. 3 for each of them:
+ *   y[m][T, d_out[m]] = W0[m] x + sum over module m's own top-k picks.
+ * W0, A, B, Wg, y are HOST arrays of n_modules DEVICE pointers (1 <= n_modules <= METEORA_MAX_GROUP), d_out a host
+ * array; T, d_in, N, r, k, dtype, temperature come from `shape` (its d_out is ignored).  Results per module are
+ * those of meteora_linear_forward up to the rounding order of fp32 sums.  Decode batches (T <= 256, rank 8,
+ * bf16, all modules together at most about 120 row tiles of 128) run as ONE kernel launch for the whole group;
+ * anything else runs module by module.  workspace: meteora_group_workspace_bytes(shape, d_out, n_modules) bytes of
+ * device memory, its first 4 KB zeroed once (meteora_workspace_init); meteora_workspace_status reads the group's
+ * status word.  meteora_group_workspace_routing returns where module `module` left its routing.
+ */
+#define METEORA_MAX_GROUP 4
+size_t meteora_group_workspace_bytes(const meteora_shape_t* shape, const int* d_out, int n_modules);
+int meteora_group_workspace_routing(const meteora_shape_t* shape, const int* d_out, int n_modules, int module,
+                                    void* workspace, int32_t** topk_idx, float** topk_w);
+int meteora_linear_forward_group(const void* x, const void* const* W0, const void* const* A, const void* const* B,
+                                 const void* const* Wg, const int* d_out, int n_modules,
+                                 const meteora_shape_t* shape, void* const* y, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
+/*
  * Same as meteora_linear_forward with the activations in HOST memory: x_host[T,d_in] is copied to
  * the device, the layer runs, y_host[T,d_out] is copied back, all on `stream` (pinned host memory
  * makes the copies asynchronous).  Weights and workspace stay device pointers.  The call does not

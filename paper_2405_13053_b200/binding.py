@@ -23,7 +23,8 @@ STATUS = {0: "METEORA_OK", -1: "METEORA_ERR_INVALID_ARG", -2: "METEORA_ERR_UNSUP
           -6: "METEORA_ERR_TIMEOUT"}
 
 EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_lora_delta_static",
-           "meteora_linear_forward",
+           "meteora_linear_forward", "meteora_linear_forward_group", "meteora_group_workspace_bytes",
+           "meteora_group_workspace_routing",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
            "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
            "meteora_describe_plan", "meteora_set_tuning", "meteora_status_string"]
@@ -60,6 +61,12 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_lora_delta_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, shp, vp, vp]
     lib.meteora_linear_forward.argtypes = [vp, vp, vp, vp, vp, shp, vp, vp, sz, vp]
     lib.meteora_linear_forward_host.argtypes = [vp, vp, vp, vp, vp, shp, vp, vp, sz, vp]
+    ip = ctypes.POINTER(ci)
+    lib.meteora_linear_forward_group.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                                 ctypes.POINTER(vp), ip, ci, shp, ctypes.POINTER(vp), vp, sz, vp]
+    lib.meteora_group_workspace_bytes.argtypes = [shp, ip, ci]
+    lib.meteora_group_workspace_bytes.restype = sz
+    lib.meteora_group_workspace_routing.argtypes = [shp, ip, ci, ci, vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.meteora_workspace_bytes.argtypes = [shp]
     lib.meteora_workspace_bytes.restype = sz
     lib.meteora_workspace_routing.argtypes = [shp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
@@ -72,7 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_status_string.argtypes = [ci]
     lib.meteora_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("meteora_workspace_bytes", "meteora_status_string"):
+        if name not in ("meteora_workspace_bytes", "meteora_group_workspace_bytes", "meteora_status_string"):
             getattr(lib, name).restype = ci
     _lib = lib
     return lib
@@ -221,6 +228,48 @@ def meteora_linear_forward(x, W0, A, B, Wg, k: int, temperature: float = 1.0,
         return y
     idx, w = meteora_workspace_routing(shape, workspace)
     return y, idx, w
+
+
+def meteora_linear_forward_group(x, W0s, As, Bs, Wgs, k: int, temperature: float = 1.0,
+                                 workspace: Optional[torch.Tensor] = None, return_routing: bool = False):
+    """Several MeteoRA linears on the same x (lists of per-module tensors).  Returns the list of y, or
+    (ys, [(topk_idx, topk_w) per module]) with views of the workspace."""
+    lib = load_library()
+    T, d_in = x.shape
+    G = len(W0s)
+    N, r, _ = As[0].shape
+    d_outs = [int(W0.shape[0]) for W0 in W0s]
+    shape = make_shape(T, d_in, d_outs[0], N, r, k, x.dtype, temperature)
+    _dtype_code(x)
+    c_d_out = (ctypes.c_int * G)(*d_outs)
+    if workspace is None:
+        n = lib.meteora_group_workspace_bytes(ctypes.byref(shape), c_d_out, G)
+        if n == 0:
+            raise MeteoraError(-1, "meteora_group_workspace_bytes")
+        workspace = torch.zeros(n, dtype=torch.uint8, device=x.device)
+    ys = [torch.empty((T, d), dtype=x.dtype, device=x.device) for d in d_outs]
+    vpa = ctypes.c_void_p * G
+    c_W0 = vpa(*[_dev(W0s[m], (d_outs[m], d_in), x.dtype, "W0") for m in range(G)])
+    c_A = vpa(*[_dev(As[m], (N, r, d_in), x.dtype, "A") for m in range(G)])
+    c_B = vpa(*[_dev(Bs[m], (N, d_outs[m], r), x.dtype, "B") for m in range(G)])
+    c_Wg = vpa(*[_dev(Wgs[m], (N, d_in), x.dtype, "Wg") for m in range(G)])
+    c_y = vpa(*[y.data_ptr() for y in ys])
+    _check(lib.meteora_linear_forward_group(_dev(x, (T, d_in), x.dtype, "x"), c_W0, c_A, c_B, c_Wg, c_d_out, G,
+                                            ctypes.byref(shape), c_y, workspace.data_ptr(), workspace.numel(),
+                                            _stream()), "meteora_linear_forward_group")
+    if not return_routing:
+        return ys
+    routing = []
+    for m in range(G):
+        p_idx, p_w = ctypes.c_void_p(), ctypes.c_void_p()
+        _check(lib.meteora_group_workspace_routing(ctypes.byref(shape), c_d_out, G, m, workspace.data_ptr(),
+                                                   ctypes.byref(p_idx), ctypes.byref(p_w)),
+               "meteora_group_workspace_routing")
+        off_i, off_w = p_idx.value - workspace.data_ptr(), p_w.value - workspace.data_ptr()
+        idx = workspace[off_i:off_i + T * k * 4].view(torch.int32).view(T, k)
+        w = workspace[off_w:off_w + T * k * 4].view(torch.float32).view(T, k)
+        routing.append((idx, w))
+    return ys, routing
 
 
 def meteora_linear_forward_host(x_host, W0, A, B, Wg, k: int, y_host: torch.Tensor, workspace: torch.Tensor,

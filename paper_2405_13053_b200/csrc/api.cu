@@ -103,6 +103,44 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
     return launch_gemm_simt(x, W0, B, ws.topk_idx, ws.uw, s, y, st);
 }
 
+// Workspace of a group call: the modules' own workspaces one after the other (module 0's header serves the
+// group: status word, counters), then the partial tiles of the one-launch decode kernel for all row tiles.
+struct GroupWorkspace {
+    Workspace mod[kMaxGroupModules];
+    float* part_g;
+    size_t bytes;
+};
+static GroupWorkspace carve_group(const meteora_shape_t& s, const int* d_outs, int G, void* base) {
+    GroupWorkspace gw = {};
+    uint8_t* p = (uint8_t*)base;
+    size_t off = 0, tiles = 0;
+    for (int m = 0; m < G; ++m) {
+        meteora_shape_t sm = s;
+        sm.d_out = d_outs[m];
+        gw.mod[m] = carve_workspace(sm, p ? p + off : nullptr);
+        off += align_up(gw.mod[m].bytes, 256);
+        tiles += ((size_t)d_outs[m] + 127) / 128;
+    }
+    const size_t bn = ((size_t)s.T + 15) / 16 * 16;
+    const size_t part_tiles = s.T <= 256 ? std::min<size_t>(tiles * 28, 296) : 0;
+    gw.part_g = (float*)(p ? p + off : nullptr);
+    off += align_up(part_tiles * bn * 128 * sizeof(float), 256);
+    gw.bytes = off;
+    return gw;
+}
+
+static int check_group(const meteora_shape_t* shape, const int* d_out, int n_modules) {
+    if (!shape || !d_out || n_modules < 1) return METEORA_ERR_INVALID_ARG;
+    if (n_modules > kMaxGroupModules) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    for (int m = 0; m < n_modules; ++m) {
+        meteora_shape_t sm = *shape;
+        sm.d_out = d_out[m];
+        const int rc = check_shape(&sm, true, true);
+        if (rc != METEORA_OK) return rc;
+    }
+    return METEORA_OK;
+}
+
 }  // namespace meteora
 
 using namespace meteora;
@@ -159,6 +197,60 @@ int meteora_linear_forward(const void* x, const void* W0, const void* A, const v
     const Workspace ws = carve_workspace(*shape, workspace);
     if (workspace_bytes < ws.bytes) return METEORA_ERR_WORKSPACE_TOO_SMALL;
     return forward_device(x, W0, A, B, Wg, *shape, y, ws, (cudaStream_t)stream);
+}
+
+size_t meteora_group_workspace_bytes(const meteora_shape_t* shape, const int* d_out, int n_modules) {
+    if (check_group(shape, d_out, n_modules) != METEORA_OK) return 0;
+    return carve_group(*shape, d_out, n_modules, nullptr).bytes;
+}
+
+int meteora_group_workspace_routing(const meteora_shape_t* shape, const int* d_out, int n_modules, int module,
+                                    void* workspace, int32_t** topk_idx, float** topk_w) {
+    const int rc = check_group(shape, d_out, n_modules);
+    if (rc != METEORA_OK) return rc;
+    if (!workspace || module < 0 || module >= n_modules) return METEORA_ERR_INVALID_ARG;
+    const GroupWorkspace gw = carve_group(*shape, d_out, n_modules, workspace);
+    if (topk_idx) *topk_idx = gw.mod[module].topk_idx;
+    if (topk_w) *topk_w = gw.mod[module].topk_w;
+    return METEORA_OK;
+}
+
+int meteora_linear_forward_group(const void* x, const void* const* W0, const void* const* A, const void* const* B,
+                                 const void* const* Wg, const int* d_out, int n_modules,
+                                 const meteora_shape_t* shape, void* const* y, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+    int rc = check_group(shape, d_out, n_modules);
+    if (rc != METEORA_OK) return rc;
+    if (shape->T == 0) return METEORA_OK;
+    if (!x || !W0 || !A || !B || !Wg || !y || !workspace) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(workspace)) return METEORA_ERR_MISALIGNED;
+    for (int m = 0; m < n_modules; ++m) {
+        if (!W0[m] || !A[m] || !B[m] || !Wg[m] || !y[m]) return METEORA_ERR_INVALID_ARG;
+        if (!aligned16(W0[m]) || !aligned16(A[m]) || !aligned16(B[m]) || !aligned16(Wg[m]) || !aligned16(y[m]))
+            return METEORA_ERR_MISALIGNED;
+    }
+    GroupWorkspace gw = carve_group(*shape, d_out, n_modules, workspace);
+    if (workspace_bytes < gw.bytes) return METEORA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    // one status word and one set of counters for the whole group: module 0's header
+    for (int m = 1; m < n_modules; ++m) {
+        gw.mod[m].status = gw.mod[0].status;
+        gw.mod[m].tile_ctr = gw.mod[0].tile_ctr;
+    }
+    if (n_modules > 1 && decode_group_supported(*shape, d_out, n_modules)) {
+        GroupModule gm[kMaxGroupModules];
+        for (int m = 0; m < n_modules; ++m) gm[m] = GroupModule{W0[m], A[m], B[m], Wg[m], y[m], d_out[m], gw.mod[m]};
+        rc = launch_decode_group(x, gm, n_modules, *shape, gw.mod[0].status, gw.part_g, gw.mod[0].tile_ctr, st);
+        if (rc != METEORA_ERR_CUDA) return rc;
+        cudaGetLastError();   // the cooperative launch was refused: one call per module instead
+        tuning().fused_refused += 1;
+    }
+    for (int m = 0; m < n_modules; ++m) {
+        meteora_shape_t sm = *shape;
+        sm.d_out = d_out[m];
+        if ((rc = forward_device(x, W0[m], A[m], B[m], Wg[m], sm, y[m], gw.mod[m], st)) != METEORA_OK) return rc;
+    }
+    return METEORA_OK;
 }
 
 int meteora_linear_forward_host(const void* x_host, const void* W0, const void* A, const void* B,

@@ -69,6 +69,20 @@ int launch_base_lora_tc(const void* x, const void* W0, const void* B, const mete
 
 // fused decode kernel (wgemm_tcgen05.cu + decode_fused.cuh)
 bool decode_fused_supported(const meteora_shape_t& s);
+constexpr int kMaxGroupModules = 4;   // modules per group call (= kMaxGroup of the decode kernel)
+// Several modules that share x (their own W0, A, B, Wg, y, d_out and routing scratch) in one launch of the decode kernel.
+struct GroupModule {
+    const void* W0;
+    const void* A;
+    const void* B;
+    const void* Wg;
+    void* y;
+    int d_out;
+    Workspace ws;       // topk_idx, topk_w, uw, u_all, ld_u, col_logits of this module
+};
+bool decode_group_supported(const meteora_shape_t& s, const int* d_outs, int n_modules);
+int launch_decode_group(const void* x, const GroupModule* mods, int n_modules, const meteora_shape_t& s,
+                        int32_t* status, float* part_g, int32_t* tile_ctr, cudaStream_t st);
 int describe_plan(const meteora_shape_t& s, char* buf, size_t n);
 int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);

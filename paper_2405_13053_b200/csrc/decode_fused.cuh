@@ -22,8 +22,27 @@
 
 namespace meteora {
 
+constexpr int kMaxGroup = kMaxGroupModules;   // modules one launch can serve (they share x: q/k/v, gate/up)
+
+// What differs between the modules of a group: weights come through the tensor maps, the rest is here.
+struct DecodeModule {
+    const __nv_bfloat16* B;
+    __nv_bfloat16* y;
+    int d_out;
+    int tile0;             // first row tile of the module in the group-wide numbering of 128-row tiles
+    int32_t* topk_idx;     // selection results, written by aux CTAs, read by main CTAs
+    float* topk_w;
+    float* uw;
+    float* u_part;         // [aux_slices][T][ld_u] partial stacked shrink
+};
+struct DecodeMaps {
+    CUtensorMap W0[kMaxGroup], A[kMaxGroup], At[kMaxGroup], G[kMaxGroup];
+};
+
 struct DecodeParams {
-    WGemmParams main;      // base product: ring geometry, staging offsets, outputs
+    WGemmParams main;      // base product: ring geometry, staging offsets (B, y, d_out, topk_idx, uw unused here)
+    int n_mod;             // modules of the group; their row tiles are numbered one after the other
+    DecodeModule mod[kMaxGroup];
     int n_main;            // main CTAs (M)
     int upt;               // units per row tile = k-steps / kc
     int units;             // row tiles * upt (U); U * M stays below 2^31 (checked by the host)
@@ -35,17 +54,13 @@ struct DecodeParams {
     int aux_slices;        // contraction slices per aux row tile; active aux CTAs = aux_tiles * aux_slices
     int aux_stages;        // ring depth of the aux main loop (one k-step per stage)
     int bar_stages;        // barriers are laid out for max(main stages, aux stages) ring slots
-    float* u_part;         // [aux_slices][T][ld_u] partial stacked shrink
     int ld_u, col_logits;
-    int32_t* topk_idx;     // selection results, written by aux CTAs, read by main CTAs
-    float* topk_w;
-    float* uw;
     float inv_tau;
     int hold;              // main CTAs start loading only after the aux CTAs have issued their first loads
     int32_t* ctr;          // [0] aux partials written, [1] selections published, [2] CTAs exited, [3] aux loads issued
     float* part_g;         // [main CTA][segment 0/1][BN][128] fp32 partial accumulator tiles of the base product
     int32_t* tile_ctr;     // [row tiles] partials delivered per tile
-    int row_tiles;
+    int row_tiles;         // of all modules together
     int trace_call;        // trace builds: which record of the trace buffer this launch fills
 };
 
@@ -124,13 +139,14 @@ __device__ __forceinline__ void select_token_wide(const float* u_part, int ld_u,
 
 // B rows [row0, row0 + nrows) of every adapter (8 bf16 = 16 bytes each) as slab[e][row % 4][row / 4], so that
 // threads owning consecutive groups of 4 rows read consecutive 16-byte words; rows past d_out are zero.
-__device__ __forceinline__ void stage_slab_rows(const WGemmParams& p, uint4* slab, int row0, int nrows, int etid) {
-    const uint4* Bg = reinterpret_cast<const uint4*>(p.B);
-    const int total = p.N * nrows, nq = nrows / 4;
+__device__ __forceinline__ void stage_slab_rows(const __nv_bfloat16* B, int d_out, int N, uint4* slab, int row0,
+                                                int nrows, int etid) {
+    const uint4* Bg = reinterpret_cast<const uint4*>(B);
+    const int total = N * nrows, nq = nrows / 4;
     for (int i = etid; i < total; i += kEpiThreads) {
         const int e = i / nrows, rl = i - e * nrows, o = row0 + rl;
         slab[e * nrows + (rl & 3) * nq + (rl >> 2)] =
-            o < p.d_out ? __ldg(Bg + (size_t)e * p.d_out + o) : make_uint4(0u, 0u, 0u, 0u);
+            o < d_out ? __ldg(Bg + (size_t)e * d_out + o) : make_uint4(0u, 0u, 0u, 0u);
     }
 }
 
@@ -142,7 +158,7 @@ __device__ __forceinline__ void stage_slab_rows(const WGemmParams& p, uint4* sla
 // barrier once (`routing_pending`), after issuing their first loads.  `nthr` threads (etid = 0 .. nthr-1) share
 // the tile: all 256 epilogue threads, or half of them when the CTA finishes rows of two tiles at once.
 template <int C, int U>
-__device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* const (&parts)[C], int c,
+__device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, const float* const (&parts)[C], int c,
                                             int tile_row0, int q0, int nq, int ntok, const uint4* slab,
                                             const float* s_uw, const int* s_idx, int etid, int nthr,
                                             bool& routing_pending) {
@@ -176,8 +192,8 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* c
                 acc.z += v[u][q].z;
                 acc.w += v[u][q].w;
             }
-            for (int j = 0; j < p.k; ++j) {
-                const int slot = t * p.k + j;
+            for (int j = 0; j < k; ++j) {
+                const int slot = t * k + j;
                 const float4 u0 = s_uw4[2 * slot], u1 = s_uw4[2 * slot + 1];
                 const uint4* b = slab + (size_t)s_idx[slot] * slab_rows + ql;
                 fma8(b[0], u0, u1, acc.x);
@@ -186,8 +202,8 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* c
                 fma8(b[3 * nq], u0, u1, acc.w);
             }
             const int o = tile_row0 + (q0 + ql) * 4;
-            __nv_bfloat16* dst = p.y + (size_t)t * p.d_out + o;
-            if ((p.d_out & 3) == 0 && o + 3 < p.d_out) {
+            __nv_bfloat16* dst = y + (size_t)t * d_out + o;
+            if ((d_out & 3) == 0 && o + 3 < d_out) {
                 const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
                 uint2 pk;
                 pk.x = *reinterpret_cast<const uint32_t*>(&lo);
@@ -197,15 +213,23 @@ __device__ __forceinline__ void finish_rows(const WGemmParams& p, const float* c
                 const float f[4] = {acc.x, acc.y, acc.z, acc.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
-                    if (o + i < p.d_out) dst[i] = __float2bfloat16_rn(f[i]);
+                    if (o + i < d_out) dst[i] = __float2bfloat16_rn(f[i]);
             }
         }
     }
 }
 
+// Module that owns a row tile of the group-wide numbering.
+__device__ __forceinline__ int module_of_tile(const DecodeModule* mod, int n_mod, int tile) {
+    int m = 0;
+    for (int i = 1; i < n_mod; ++i)
+        if (tile >= mod[i].tile0) m = i;
+    return m;
+}
+
 template <int C, int U>
-__device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* part_g, size_t part_stride,
-                                            int units, int M, int upt, int tile, int first_cta, int c,
+__device__ __forceinline__ void finish_tile(__nv_bfloat16* y, int d_out, int k, int tile_row0, const float* part_g,
+                                            size_t part_stride, int units, int M, int upt, int tile, int first_cta, int c,
                                             int q0, int nq, int ntok, const uint4* slab, const float* s_uw,
                                             const int* s_idx, int etid, int nthr, bool& routing_pending) {
     // partial of contributor q: CTA first_cta + q, its segment 0 if its range starts in this tile, else 1
@@ -216,7 +240,7 @@ __device__ __forceinline__ void finish_tile(const WGemmParams& p, const float* p
         const int seg = (int)((unsigned)units * (unsigned)cta / (unsigned)M) / upt == tile ? 0 : 1;
         parts[q] = part_g + ((size_t)cta * 2 + seg) * part_stride;
     }
-    finish_rows<C, U>(p, parts, c, tile * kBM, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
+    finish_rows<C, U>(y, d_out, k, parts, c, tile_row0, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
 }
 
 #ifdef METEORA_TRACE
@@ -301,10 +325,8 @@ __device__ __forceinline__ bool fused_mma(const RingGeom& g, uint32_t tmem_base,
 }
 
 __global__ void __launch_bounds__(kThreads)
-k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmX,
-               const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAt,
-               const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmX1,
-               const DecodeParams d) {
+k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ CUtensorMap tmX,
+               const __grid_constant__ CUtensorMap tmX1, const DecodeParams d) {
     const WGemmParams& p = d.main;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -321,7 +343,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool is_aux = (int)blockIdx.x < d.n_aux;
     const int main_id = (int)blockIdx.x - d.n_aux;
-    const int n_active = d.aux_tiles * d.aux_slices;
+    const int n_active = d.n_mod * d.aux_tiles * d.aux_slices;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < nbar; ++s) mbar_init(bar_base + s * 8, 1);
@@ -359,7 +381,9 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         // ================================================================== aux CTA
         const int aux_id = blockIdx.x;
         const bool active = aux_id < n_active;
-        const int tile = aux_id % d.aux_tiles, slice = aux_id / d.aux_tiles;
+        const int group_tiles = d.n_mod * d.aux_tiles;                       // (module, tile) pairs of the stacked shrinks
+        const int am = active ? (aux_id % group_tiles) / d.aux_tiles : 0;    // module
+        const int tile = (aux_id % group_tiles) % d.aux_tiles, slice = aux_id / group_tiles;
         const int ks0 = active ? (int)(((long long)p.ksteps * slice) / d.aux_slices) : 0;
         const int ks1 = active ? (int)(((long long)p.ksteps * (slice + 1)) / d.aux_slices) : 0;
         const int niter = ks1 - ks0;
@@ -368,8 +392,8 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         if (warp == 0) {
             if (lane == 0 && active) {
                 // A's last tile has its own map (its box stops at A's last row when Wg follows in the same tile)
-                const CUtensorMap* mA = tile >= d.a_tiles ? nullptr : tile == d.a_tiles - 1 ? &tmAt : &tmA;
-                const CUtensorMap* mG = tile == d.gate_tile ? &tmG : nullptr;
+                const CUtensorMap* mA = tile >= d.a_tiles ? nullptr : tile == d.a_tiles - 1 ? &maps.At[am] : &maps.A[am];
+                const CUtensorMap* mG = tile == d.gate_tile ? &maps.G[am] : nullptr;
                 if (!fused_producer(geom, mA, &tmX1, tile * kBM, ks0, niter, d.ctr + 3, mG, (uint32_t)d.gate_row0 * 128u))
                     flag_error(p, 1, 400);
             }
@@ -391,7 +415,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 col = tile * kBM + trow;
             if (tile == d.gate_tile && trow >= d.gate_row0 && trow < d.gate_row0 + p.N)
                 col = d.col_logits + trow - d.gate_row0;
-            float* dst = d.u_part + (size_t)slice * p.T * d.ld_u + max(col, 0);
+            float* dst = d.mod[am].u_part + (size_t)slice * p.T * d.ld_u + max(col, 0);
             for (int c = c_begin; c < c_end; c += 16) {
                 float v[16];
                 if (acc_ok) {
@@ -418,11 +442,14 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 if (tr_aux) FUSED_STAMP(p, 48, 3);
             }
             __syncthreads();
-            const int nwarps = kThreads / 32;                                    // tokens dealt round-robin
+            const int nwarps = kThreads / 32;                                    // (module, token) items dealt round-robin
             float* wbuf = reinterpret_cast<float*>(ring_ptr) + warp * d.ld_u;     // the ring is idle by now
-            for (int t = aux_id * nwarps + warp; t < p.T; t += n_active * nwarps)
-                select_token_wide(d.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.k,
-                                  d.inv_tau, lane, wbuf, d.topk_idx, d.topk_w, d.uw);
+            for (int it = aux_id * nwarps + warp; it < d.n_mod * p.T; it += n_active * nwarps) {
+                const int sm = it / p.T, t = it - sm * p.T;
+                const DecodeModule& mo = d.mod[sm];
+                select_token_wide(mo.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.k,
+                                  d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
+            }
             __syncthreads();
             if (threadIdx.x == 0) {
                 __threadfence();
@@ -448,18 +475,26 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 // let the stacked shrink get its loads into the memory queues first
                 bool ok = d.hold ? wait_counter(d.ctr + 3, n_active) : true;
                 if (tr_main) FUSED_STAMP(p, 32, 1);
+                int cur_tile = -1, row0 = 0;
+                const CUtensorMap* tmW0 = &maps.W0[0];
                 for (int it = 0; it < n_it && ok; ++it) {
                     const int st = it % geom.stages, round = it / geom.stages;
                     if (round > 0) ok = mbar_wait(bar_base + (geom.stages + st) * 8, (round & 1) ^ 1);
                     if (!ok) break;
                     const uint32_t full = bar_base + st * 8, dst = ring + st * stage_bytes;
                     const int unit = u0 + it, tile = unit / upt, kstep = (unit - tile * upt) * p.kc;
+                    if (tile != cur_tile) {                      // rows of which module's W0
+                        const int wm = module_of_tile(d.mod, d.n_mod, tile);
+                        cur_tile = tile;
+                        tmW0 = &maps.W0[wm];
+                        row0 = (tile - d.mod[wm].tile0) * kBM;
+                    }
                     mbar_expect_tx(full, stage_bytes);
                     if (p.maps3d) {
-                        tma_load_3d(dst, &tmW0, 0, tile * kBM, kstep, full);
+                        tma_load_3d(dst, tmW0, 0, row0, kstep, full);
                         tma_load_3d(dst + p.kc * kWTileBytes, &tmX, 0, 0, kstep, full);
                     } else {
-                        tma_load_2d(dst, &tmW0, kstep * kBK, tile * kBM, full);
+                        tma_load_2d(dst, tmW0, kstep * kBK, row0, full);
                         tma_load_2d(dst + kWTileBytes, &tmX, kstep * kBK, 0, full);
                     }
                 }
@@ -468,17 +503,21 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 if (tr_main) FUSED_STAMP(p, 32, 4);
             }
             __syncwarp();
-            // The routing into shared memory for the epilogue warps (it was written by other CTAs of this kernel:
-            // loads that bypass L1), then named barrier 2.
+            // The routing into shared memory for the epilogue warps, once per tile this CTA finishes rows of (two
+            // tiles may belong to two modules of a group); it was written by other CTAs of this kernel: loads
+            // that bypass L1.  Then named barrier 2.
             {
-                int* s_idx = reinterpret_cast<int*>(epi + p.idx_off);
-                float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off);
                 const int slots = ntok * p.k;
-                const float4* uw4 = reinterpret_cast<const float4*>(p.uw);
+                for (int sg = 0; sg < nseg; ++sg) {
+                    const DecodeModule& mo = d.mod[module_of_tile(d.mod, d.n_mod, tile_a + sg)];
+                    int* s_idx = reinterpret_cast<int*>(epi + p.idx_off) + sg * p.BN * p.k;
+                    float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off) + sg * p.BN * p.k * 2;
+                    const float4* uw4 = reinterpret_cast<const float4*>(mo.uw);
 #pragma unroll 8
-                for (int i = lane; i < slots; i += 32) s_idx[i] = min(max(__ldcg(p.topk_idx + i), 0), p.N - 1);
+                    for (int i = lane; i < slots; i += 32) s_idx[i] = min(max(__ldcg(mo.topk_idx + i), 0), p.N - 1);
 #pragma unroll 8
-                for (int i = lane; i < 2 * slots; i += 32) s_uw4[i] = __ldcg(uw4 + i);
+                    for (int i = lane; i < 2 * slots; i += 32) s_uw4[i] = __ldcg(uw4 + i);
+                }
                 __syncwarp();
                 asm volatile("bar.arrive 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
                 if (lane == 0 && tr_main) FUSED_STAMP(p, 32, 9);
@@ -516,7 +555,7 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
         } else {
             // Which rows of which tile this CTA finishes: tile `t` is shared by the CTAs owner(first unit) ..
             // owner(last unit), in that order; contributor j of c takes the groups of 4 rows [32j/c, 32(j+1)/c).
-            int d_tile[2], d_first[2], d_c[2], d_q0[2], d_nq[2];
+            int d_tile[2], d_first[2], d_c[2], d_q0[2], d_nq[2], d_mod[2], d_row0[2];
             uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
             uint4* d_slab[2];
             int slab_words = 0;
@@ -532,12 +571,13 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 d_q0[sg] = 32 * j / c;
                 d_nq[sg] = 32 * (j + 1) / c - d_q0[sg];
                 d_slab[sg] = slab + slab_words;
+                d_mod[sg] = module_of_tile(d.mod, d.n_mod, tile);
+                d_row0[sg] = (tile - d.mod[d_mod[sg]].tile0) * kBM;          // the tile's first row inside its module
                 // B rows of that slice for every adapter: no routing needed yet
-                stage_slab_rows(p, d_slab[sg], tile * kBM + 4 * d_q0[sg], 4 * d_nq[sg], etid);
+                stage_slab_rows(d.mod[d_mod[sg]].B, d.mod[d_mod[sg]].d_out, p.N, d_slab[sg], d_row0[sg] + 4 * d_q0[sg],
+                                4 * d_nq[sg], etid);
                 slab_words += p.N * 4 * d_nq[sg];
             }
-            float* s_uw = reinterpret_cast<float*>(epi + p.uw_off);
-            int* s_idx = reinterpret_cast<int*>(epi + p.idx_off);
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
             // Accumulators out of TMEM to the fp32 scratch, segment by segment (lane = row, a warp writes 128
             // contiguous bytes per token); each delivery bumps the tile's counter.
@@ -578,16 +618,19 @@ k_decode_fused(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__
                 }
                 asm volatile("bar.sync %0, %1;" ::"r"(3 + sg), "r"(nthr) : "memory");
                 const int c = d_c[sg];
+                const DecodeModule& mo = d.mod[d_mod[sg]];
+                const float* s_uw = reinterpret_cast<const float*>(epi + p.uw_off) + sg * p.BN * p.k * 8;
+                const int* s_idx = reinterpret_cast<const int*>(epi + p.idx_off) + sg * p.BN * p.k;
                 if (c <= 1)
-                    finish_tile<1, 4>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<1, 4>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 2)
-                    finish_tile<2, 4>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<2, 4>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 4)
-                    finish_tile<4, 4>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<4, 4>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 8)
-                    finish_tile<8, 2>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<8, 2>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else
-                    finish_tile<16, 1>(p, d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<16, 1>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
             }
             if (routing_pending) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);

@@ -1276,21 +1276,30 @@ struct FusedPlan {
     int why;   // why not: 1 knob/shape, 2 more row tiles than main CTAs, 4 residency, 5 shared memory
     Plan main; // BN, stages, kc, maps3d, tmem_cols, staging offsets, smem of the decode kernel
     int row_tiles, n_main, upt, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages;
+    size_t w0_bytes;
 };
 
-// Launch plan of the single-launch decode kernel.  Main CTAs: as many as the SMs the aux CTAs leave, at most 14
+// Launch plan of the single-launch decode kernel, for one module or a group of modules that share x.  Main CTAs: as many as the SMs the aux CTAs leave, at most 14
 // per row tile (16 partial tiles is the most the last step sums) and at least one per row tile (a CTA's unit
 // range then spans at most two tiles).  Aux CTAs: about 20, the row tiles of the stacked shrink times up to 16
 // slices of the contraction axis.
-static FusedPlan make_fused_plan(const meteora_shape_t& s) {
+static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, int G) {
     const Tuning& tn = tuning();
     FusedPlan fp = {};
     fp.why = 1;
+    if (G < 1 || G > kMaxGroup) return fp;
     // Measured on B200 (4096 -> 4096): the single launch is ahead of the three-launch chain at every decode
     // batch size (15.7 vs 16.5 us at T = 1, 19.5 vs 25 us at T = 128).
     if (!tn.fused) return fp;
     if (!tc_path_supported(s) || s.T > 256 || s.r != 8 || tn.simt_expand) return fp;
-    fp.row_tiles = (s.d_out + kBM - 1) / kBM;
+    fp.row_tiles = 0;                                            // of all modules of the group together
+    size_t w0_bytes = 0;
+    for (int m = 0; m < G; ++m) {
+        if (d_outs[m] <= 0) return fp;
+        fp.row_tiles += (d_outs[m] + kBM - 1) / kBM;
+        w0_bytes += (size_t)d_outs[m] * s.d_in * 2;
+    }
+    fp.w0_bytes = w0_bytes;
     if (fp.row_tiles > kMaxFusedRowTiles) return fp;
     Plan& pl = fp.main;
     const int sms = std::min(sm_count(), 148);                   // the workspace holds partial tiles for 148 CTAs
@@ -1305,7 +1314,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     {
         // staging of the last step (B rows, routing) comes first; with 256-token tiles two k-steps per stage
         // would leave room for one stage only
-        const size_t staged = (size_t)s.N * kBM * 16 + (size_t)pl.BN * s.k * (s.r * 4 + 4) + 2048;
+        const size_t staged = (size_t)s.N * kBM * 16 + 2 * (size_t)pl.BN * s.k * (s.r * 4 + 4) + 2048;
         const size_t one = kWTileBytes + (size_t)pl.BN * 128;
         while (pl.kc > 1 && staged + 2 * pl.kc * one > 226 * 1024) pl.kc /= 2;
     }
@@ -1319,11 +1328,12 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     fp.gate_tile = fp.aux_tiles - 1;
     fp.gate_row0 = merged ? tail_rows : 0;
     fp.why = 2;
-    if (fp.aux_tiles + fp.row_tiles > sms) return fp;
-    const int aux_budget = std::min(std::max(20, fp.aux_tiles), sms - fp.row_tiles);
-    fp.aux_slices = std::min(std::min(aux_budget / fp.aux_tiles, ksteps), 16);   // 16: the selection reads all slices at once
+    const int group_tiles = G * fp.aux_tiles;                    // every module has its own stacked shrink
+    if (group_tiles + fp.row_tiles > sms) return fp;
+    const int aux_budget = std::min(std::max(std::max(20, 4 * group_tiles), group_tiles), sms - fp.row_tiles);
+    fp.aux_slices = std::min(std::min(aux_budget / group_tiles, ksteps), 16);   // 16: the selection reads all slices at once
     if (fp.aux_slices < 1) return fp;
-    fp.n_aux = fp.aux_tiles * fp.aux_slices;
+    fp.n_aux = group_tiles * fp.aux_slices;
     const long long units = (long long)fp.row_tiles * fp.upt;
     // Main CTAs: at most 8 per row tile share a tile's rows in the last step.  A multiple of the row tiles keeps
     // every CTA inside one tile (one accumulator, one finishing duty); it is taken unless it idles more than a
@@ -1343,9 +1353,11 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     // rows a CTA finishes: 128 / c when every tile belongs to exactly c CTAs, up to 128 (two tiles) otherwise
     const bool whole = n_main % fp.row_tiles == 0;
     const int own_rows = whole ? 4 * ((32 + n_main / fp.row_tiles - 1) / (n_main / fp.row_tiles)) : kBM;
+    // the routing once per tile a CTA finishes rows of (one tile, or two that may belong to two modules)
+    const int duties = whole ? 1 : 2;
     pl.uw_off = (int)align_up((size_t)s.N * own_rows * 16, 16);
-    pl.idx_off = pl.uw_off + pl.BN * s.k * s.r * 4;
-    const size_t epi_bytes = (size_t)pl.idx_off + (size_t)pl.BN * s.k * 4;
+    pl.idx_off = pl.uw_off + duties * pl.BN * s.k * s.r * 4;
+    const size_t epi_bytes = (size_t)pl.idx_off + (size_t)duties * pl.BN * s.k * 4;
     pl.epi_off = (int)align_up((size_t)(2 * 16 + 3) * 8 + 16, 128);
     const size_t fixed = 1024 + pl.epi_off + epi_bytes;
     if (fixed + 48 * 1024 > 226 * 1024) return fp;
@@ -1373,7 +1385,13 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s) {
     return fp;
 }
 
+static FusedPlan make_fused_plan(const meteora_shape_t& s) { return make_fused_plan(s, &s.d_out, 1); }
+
 bool decode_fused_supported(const meteora_shape_t& s) { return make_fused_plan(s).ok; }
+
+bool decode_group_supported(const meteora_shape_t& s, const int* d_outs, int G) {
+    return make_fused_plan(s, d_outs, G).ok;
+}
 
 // Human-readable launch plan of meteora_linear_forward for this shape (for logs and benchmark records).
 int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
@@ -1400,34 +1418,48 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
                     pl.lora_mma ? "mma" : "simt");
 }
 
-int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
-                        const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st) {
-    const FusedPlan fp = make_fused_plan(s);
+int launch_decode_group(const void* x, const GroupModule* mods, int G, const meteora_shape_t& s, int32_t* status,
+                        float* part_g, int32_t* tile_ctr, cudaStream_t st) {
+    int d_outs[kMaxGroup] = {};
+    if (G < 1 || G > kMaxGroup) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    for (int m = 0; m < G; ++m) d_outs[m] = mods[m].d_out;
+    const FusedPlan fp = make_fused_plan(s, d_outs, G);
     if (!fp.ok) return METEORA_ERR_UNSUPPORTED_SHAPE;
     const Plan& pl = fp.main;
     const int depth = pl.maps3d ? pl.kc : 0, depth1 = pl.maps3d ? 1 : 0;
-    CUtensorMap mW, mX, mA, mAt, mG, mX1;
+    DecodeMaps maps;
+    CUtensorMap mX, mX1;
     int rc;
     const int tail_box = fp.gate_row0 > 0 ? fp.gate_row0 : kBM, gate_box = kBM - fp.gate_row0;
-    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, depth, &mW)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, depth, &mX)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, depth1, &mA)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, tail_box, depth1, &mAt)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(Wg, s.d_in, s.N, gate_box, depth1, &mG)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, depth1, &mX1)) != METEORA_OK) return rc;
     DecodeParams d = {};
-    fill_common(d.main, pl, s.T, s.d_in, ws.status);
+    fill_common(d.main, pl, s.T, s.d_in, status);
     d.main.split_tile = 0x7FFFFFFF;
-    d.main.rows0 = s.d_out;
     d.main.mode = MODE_LORA;
-    d.main.topk_idx = ws.topk_idx;
-    d.main.uw = ws.uw;
-    d.main.B = (const __nv_bfloat16*)B;
-    d.main.y = (__nv_bfloat16*)y;
-    d.main.d_out = s.d_out;
     d.main.N = s.N;
     d.main.r = s.r;
     d.main.k = s.k;
+    d.n_mod = G;
+    int tile0 = 0;
+    for (int m = 0; m < kMaxGroup; ++m) {
+        const GroupModule& gm = mods[m < G ? m : 0];             // unused slots repeat module 0's (valid) maps
+        if ((rc = get_tensor_map(gm.W0, s.d_in, gm.d_out, kBM, depth, &maps.W0[m])) != METEORA_OK) return rc;
+        if ((rc = get_tensor_map(gm.A, s.d_in, s.N * s.r, kBM, depth1, &maps.A[m])) != METEORA_OK) return rc;
+        if ((rc = get_tensor_map(gm.A, s.d_in, s.N * s.r, tail_box, depth1, &maps.At[m])) != METEORA_OK) return rc;
+        if ((rc = get_tensor_map(gm.Wg, s.d_in, s.N, gate_box, depth1, &maps.G[m])) != METEORA_OK) return rc;
+        if (m >= G) continue;
+        DecodeModule& mo = d.mod[m];
+        mo.B = (const __nv_bfloat16*)gm.B;
+        mo.y = (__nv_bfloat16*)gm.y;
+        mo.d_out = gm.d_out;
+        mo.tile0 = tile0;
+        mo.topk_idx = gm.ws.topk_idx;
+        mo.topk_w = gm.ws.topk_w;
+        mo.uw = gm.ws.uw;
+        mo.u_part = gm.ws.u_all;
+        tile0 += (gm.d_out + kBM - 1) / kBM;
+    }
     d.n_main = fp.n_main;
     d.upt = fp.upt;
     d.units = fp.row_tiles * fp.upt;
@@ -1440,19 +1472,15 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     d.aux_slices = fp.aux_slices;
     d.aux_stages = fp.aux_stages;
     d.bar_stages = std::max(fp.aux_stages, pl.stages);
-    d.u_part = ws.u_all;
-    d.ld_u = ws.ld_u;
-    d.col_logits = ws.col_logits;
-    d.topk_idx = ws.topk_idx;
-    d.topk_w = ws.topk_w;
-    d.uw = ws.uw;
+    d.ld_u = mods[0].ws.ld_u;
+    d.col_logits = mods[0].ws.col_logits;
     d.inv_tau = 1.0f / s.temperature;
     // Holding the main CTAs back until the aux CTAs have issued their loads pays only while the base product is
     // short: from about 64 MB of W0 on the routing is ready long before it is needed either way.
-    d.hold = (tuning().no_hold || (size_t)s.d_in * s.d_out * 2 > ((size_t)64 << 20)) ? 0 : 1;
-    d.ctr = ws.status + 16;
-    d.part_g = ws.part_g;
-    d.tile_ctr = ws.tile_ctr;
+    d.hold = (tuning().no_hold || fp.w0_bytes > ((size_t)64 << 20)) ? 0 : 1;
+    d.ctr = status + 16;
+    d.part_g = part_g;
+    d.tile_ctr = tile_ctr;
     d.row_tiles = fp.row_tiles;
     if (pl.smem > 227 * 1024) return METEORA_ERR_UNSUPPORTED_SHAPE;
     cudaLaunchConfig_t cfg = {};
@@ -1469,7 +1497,13 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
     static int trace_calls = 0;
     d.trace_call = trace_calls++;
 #endif
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, mW, mX, mA, mAt, mG, mX1, d));
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, maps, mX, mX1, d));
+}
+
+int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                        const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st) {
+    GroupModule gm = {W0, A, B, Wg, y, s.d_out, ws};
+    return launch_decode_group(x, &gm, 1, s, ws.status, ws.part_g, ws.tile_ctr, st);
 }
 
 }  // namespace meteora
