@@ -7,7 +7,7 @@ import torch
 import oracle
 from paper_2405_13053_b200 import binding as mb
 from paper_2405_13053_b200 import workloads
-from gpu_util import check_selection, rel_l2, to_dev
+from .gpu_util import check_selection, rel_l2, to_dev
 
 pytestmark = pytest.mark.gpu
 
