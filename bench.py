@@ -540,7 +540,7 @@ def run_layer_sweep():
             nbytes += (d_in * d_out + N_ADAPTERS * d_in + touched * RANK * (d_in + d_out) + T * (d_in + d_out)) * es
             flops += 2.0 * T * d_in * d_out + 2.0 * T * N_ADAPTERS * d_in + 2.0 * T * TOPK * RANK * (d_in + d_out)
 
-        def step():
+        def step_calls():
             for m in mods:
                 rc = lib.meteora_linear_forward(m["x"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(),
                                                 m["B"].data_ptr(), m["Wg"].data_ptr(), ctypes.byref(m["shape"]),
@@ -549,41 +549,70 @@ def run_layer_sweep():
                 if rc != 0:
                     raise mb.MeteoraError(rc, "meteora_linear_forward")
 
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            step()
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            step()
-        iters = 100 if T <= 256 else 10
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(iters):
-            graph.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        for m in mods:
-            st = mb.meteora_workspace_status(m["ws"])
-            if st != 0:
-                raise mb.MeteoraError(st, "device status")
-        us = e0.elapsed_time(e1) * 1e3 / iters
-        t_mem, t_tc = nbytes / hbm / 1e3, flops / tc / 1e6
-        bound = "hbm" if t_mem >= t_tc else "tensor"
-        print(json.dumps({"config": "config4", "shape": "LLaMA3-8B layer: q k v o gate up down, 7 calls", "T": T,
-                          "us_per_layer": round(us, 2), "tokens_per_s": round(T / us * 1e6), "bound": bound,
-                          "roofline_us": round(max(t_mem, t_tc), 2),
-                          "frac_of_roofline": round(max(t_mem, t_tc) / us, 3),
-                          "achieved": round(nbytes / us / 1e3, 1) if bound == "hbm" else round(flops / us / 1e6, 1),
-                          "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
-                          "l2": "436 MB of W0 per layer: no weight survives in the 126 MB L2 until its next visit"}),
-              flush=True)
-        del mods, graph
+        # the same layer with the linears that share their input as group calls: q/k/v, o, gate/up, down
+        by_name = {m["name"]: m for m in mods}
+        groups = []
+        for names in (("q", "k", "v"), ("o",), ("gate", "up"), ("down",)):
+            ms = [by_name[n] for n in names]
+            G = len(ms)
+            d_outs = (ctypes.c_int * G)(*[int(m["W0"].shape[0]) for m in ms])
+            n = lib.meteora_group_workspace_bytes(ctypes.byref(ms[0]["shape"]), d_outs, G)
+            vpa = ctypes.c_void_p * G
+            groups.append({"x": ms[0]["x"], "G": G, "d_outs": d_outs, "shape": ms[0]["shape"],
+                           "W0": vpa(*[m["W0"].data_ptr() for m in ms]), "A": vpa(*[m["A"].data_ptr() for m in ms]),
+                           "B": vpa(*[m["B"].data_ptr() for m in ms]), "Wg": vpa(*[m["Wg"].data_ptr() for m in ms]),
+                           "y": vpa(*[m["y"].data_ptr() for m in ms]),
+                           "ws": torch.zeros(n, dtype=torch.uint8, device="cuda"),
+                           "one_launch": lib.meteora_group_plan(ctypes.byref(ms[0]["shape"]), d_outs, G)})
+
+        def step_groups():
+            for gq in groups:
+                rc = lib.meteora_linear_forward_group(gq["x"].data_ptr(), gq["W0"], gq["A"], gq["B"], gq["Wg"],
+                                                      gq["d_outs"], gq["G"], ctypes.byref(gq["shape"]), gq["y"],
+                                                      gq["ws"].data_ptr(), gq["ws"].numel(),
+                                                      torch.cuda.current_stream().cuda_stream)
+                if rc != 0:
+                    raise mb.MeteoraError(rc, "meteora_linear_forward_group")
+
+        for mode, step in (("7 calls", step_calls), ("4 group calls: q/k/v, o, gate/up, down", step_groups)):
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            iters = 100 if T <= 256 else 10
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            for m in mods + groups:
+                st = mb.meteora_workspace_status(m["ws"])
+                if st != 0:
+                    raise mb.MeteoraError(st, "device status")
+            us = e0.elapsed_time(e1) * 1e3 / iters
+            t_mem, t_tc = nbytes / hbm / 1e3, flops / tc / 1e6
+            bound = "hbm" if t_mem >= t_tc else "tensor"
+            print(json.dumps({"config": "config4", "shape": "LLaMA3-8B layer: q k v o gate up down, " + mode, "T": T,
+                              "us_per_layer": round(us, 2), "tokens_per_s": round(T / us * 1e6), "bound": bound,
+                              "roofline_us": round(max(t_mem, t_tc), 2),
+                              "frac_of_roofline": round(max(t_mem, t_tc) / us, 3),
+                              "achieved": round(nbytes / us / 1e3, 1) if bound == "hbm" else round(flops / us / 1e6, 1),
+                              "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
+                              "launches": (sum(1 if gq["one_launch"] else 3 * gq["G"] if T > 256 else gq["G"]
+                                               for gq in groups) if step is step_groups
+                                           else len(mods) * (3 if T > 256 else 1)),
+                              "l2": "436 MB of W0 per layer: no weight survives in the 126 MB L2 until its next visit"}),
+                  flush=True)
+        del mods, graph, groups
 
 
 def main():

@@ -158,10 +158,12 @@ int meteora_linear_forward(const void* x, const void* W0, const void* A, const v
  * bf16, all modules together at most about 120 row tiles of 128) run as ONE kernel launch for the whole group;
  * anything else runs module by module.  workspace: meteora_group_workspace_bytes(shape, d_out, n_modules) bytes of
  * device memory, its first 4 KB zeroed once (meteora_workspace_init); meteora_workspace_status reads the group's
- * status word.  meteora_group_workspace_routing returns where module `module` left its routing.
+ * status word.  meteora_group_workspace_routing returns where module `module` left its routing;
+ * meteora_group_plan returns 1 if the group runs as one launch, 0 if module by module, or an error code.
  */
 #define METEORA_MAX_GROUP 4
 size_t meteora_group_workspace_bytes(const meteora_shape_t* shape, const int* d_out, int n_modules);
+int meteora_group_plan(const meteora_shape_t* shape, const int* d_out, int n_modules);
 int meteora_group_workspace_routing(const meteora_shape_t* shape, const int* d_out, int n_modules, int module,
                                     void* workspace, int32_t** topk_idx, float** topk_w);
 int meteora_linear_forward_group(const void* x, const void* const* W0, const void* const* A, const void* const* B,

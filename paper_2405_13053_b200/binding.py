@@ -24,7 +24,7 @@ STATUS = {0: "METEORA_OK", -1: "METEORA_ERR_INVALID_ARG", -2: "METEORA_ERR_UNSUP
 
 EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_lora_delta_static",
            "meteora_linear_forward", "meteora_linear_forward_group", "meteora_group_workspace_bytes",
-           "meteora_group_workspace_routing",
+           "meteora_group_workspace_routing", "meteora_group_plan",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
            "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
            "meteora_describe_plan", "meteora_set_tuning", "meteora_status_string"]
@@ -64,6 +64,7 @@ def load_library() -> ctypes.CDLL:
     ip = ctypes.POINTER(ci)
     lib.meteora_linear_forward_group.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
                                                  ctypes.POINTER(vp), ip, ci, shp, ctypes.POINTER(vp), vp, sz, vp]
+    lib.meteora_group_plan.argtypes = [shp, ip, ci]
     lib.meteora_group_workspace_bytes.argtypes = [shp, ip, ci]
     lib.meteora_group_workspace_bytes.restype = sz
     lib.meteora_group_workspace_routing.argtypes = [shp, ip, ci, ci, vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
@@ -228,6 +229,16 @@ def meteora_linear_forward(x, W0, A, B, Wg, k: int, temperature: float = 1.0,
         return y
     idx, w = meteora_workspace_routing(shape, workspace)
     return y, idx, w
+
+
+def meteora_group_plan(T, d_in, d_outs, N, r, k, dtype: torch.dtype) -> int:
+    """1 if meteora_linear_forward_group runs these modules as one kernel launch, 0 if module by module."""
+    lib = load_library()
+    shape = make_shape(T, d_in, d_outs[0], N, r, k, dtype)
+    rc = lib.meteora_group_plan(ctypes.byref(shape), (ctypes.c_int * len(d_outs))(*d_outs), len(d_outs))
+    if rc < 0:
+        raise MeteoraError(rc, "meteora_group_plan")
+    return rc
 
 
 def meteora_linear_forward_group(x, W0s, As, Bs, Wgs, k: int, temperature: float = 1.0,

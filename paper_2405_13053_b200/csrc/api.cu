@@ -204,6 +204,12 @@ size_t meteora_group_workspace_bytes(const meteora_shape_t* shape, const int* d_
     return carve_group(*shape, d_out, n_modules, nullptr).bytes;
 }
 
+int meteora_group_plan(const meteora_shape_t* shape, const int* d_out, int n_modules) {
+    const int rc = check_group(shape, d_out, n_modules);
+    if (rc != METEORA_OK) return rc;
+    return n_modules > 1 && decode_group_supported(*shape, d_out, n_modules) ? 1 : 0;
+}
+
 int meteora_group_workspace_routing(const meteora_shape_t* shape, const int* d_out, int n_modules, int module,
                                     void* workspace, int32_t** topk_idx, float** topk_w) {
     const int rc = check_group(shape, d_out, n_modules);

@@ -55,6 +55,7 @@ def check_group(ws, y_tol):
 ])
 def test_group_of_decode_modules_matches_oracle(d_in, d_outs, T):
     ws = make_group(T, d_in, d_outs, seed=6000 + T)
+    assert mb.meteora_group_plan(T, d_in, list(d_outs), 28, 8, 2, torch.bfloat16) == 1
     ys1, r1 = check_group(ws, y_tol=1e-2)
     ys2, r2 = run_group(ws)
     for a, b in zip(ys1, ys2):
@@ -89,10 +90,12 @@ def test_group_workspace_reused_across_calls():
     assert mb.meteora_workspace_status(workspace) == 0
 
 
-# What the one-launch kernel does not take runs module by module: a prefill batch, fp32 modules, rank 16.
+# What the one-launch kernel does not take runs module by module: a prefill batch, fp32 modules.
 @pytest.mark.parametrize("T,dtype,r,tol", [(300, "bf16", 8, 1e-2), (20, "f32", 8, 1e-4)])
 def test_group_falls_back_module_by_module(T, dtype, r, tol):
-    ws = make_group(T, 256, (128, 200), seed=6300 + T, dtype=dtype, N=6 if dtype == "f32" else 28)
+    N = 6 if dtype == "f32" else 28
+    ws = make_group(T, 256, (128, 200), seed=6300 + T, dtype=dtype, N=N)
+    assert mb.meteora_group_plan(T, 256, [128, 200], N, 8, 2, torch.float32 if dtype == "f32" else torch.bfloat16) == 0
     check_group(ws, y_tol=tol)
 
 
