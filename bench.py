@@ -53,6 +53,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="time every (shape, T) of configs 1-3 instead of the headline step; one JSON line each")
+    ap.add_argument("--variants", action="store_true",
+                    help="time the variants of the method at 4096 -> 4096 (top-k, rank, adapter count, temperature), "
+                         "the axes of the paper's synthetic sweep (App. A.7); one JSON line each")
     return ap.parse_args()
 
 
@@ -615,9 +618,98 @@ def run_layer_sweep():
         del mods, graph, groups
 
 
+def run_variants():
+    """The paper's synthetic sweep axes (App. A.7: k, r, number of adapters; temperature of App. A.5) at the
+    LLaMA3-8B q_proj shape, a decode batch (T = 32) and a prefill batch (T = 2048), one axis at a time around
+    the base point N = 28, r = 8, k = 2."""
+    import ctypes
+
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import build as lib_build
+
+    lib_build.build_library()
+    lib = mb.load_library()
+    torch.cuda.set_device(0)
+    hbm, _ = measured_peaks()
+    tc, _ = measured_tensor_peak()
+    dt, es = torch.bfloat16, 2
+    d_in = d_out = 4096
+    base = {"N": 28, "r": 8, "k": 2, "tau": 1.0}
+    points = [dict(base)]
+    points += [dict(base, k=k) for k in (1, 4)]
+    points += [dict(base, r=r) for r in (4, 16, 32, 64)]
+    points += [dict(base, N=N) for N in (8, 64)]
+    points += [dict(base, tau=20.0)]
+    for T in (32, 2048):
+        for pt in points:
+            N, r, k, tau = pt["N"], pt["r"], pt["k"], pt["tau"]
+            R = 8 if T <= 256 else 1
+            shape = mb.make_shape(T, d_in, d_out, N, r, k, dt, tau)
+            g = torch.Generator(device="cuda").manual_seed(3)
+            mods = []
+            for i in range(R):
+                x = torch.randn(T, d_in, device="cuda", generator=g)
+                x = (x / x.pow(2).mean(dim=1, keepdim=True).sqrt()).to(dt)
+                mods.append({"x": x, "W0": (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt),
+                             "A": ((torch.rand(N, r, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt),
+                             "B": (0.01 * torch.randn(N, d_out, r, device="cuda", generator=g)).to(dt),
+                             "Wg": (torch.randn(N, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt),
+                             "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": mb.alloc_workspace(shape)})
+
+            def step():
+                for m in mods:
+                    rc = lib.meteora_linear_forward(m["x"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(),
+                                                    m["B"].data_ptr(), m["Wg"].data_ptr(), ctypes.byref(shape),
+                                                    m["y"].data_ptr(), m["ws"].data_ptr(), m["ws"].numel(),
+                                                    torch.cuda.current_stream().cuda_stream)
+                    if rc != 0:
+                        raise mb.MeteoraError(rc, "meteora_linear_forward")
+
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            iters = 50 if T <= 256 else 10
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            for m in mods:
+                st = mb.meteora_workspace_status(m["ws"])
+                if st != 0:
+                    raise mb.MeteoraError(st, "device status")
+            us = e0.elapsed_time(e1) * 1e3 / (iters * R)
+            idx0, _ = mb.meteora_workspace_routing(shape, mods[0]["ws"])
+            touched = int(torch.unique(idx0).numel())
+            nbytes = (d_in * d_out + N * d_in + touched * r * (d_in + d_out) + T * (d_in + d_out)) * es
+            flops = 2.0 * T * d_in * d_out + 2.0 * T * N * d_in + 2.0 * T * k * r * (d_in + d_out)
+            t_mem, t_tc = nbytes / hbm / 1e3, flops / tc / 1e6
+            bound = "hbm" if t_mem >= t_tc else "tensor"
+            print(json.dumps({"variant": pt, "shape": "4096->4096", "T": T, "us_per_call": round(us, 2),
+                              "tokens_per_s": round(T / us * 1e6), "bound": bound,
+                              "roofline_us": round(max(t_mem, t_tc), 2),
+                              "frac_of_roofline": round(max(t_mem, t_tc) / us, 3),
+                              "plan": mb.meteora_describe_plan(shape).split(" fused_refused")[0]}), flush=True)
+            del mods, graph
+
+
 def main():
     args = parse_args()
-    if args.sweep:
+    if args.variants:
+        run_variants()
+    elif args.sweep:
         run_sweep(args)
         run_layer_sweep()
     elif args.impl == "reference":
