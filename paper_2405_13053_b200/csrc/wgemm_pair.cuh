@@ -13,9 +13,12 @@
 //                       released, and completion is announced, by tcgen05.commit multicast to both CTAs.
 //   warps 2-9 (both)    stage the B rows of the own 128 rows for every adapter while the main loop runs; when
 //                       the ring is idle, stage the masked, gate-weighted shrink outputs of the own 128 tokens
-//                       there and tell the leader; it then issues N/2 more MMAs of K = 16 (two adapters of
-//                       rank 8) into the same accumulators.  Finally TMEM -> bf16 -> shared memory -> one TMA
-//                       store of the own 128 x 256 tile of y.
+//                       there and tell the leader; it then issues more MMAs of K = 16 into the same
+//                       accumulators.  The expand's contraction axis is cut into blocks of 8 (adapter a, rank
+//                       entries 8c..8c+7): N * r / 8 blocks, two per MMA, at most 28 blocks (56 KB of B rows) per
+//                       round; rank 8 with 28 adapters is one round, larger ranks take several, each staged
+//                       after the previous round's MMAs have completed.  Finally TMEM -> bf16 -> shared
+//                       memory -> one TMA store of the own 128 x 256 tile of y.
 // Every wait is bounded; the pair leaves together (cluster barrier) so that no signal arrives in a CTA that is gone.
 #pragma once
 
@@ -83,7 +86,8 @@ __device__ __forceinline__ uint32_t instr_desc_bf16_pair() {
 
 struct PairParams {
     int T, K, ksteps, stages;
-    int d_out, N, k, na;          // na: adapters rounded up to even
+    int d_out, N, k, r;           // rank r: a multiple of 8
+    int nblk, rb;                 // blocks of 8 expand columns: N * r / 8 in all, rb (even) per round
     int row_tiles;
     int epi_off, slab_off;        // staging area behind the barriers; the B rows sit at slab_off inside it
     const int32_t* topk_idx;
@@ -181,15 +185,20 @@ k_wgemm_pair(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CU
                 umma_commit_pair(bar_base + (p.stages + s) * 8);  // both rings may refill this stage
             }
             umma_commit_pair(bar_main);                            // both rings are idle
-            if (ok) ok = mbar_wait_cluster(bar_us, 0);             // both CTAs have staged their operands
-            if (ok) {
+            // LoRA expand as a K extension of the same accumulation, round by round: rb/2 MMAs of K = 16 (two
+            // blocks of 8 expand columns) over un-swizzled core matrices, 2 KB per block and operand
+            const int rounds = (p.nblk + p.rb - 1) / p.rb;
+            for (int rho = 0; rho < rounds && ok; ++rho) {
+                ok = mbar_wait_cluster(bar_us, rho & 1);           // both CTAs have staged this round's operands
+                if (!ok) break;
                 tc_fence_after();
-                // LoRA expand as a K extension of the same accumulation: na/2 MMAs of K = 16 (two adapters)
                 const uint32_t slab_a = smem_u32(epi + p.slab_off), us_a = ring;
-                const uint32_t ka = kBM * 16, kb = kPairHalf * 16;   // bytes from one adapter to the next
-                for (int m = 0; m < p.na / 2; ++m)
+                const uint32_t ka = kBM * 16, kb = kPairHalf * 16;   // bytes from one block to the next
+                const int nb = min(p.rb, (p.nblk - rho * p.rb + 1) / 2 * 2);
+                for (int m = 0; m < nb / 2; ++m)
                     umma_bf16_pair(tmem_base, smem_desc_plain(slab_a + 2 * m * ka, ka, 128),
-                                   smem_desc_plain(us_a + 2 * m * kb, kb, 128), idesc, (niter | m) != 0);
+                                   smem_desc_plain(us_a + 2 * m * kb, kb, 128), idesc, (niter | rho | m) != 0);
+                if (rho + 1 < rounds) umma_commit_pair(bar_main);  // staging buffers free for the next round
             }
             umma_commit_pair(bar_acc);                             // accumulators complete in both CTAs
             if (!ok) {
@@ -201,63 +210,79 @@ k_wgemm_pair(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CU
         // ------------------------------------------------------------------ epilogue warps (both CTAs)
         const int quad = warp & 3;
         const int etid = threadIdx.x - 64;
-        // B rows of the own 128 output rows for every adapter: un-swizzled K-major core matrices as stored
-        {
-            uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
-            const uint4* Bv = reinterpret_cast<const uint4*>(p.B);
-            const int total = p.na * kBM;
-            constexpr int U = 4;
-            for (int v0 = etid; v0 < total; v0 += U * kEpiThreads) {
-                uint4 val[U];
+        // Round by round: B rows of the own 128 output rows (block q = adapter q / (r/8), rank entries 8 (q % (r/8)) ..,
+        // 16 bytes per row: un-swizzled K-major core matrices) and us[q][t 0..128)[8] = bf16(w_j * (A_a x_t)[8c..])
+        // where own token t picked adapter a at rank j, else 0.  Round 0's B rows are staged while the main loop
+        // runs; everything else waits until the MMAs that read the buffers before have completed.
+        const int cpa = p.r >> 3;                                   // blocks per adapter
+        const int rounds = (p.nblk + p.rb - 1) / p.rb;
+        const int ntok = max(0, min(kPairHalf, p.T - tokh));
+        bool ring_ok = true;
+        for (int rho = 0; rho < rounds; ++rho) {
+            const int q0 = rho * p.rb, nb = min(p.rb, (p.nblk - q0 + 1) / 2 * 2);
+            if (rho > 0) {
+                ring_ok = ring_ok && mbar_wait(bar_main, rho & 1);   // previous round's MMAs done
+            }
+            {
+                uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
+                const uint4* Bv = reinterpret_cast<const uint4*>(p.B);
+                const int total = nb * kBM;
+                constexpr int U = 4;
+                for (int v0 = etid; v0 < total; v0 += U * kEpiThreads) {
+                    uint4 val[U];
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int v = v0 + u * kEpiThreads;
-                    const int a = v / kBM, row = v - a * kBM;
-                    val[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (v < total && a < p.N && tile_m * kBM + row < p.d_out)
-                        val[u] = __ldg(Bv + (size_t)a * p.d_out + tile_m * kBM + row);
-                }
+                    for (int u = 0; u < U; ++u) {
+                        const int v = v0 + u * kEpiThreads;
+                        const int q = q0 + v / kBM, row = v % kBM;
+                        const int a = q / cpa, c = q - a * cpa;
+                        val[u] = make_uint4(0u, 0u, 0u, 0u);
+                        if (v < total && a < p.N && tile_m * kBM + row < p.d_out)
+                            val[u] = __ldg(Bv + ((size_t)a * p.d_out + tile_m * kBM + row) * cpa + c);
+                    }
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int v = v0 + u * kEpiThreads;
-                    if (v < total) slab[v] = val[u];
+                    for (int u = 0; u < U; ++u) {
+                        const int v = v0 + u * kEpiThreads;
+                        if (v < total) slab[v] = val[u];
+                    }
                 }
             }
-        }
-        if (p.pdl_wait) asm volatile("griddepcontrol.wait;" ::: "memory");   // the routing comes from the previous kernel
-        bool ring_ok = mbar_wait(bar_main, 0);
-        if (!ring_ok && lane == 0) {
-            atomicExch(p.status, 1);
-            atomicExch(p.status + 4, 1350);
-        }
-        // us[a][t 0..128)[8] = bf16(w_j * A_a x_t) where own token t picked adapter a at rank j, else 0
-        {
-            uint4* us = reinterpret_cast<uint4*>(ring_ptr);
-            const int total = p.na * kPairHalf;
-            for (int v = etid; v < total; v += kEpiThreads) us[v] = make_uint4(0u, 0u, 0u, 0u);
+            if (rho == 0) {
+                if (p.pdl_wait) asm volatile("griddepcontrol.wait;" ::: "memory");   // the routing comes from the previous kernel
+                ring_ok = mbar_wait(bar_main, 0);                   // main loop done: the ring is idle
+            }
+            if (!ring_ok && lane == 0) {
+                atomicExch(p.status, 1);
+                atomicExch(p.status + 4, 1350);
+            }
+            {
+                uint4* us = reinterpret_cast<uint4*>(ring_ptr);
+                const int total = nb * kPairHalf;
+                for (int v = etid; v < total; v += kEpiThreads) us[v] = make_uint4(0u, 0u, 0u, 0u);
+                epi_barrier();
+                const int items = ntok * p.k * cpa;                  // (token, pick, chunk of 8 rank entries)
+                const int32_t* idx = p.topk_idx + (size_t)tokh * p.k;
+                const float4* uw4 = reinterpret_cast<const float4*>(p.uw + (size_t)tokh * p.k * p.r);
+                for (int i = etid; i < items; i += kEpiThreads) {
+                    const int slot = i / cpa, c = i - slot * cpa;
+                    const int a = __ldg(idx + slot);
+                    const int q = a * cpa + c - q0;
+                    if (a >= 0 && a < p.N && q >= 0 && q < nb) {
+                        const float4 lo = __ldg(uw4 + 2 * i), hi = __ldg(uw4 + 2 * i + 1);
+                        const __nv_bfloat162 h0 = __floats2bfloat162_rn(lo.x, lo.y), h1 = __floats2bfloat162_rn(lo.z, lo.w);
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(hi.x, hi.y), h3 = __floats2bfloat162_rn(hi.z, hi.w);
+                        uint4 val;
+                        val.x = *reinterpret_cast<const uint32_t*>(&h0);
+                        val.y = *reinterpret_cast<const uint32_t*>(&h1);
+                        val.z = *reinterpret_cast<const uint32_t*>(&h2);
+                        val.w = *reinterpret_cast<const uint32_t*>(&h3);
+                        us[q * kPairHalf + slot / p.k] = val;
+                    }
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
             epi_barrier();
-            const int ntok = max(0, min(kPairHalf, p.T - tokh));
-            const int slots = ntok * p.k;
-            const int32_t* idx = p.topk_idx + (size_t)tokh * p.k;
-            const float4* uw4 = reinterpret_cast<const float4*>(p.uw + (size_t)tokh * p.k * 8);
-            for (int i = etid; i < slots; i += kEpiThreads) {
-                const int a = __ldg(idx + i);
-                if (a >= 0 && a < p.N) {
-                    const float4 lo = __ldg(uw4 + 2 * i), hi = __ldg(uw4 + 2 * i + 1);
-                    const __nv_bfloat162 q0 = __floats2bfloat162_rn(lo.x, lo.y), q1 = __floats2bfloat162_rn(lo.z, lo.w);
-                    const __nv_bfloat162 q2 = __floats2bfloat162_rn(hi.x, hi.y), q3 = __floats2bfloat162_rn(hi.z, hi.w);
-                    uint4 val;
-                    val.x = *reinterpret_cast<const uint32_t*>(&q0);
-                    val.y = *reinterpret_cast<const uint32_t*>(&q1);
-                    val.z = *reinterpret_cast<const uint32_t*>(&q2);
-                    val.w = *reinterpret_cast<const uint32_t*>(&q3);
-                    us[a * kPairHalf + i / p.k] = val;
-                }
-            }
+            if (etid == 0) mbar_arrive_cluster(map_to_cta(bar_us, 0));
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
-        epi_barrier();
-        if (etid == 0) mbar_arrive_cluster(map_to_cta(bar_us, 0));
         bool acc_ok = mbar_wait(bar_acc, 0);
         if (!acc_ok && lane == 0) {
             atomicExch(p.status, 1);

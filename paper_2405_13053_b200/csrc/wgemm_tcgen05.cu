@@ -818,7 +818,8 @@ int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits) {
 }
 
 struct Plan;
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi = false);
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi = false,
+                      int bn_force = 0);
 
 struct Plan {
     int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
@@ -840,7 +841,7 @@ int stacked_zsplits_bound(int T) {
     return std::min(kMaxZSplits, std::max(1, 148 / tiles));
 }
 
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi) {
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi, int bn_force) {
     const Tuning& tn = tuning();
     Plan pl = {};
     const int ksteps = (K + kBK - 1) / kBK;
@@ -849,6 +850,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     // tiles across a cluster costs more than it gains)
     int bn = tn.tile_tokens > 0 ? tn.tile_tokens : (T <= 256 ? (T + 15) / 16 * 16 : 256);
     if (tn.tile_tokens == 0 && T > 256 && row_tiles * ((T + 255) / 256) < sm_count()) bn = 128;
+    if (bn_force > 0) bn = bn_force;
     bn = std::min(256, std::max(16, (bn + 15) / 16 * 16));
     pl.BN = bn;
     pl.n_tiles = (T + bn - 1) / bn;
@@ -959,6 +961,15 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     pl.tmem_cols = cols;
     pl.epi_off = (int)align_up((size_t)(2 * std::max(stages, 16) + 3) * 8 + 16, 128);
     pl.smem = 1024 + (size_t)stages * stage_bytes + pl.epi_off + epi_bytes;
+    // Large ranks with the expand on CUDA cores stage k * r floats per token: if that does not leave room for two
+    // ring stages, take fewer tokens per tile.
+    if (pl.smem > 227 * 1024 && bn_force == 0 && tn.tile_tokens == 0) {
+        for (int cand = 128; cand >= 16; cand /= 2) {
+            if (cand >= bn) continue;
+            const Plan q = make_plan(row_tiles, T, K, lora, N, r, k, fused_epi, cand);
+            if (q.smem <= 227 * 1024) return q;
+        }
+    }
     return pl;
 }
 
@@ -1132,20 +1143,21 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
 // Prefill batches on pairs of SMs (wgemm_pair.cuh): 256 x 256 tiles, rank 8, y stored by TMA.
 struct PairPlan {
     bool ok;
-    int stages, na, epi_off;
+    int stages, nblk, rb, epi_off;   // blocks of 8 expand columns (adapter, 8 rank entries): all, per round
     size_t smem;
 };
 static PairPlan make_pair_plan(const meteora_shape_t& s) {
     PairPlan pp = {};
     if (!tuning().pair || tuning().simt_expand || tuning().no_tma_store || tuning().tile_tokens || tuning().splits > 1)
         return pp;
-    if (!tc_path_supported(s) || s.r != 8 || s.T <= 256 || s.d_out % 8 != 0) return pp;
+    if (!tc_path_supported(s) || s.r % 8 != 0 || s.T <= 256 || s.d_out % 8 != 0) return pp;
     // Measured on B200: ahead of the one-CTA tiles (by 8 - 17 %, and by more where those fall back to 128-token
     // tiles) as soon as the pairs cover a quarter of the SMs; below that too few SMs work at all.
     const int pairs = ((s.d_out + 2 * kBM - 1) / (2 * kBM)) * ((s.T + kPairTokens - 1) / kPairTokens);
     if (tuning().pair == 1 && pairs * 4 < sm_count()) return pp;
-    pp.na = (s.N + 1) / 2 * 2;
-    const size_t slab = (size_t)pp.na * kBM * 16, us = (size_t)pp.na * kPairHalf * 16;
+    pp.nblk = s.N * (s.r / 8);
+    pp.rb = std::min((pp.nblk + 1) / 2 * 2, 28);                  // 28 blocks: 56 KB of B rows, 56 KB of us per round
+    const size_t slab = (size_t)pp.rb * kBM * 16, us = (size_t)pp.rb * kPairHalf * 16;
     const size_t ystage = (size_t)kPairTokens * kBM * 2, stage = kWTileBytes + kPairHalf * 128;
     for (int stages = 6; stages >= 2; --stages) {
         const size_t epi_off = align_up((size_t)(2 * stages + 3) * 8 + 16, 128);
@@ -1177,7 +1189,9 @@ static int launch_base_lora_pair(const void* x, const void* W0, const void* B, c
     p.d_out = s.d_out;
     p.N = s.N;
     p.k = s.k;
-    p.na = pp.na;
+    p.r = s.r;
+    p.nblk = pp.nblk;
+    p.rb = pp.rb;
     p.row_tiles = row_tiles;
     p.epi_off = pp.epi_off;
     p.slab_off = 0;

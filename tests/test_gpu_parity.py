@@ -177,6 +177,8 @@ FORWARD_CASES = [
     dict(T=300, d_in=2048, d_out=640, N=28, r=8, k=2, dtype="bf16"),              # two token tiles, ragged tail
     dict(T=50, d_in=512, d_out=128, N=40, r=16, k=3, dtype="bf16"),               # 40 adapters, rank 16, top-3
     dict(T=20, d_in=256, d_out=128, N=8, r=8, k=1, dtype="bf16"),                 # top-1
+    dict(T=40, d_in=512, d_out=256, N=28, r=32, k=4, dtype="bf16"),               # rank 32, top-4, decode batch
+    dict(T=600, d_in=512, d_out=200, N=28, r=64, k=2, dtype="bf16"),              # rank 64 prefill, d_out % 8 == 0 only
     dict(T=24, d_in=256, d_out=136, N=4, r=8, k=4, dtype="bf16", temperature=20.0),  # k = N with temperature
 ]
 
@@ -287,12 +289,13 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T):
 # one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
 # (257), a contraction length that is no multiple of 64, and adapters up to an odd count.  The stacked shrink of
 # these calls runs on pairs as well: its rows are [A; Wg] packed into 128-row tiles, two tiles per pair.
-@pytest.mark.parametrize("d_in,d_out,T,N,k", [
-    (1024, 640, 600, 28, 2), (512, 256, 257, 28, 2), (1096, 512, 300, 28, 2), (768, 1024, 1024, 7, 3),
-    (512, 512, 520, 16, 4), (512, 384, 300, 33, 3),      # Wg in a tile of its own; three tiles of stacked rows
+@pytest.mark.parametrize("d_in,d_out,T,N,k,r", [
+    (1024, 640, 600, 28, 2, 8), (512, 256, 257, 28, 2, 8), (1096, 512, 300, 28, 2, 8), (768, 1024, 1024, 7, 3, 8),
+    (512, 512, 520, 16, 4, 8), (512, 384, 300, 33, 3, 8),      # Wg in a tile of its own; three tiles of stacked rows
+    (512, 384, 700, 28, 2, 16), (512, 256, 300, 28, 4, 64), (512, 256, 520, 5, 2, 24),   # ranks 16, 64, 24: 2, 8, 1 rounds
 ])
-def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k):
-    w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, dtype="bf16", x_kind="normal",
+def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k, r):
+    w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
                                 seed=700 + T, b_std=0.3)
     mb.meteora_set_tuning("pair", 2)                                 # 2: also where only a few pairs result
     try:
