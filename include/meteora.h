@@ -139,7 +139,8 @@ int meteora_lora_delta_static(const void* x, const void* A, const void* B, const
  * decode batches (T <= 256, rank 8, d_out <= 16384) as ONE cooperative kernel launch in which
  * the CTAs exchange partial results through the workspace, everything else as three launches
  * (stacked shrink [A; Wg] x, selection, base product with the LoRA expand; for prefill batches of
- * rank 8 on pairs of SMs with two-CTA MMAs).  Every other shape
+ * rank 8 on pairs of SMs with two-CTA MMAs).  A bf16 layer whose rank is no multiple of 8 takes the same
+ * paths with A and B zero-padded to the next multiple of 8 inside the workspace (rewritten by every call).  Every other shape
  * runs on a plain CUDA-core path with the same results up to rounding order.  The workspace header
  * must have been zeroed once (meteora_workspace_init) before its first use; the kernels leave it
  * ready for the next call.  meteora_describe_plan tells which path a shape takes.

@@ -14,7 +14,8 @@ Tuning& tuning() {
     return t;
 }
 
-Workspace carve_workspace(const meteora_shape_t& s, void* base) {
+Workspace carve_workspace(const meteora_shape_t& s_in, void* base) {
+    const meteora_shape_t s = rank_padded(s_in);                 // scratch is sized for the padded rank
     Workspace ws;
     uint8_t* p = (uint8_t*)base;
     size_t off = 0;
@@ -41,8 +42,32 @@ Workspace carve_workspace(const meteora_shape_t& s, void* base) {
     ws.part_g = (float*)take(part_tiles * bn * 128 * sizeof(float));
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);
+    const bool pad = rank_pad_applies(s_in);
+    ws.A_pad = pad ? take((size_t)s.N * s.r * s.d_in * es) : nullptr;
+    ws.B_pad = pad ? take((size_t)s.N * s.d_out * s.r * es) : nullptr;
     ws.bytes = off;
     return ws;
+}
+
+// A[N,r,d_in] -> Ap[N,r8,d_in] and B[N,d_out,r] -> Bp[N,d_out,r8], the new rank entries zero.
+__global__ void k_pad_rank(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ B,
+                           __nv_bfloat16* __restrict__ Ap, __nv_bfloat16* __restrict__ Bp, int N, int r, int r8,
+                           int d_in, int d_out) {
+    const size_t vec_per_row = (size_t)d_in / 8;                 // d_in % 8 == 0: rows of A move as 16-byte vectors
+    const size_t total_a = (size_t)N * r8 * vec_per_row, total_b = (size_t)N * d_out;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_a; i += stride) {
+        const size_t row = i / vec_per_row, v = i - row * vec_per_row;
+        const size_t n = row / r8, q = row - n * r8;
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (q < (size_t)r) val = __ldg(reinterpret_cast<const uint4*>(A + (n * r + q) * d_in) + v);
+        reinterpret_cast<uint4*>(Ap)[i] = val;
+    }
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_b; i += stride) {
+        const __nv_bfloat16* src = B + i * r;
+        __nv_bfloat16* dst = Bp + i * r8;
+        for (int q = 0; q < r8; ++q) dst[q] = q < r ? src[q] : __float2bfloat16_rn(0.f);
+    }
 }
 
 static int check_shape(const meteora_shape_t* s, bool need_out, bool need_r) {
@@ -75,6 +100,13 @@ static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 static int forward_device(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                           const meteora_shape_t& s, void* y, const Workspace& ws, cudaStream_t st) {
     int rc;
+    if (rank_pad_applies(s) && !tuning().force_simt && ws.A_pad && ws.B_pad) {
+        const meteora_shape_t e = rank_padded(s);
+        k_pad_rank<<<296, 256, 0, st>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)B, (__nv_bfloat16*)ws.A_pad,
+                                        (__nv_bfloat16*)ws.B_pad, s.N, s.r, e.r, s.d_in, s.d_out);
+        if ((rc = last_launch_status()) != METEORA_OK) return rc;
+        return forward_device(x, W0, ws.A_pad, ws.B_pad, Wg, e, y, ws, st);
+    }
     Profile& pf = profile();
     const bool timed = pf.open && 2 * (pf.used + 1) <= (int)pf.ev.size();
     if (decode_fused_supported(s)) {
@@ -353,8 +385,10 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
     if (rc != METEORA_OK) return rc;
     if (!buf || buf_bytes == 0) return METEORA_ERR_INVALID_ARG;
     char tmp[512];
-    describe_plan(*shape, tmp, sizeof(tmp));
-    snprintf(buf, buf_bytes, "%s fused_refused=%d", tmp, tuning().fused_refused);
+    const bool pad = rank_pad_applies(*shape) && !tuning().force_simt;
+    describe_plan(pad ? rank_padded(*shape) : *shape, tmp, sizeof(tmp));
+    snprintf(buf, buf_bytes, "%s%s fused_refused=%d", tmp, pad ? " rank_padded_to_multiple_of_8" : "",
+             tuning().fused_refused);
     return METEORA_OK;
 }
 

@@ -26,12 +26,25 @@ struct Workspace {
     int col_logits;     // first logit column inside a u_all row
     float* part_g;      // fused decode: fp32 partial accumulator tiles of the base product (T <= 256 only)
     int32_t* tile_ctr;  // fused decode: one counter per 128-row tile of d_out (inside the header)
+    void* A_pad;        // bf16 layers whose rank is no multiple of 8: A and B zero-padded to the next multiple,
+    void* B_pad;        //           [N,r8,d_in] and [N,d_out,r8], rewritten by every call (nullptr otherwise)
     void* x_dev;        // [T,d_in]  staging for the host-buffer entry point
     void* y_dev;        // [T,d_out]
     size_t bytes;       // total
 };
 
 Workspace carve_workspace(const meteora_shape_t& s, void* base);
+
+// A bf16 layer whose rank is no multiple of 8 runs on the tensor-core paths with its adapters zero-padded to
+// the next multiple of 8 (the padded rank entries contribute exact zeros to Eq. 2).
+inline bool rank_pad_applies(const meteora_shape_t& s) {
+    return s.dtype == METEORA_BF16 && s.d_in % 8 == 0 && s.r > 0 && s.r % 8 != 0;
+}
+inline meteora_shape_t rank_padded(const meteora_shape_t& s) {
+    meteora_shape_t e = s;
+    if (rank_pad_applies(s)) e.r = (s.r + 7) / 8 * 8;
+    return e;
+}
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline size_t elem_size(meteora_dtype_t t) { return t == METEORA_BF16 ? 2 : 4; }
