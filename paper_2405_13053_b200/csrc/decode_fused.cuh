@@ -82,13 +82,13 @@ __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
 // Selection for one token by one warp, every partial copy of the token's row read in ONE round trip: the
 // N*r shrink values and the N logits are summed over the `zsplits` copies in slice order (two 16-byte columns
 // per lane, all loads in flight together) into `wbuf` (shared memory, ld_u floats), then top-k, softmax over
-// the picks (Eq. 3) and uw[t,j,:] = w_j * (A_{i_j} x) come from there.  Rank 8 only; N * 8 + N <= 256 floats
-// per 32 lanes and pass, further passes for larger N.
+// the picks (Eq. 3) and uw[t,j,:] = w_j * (A_{i_j} x) come from there.  The rank r is a multiple of 4; 256 floats
+// per 32 lanes and pass, further passes for more columns.
 __device__ __forceinline__ void select_token_wide(const float* u_part, int ld_u, int col_logits, int zsplits,
-                                                  size_t zstride, int t, int N, int k, float inv_tau, int lane,
+                                                  size_t zstride, int t, int N, int r, int k, float inv_tau, int lane,
                                                   float* wbuf, int32_t* topk_idx, float* topk_w, float* uw) {
     constexpr int ZMAX = 16;
-    const int n_a4 = N * 2, n_c4 = n_a4 + (N + 3) / 4;             // 16-byte chunks: shrink values, then logits
+    const int n_a4 = N * r / 4, n_c4 = n_a4 + (N + 3) / 4;         // 16-byte chunks: shrink values, then logits
     const float* row = u_part + (size_t)t * ld_u;
     for (int c0 = 0; c0 < n_c4; c0 += 64) {
         float4 acc[2];
@@ -127,26 +127,27 @@ __device__ __forceinline__ void select_token_wide(const float* u_part, int ld_u,
         topk_idx[(size_t)t * k + lane] = idx;
         topk_w[(size_t)t * k + lane] = w;
     }
-    for (int c0 = 0; c0 < k * 8; c0 += 32) {
+    for (int c0 = 0; c0 < k * r; c0 += 32) {
         const int c = c0 + lane;
-        const int j = min(c / 8, k - 1), q = c - j * 8;
+        const int j = min(c / r, k - 1), q = c - j * r;
         const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
         const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
-        if (c < k * 8) uw[(size_t)t * k * 8 + c] = wj * wbuf[ij * 8 + q];
+        if (c < k * r) uw[(size_t)t * k * r + c] = wj * wbuf[ij * r + q];
     }
     __syncwarp();
 }
 
 // B rows [row0, row0 + nrows) of every adapter (8 bf16 = 16 bytes each) as slab[e][row % 4][row / 4], so that
 // threads owning consecutive groups of 4 rows read consecutive 16-byte words; rows past d_out are zero.
-__device__ __forceinline__ void stage_slab_rows(const __nv_bfloat16* B, int d_out, int N, uint4* slab, int row0,
-                                                int nrows, int etid) {
+// (For ranks above 8 a row has cpa = r / 8 such 16-byte words: slab[e][chunk][row % 4][row / 4].)
+__device__ __forceinline__ void stage_slab_rows(const __nv_bfloat16* B, int d_out, int N, int cpa, uint4* slab,
+                                                int row0, int nrows, int etid) {
     const uint4* Bg = reinterpret_cast<const uint4*>(B);
-    const int total = N * nrows, nq = nrows / 4;
+    const int per_e = nrows * cpa, total = N * per_e, nq = nrows / 4;
     for (int i = etid; i < total; i += kEpiThreads) {
-        const int e = i / nrows, rl = i - e * nrows, o = row0 + rl;
-        slab[e * nrows + (rl & 3) * nq + (rl >> 2)] =
-            o < d_out ? __ldg(Bg + (size_t)e * d_out + o) : make_uint4(0u, 0u, 0u, 0u);
+        const int e = i / per_e, w = i - e * per_e, rl = w / cpa, c = w - rl * cpa, o = row0 + rl;
+        slab[(e * cpa + c) * nrows + (rl & 3) * nq + (rl >> 2)] =
+            o < d_out ? __ldg(Bg + ((size_t)e * d_out + o) * cpa + c) : make_uint4(0u, 0u, 0u, 0u);
     }
 }
 
@@ -158,7 +159,7 @@ __device__ __forceinline__ void stage_slab_rows(const __nv_bfloat16* B, int d_ou
 // barrier once (`routing_pending`), after issuing their first loads.  `nthr` threads (etid = 0 .. nthr-1) share
 // the tile: all 256 epilogue threads, or half of them when the CTA finishes rows of two tiles at once.
 template <int C, int U>
-__device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, const float* const (&parts)[C], int c,
+__device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, int cpa, const float* const (&parts)[C], int c,
                                             int tile_row0, int q0, int nq, int ntok, const uint4* slab,
                                             const float* s_uw, const int* s_idx, int etid, int nthr,
                                             bool& routing_pending) {
@@ -194,12 +195,14 @@ __device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, 
             }
             for (int j = 0; j < k; ++j) {
                 const int slot = t * k + j;
-                const float4 u0 = s_uw4[2 * slot], u1 = s_uw4[2 * slot + 1];
-                const uint4* b = slab + (size_t)s_idx[slot] * slab_rows + ql;
-                fma8(b[0], u0, u1, acc.x);
-                fma8(b[nq], u0, u1, acc.y);
-                fma8(b[2 * nq], u0, u1, acc.z);
-                fma8(b[3 * nq], u0, u1, acc.w);
+                for (int ch = 0; ch < cpa; ++ch) {               // 8 rank entries at a time
+                    const float4 u0 = s_uw4[2 * (slot * cpa + ch)], u1 = s_uw4[2 * (slot * cpa + ch) + 1];
+                    const uint4* b = slab + (size_t)(s_idx[slot] * cpa + ch) * slab_rows + ql;
+                    fma8(b[0], u0, u1, acc.x);
+                    fma8(b[nq], u0, u1, acc.y);
+                    fma8(b[2 * nq], u0, u1, acc.z);
+                    fma8(b[3 * nq], u0, u1, acc.w);
+                }
             }
             const int o = tile_row0 + (q0 + ql) * 4;
             __nv_bfloat16* dst = y + (size_t)t * d_out + o;
@@ -228,7 +231,7 @@ __device__ __forceinline__ int module_of_tile(const DecodeModule* mod, int n_mod
 }
 
 template <int C, int U>
-__device__ __forceinline__ void finish_tile(__nv_bfloat16* y, int d_out, int k, int tile_row0, const float* part_g,
+__device__ __forceinline__ void finish_tile(__nv_bfloat16* y, int d_out, int k, int cpa, int tile_row0, const float* part_g,
                                             size_t part_stride, int units, int M, int upt, int tile, int first_cta, int c,
                                             int q0, int nq, int ntok, const uint4* slab, const float* s_uw,
                                             const int* s_idx, int etid, int nthr, bool& routing_pending) {
@@ -240,7 +243,7 @@ __device__ __forceinline__ void finish_tile(__nv_bfloat16* y, int d_out, int k, 
         const int seg = (int)((unsigned)units * (unsigned)cta / (unsigned)M) / upt == tile ? 0 : 1;
         parts[q] = part_g + ((size_t)cta * 2 + seg) * part_stride;
     }
-    finish_rows<C, U>(y, d_out, k, parts, c, tile_row0, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
+    finish_rows<C, U>(y, d_out, k, cpa, parts, c, tile_row0, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
 }
 
 #ifdef METEORA_TRACE
@@ -447,8 +450,8 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             for (int it = aux_id * nwarps + warp; it < d.n_mod * p.T; it += n_active * nwarps) {
                 const int sm = it / p.T, t = it - sm * p.T;
                 const DecodeModule& mo = d.mod[sm];
-                select_token_wide(mo.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.k,
-                                  d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
+                select_token_wide(mo.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.r,
+                                  p.k, d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
             }
             __syncthreads();
             if (threadIdx.x == 0) {
@@ -511,12 +514,12 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 for (int sg = 0; sg < nseg; ++sg) {
                     const DecodeModule& mo = d.mod[module_of_tile(d.mod, d.n_mod, tile_a + sg)];
                     int* s_idx = reinterpret_cast<int*>(epi + p.idx_off) + sg * p.BN * p.k;
-                    float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off) + sg * p.BN * p.k * 2;
+                    float4* s_uw4 = reinterpret_cast<float4*>(epi + p.uw_off) + sg * p.BN * p.k * (p.r / 4);
                     const float4* uw4 = reinterpret_cast<const float4*>(mo.uw);
 #pragma unroll 8
                     for (int i = lane; i < slots; i += 32) s_idx[i] = min(max(__ldcg(mo.topk_idx + i), 0), p.N - 1);
 #pragma unroll 8
-                    for (int i = lane; i < 2 * slots; i += 32) s_uw4[i] = __ldcg(uw4 + i);
+                    for (int i = lane; i < slots * (p.r / 4); i += 32) s_uw4[i] = __ldcg(uw4 + i);
                 }
                 __syncwarp();
                 asm volatile("bar.arrive 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
@@ -556,6 +559,7 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             // Which rows of which tile this CTA finishes: tile `t` is shared by the CTAs owner(first unit) ..
             // owner(last unit), in that order; contributor j of c takes the groups of 4 rows [32j/c, 32(j+1)/c).
             int d_tile[2], d_first[2], d_c[2], d_q0[2], d_nq[2], d_mod[2], d_row0[2];
+            const int cpa = p.r >> 3;                                        // 16-byte words per B row
             uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
             uint4* d_slab[2];
             int slab_words = 0;
@@ -574,9 +578,9 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 d_mod[sg] = module_of_tile(d.mod, d.n_mod, tile);
                 d_row0[sg] = (tile - d.mod[d_mod[sg]].tile0) * kBM;          // the tile's first row inside its module
                 // B rows of that slice for every adapter: no routing needed yet
-                stage_slab_rows(d.mod[d_mod[sg]].B, d.mod[d_mod[sg]].d_out, p.N, d_slab[sg], d_row0[sg] + 4 * d_q0[sg],
-                                4 * d_nq[sg], etid);
-                slab_words += p.N * 4 * d_nq[sg];
+                stage_slab_rows(d.mod[d_mod[sg]].B, d.mod[d_mod[sg]].d_out, p.N, cpa, d_slab[sg],
+                                d_row0[sg] + 4 * d_q0[sg], 4 * d_nq[sg], etid);
+                slab_words += p.N * cpa * 4 * d_nq[sg];
             }
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
             // Accumulators out of TMEM to the fp32 scratch, segment by segment (lane = row, a warp writes 128
@@ -619,18 +623,18 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 asm volatile("bar.sync %0, %1;" ::"r"(3 + sg), "r"(nthr) : "memory");
                 const int c = d_c[sg];
                 const DecodeModule& mo = d.mod[d_mod[sg]];
-                const float* s_uw = reinterpret_cast<const float*>(epi + p.uw_off) + sg * p.BN * p.k * 8;
+                const float* s_uw = reinterpret_cast<const float*>(epi + p.uw_off) + sg * p.BN * p.k * p.r;
                 const int* s_idx = reinterpret_cast<const int*>(epi + p.idx_off) + sg * p.BN * p.k;
                 if (c <= 1)
-                    finish_tile<1, 4>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<1, 4>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 2)
-                    finish_tile<2, 4>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<2, 4>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 4)
-                    finish_tile<4, 4>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<4, 4>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else if (c <= 8)
-                    finish_tile<8, 2>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<8, 2>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else
-                    finish_tile<16, 1>(mo.y, mo.d_out, p.k, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+                    finish_tile<16, 1>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
             }
             if (routing_pending) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);

@@ -1305,7 +1305,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     // Measured on B200 (4096 -> 4096): the single launch is ahead of the three-launch chain at every decode
     // batch size (15.7 vs 16.5 us at T = 1, 19.5 vs 25 us at T = 128).
     if (!tn.fused) return fp;
-    if (!tc_path_supported(s) || s.T > 256 || s.r != 8 || tn.simt_expand) return fp;
+    if (!tc_path_supported(s) || s.T > 256 || s.r % 8 != 0 || tn.simt_expand) return fp;
     fp.row_tiles = 0;                                            // of all modules of the group together
     size_t w0_bytes = 0;
     for (int m = 0; m < G; ++m) {
@@ -1328,7 +1328,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     {
         // staging of the last step (B rows, routing) comes first; with 256-token tiles two k-steps per stage
         // would leave room for one stage only
-        const size_t staged = (size_t)s.N * kBM * 16 + 2 * (size_t)pl.BN * s.k * (s.r * 4 + 4) + 2048;
+        const size_t staged = (size_t)s.N * kBM * s.r * 2 + 2 * (size_t)pl.BN * s.k * (s.r * 4 + 4) + 2048;
         const size_t one = kWTileBytes + (size_t)pl.BN * 128;
         while (pl.kc > 1 && staged + 2 * pl.kc * one > 226 * 1024) pl.kc /= 2;
     }
@@ -1369,7 +1369,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     const int own_rows = whole ? 4 * ((32 + n_main / fp.row_tiles - 1) / (n_main / fp.row_tiles)) : kBM;
     // the routing once per tile a CTA finishes rows of (one tile, or two that may belong to two modules)
     const int duties = whole ? 1 : 2;
-    pl.uw_off = (int)align_up((size_t)s.N * own_rows * 16, 16);
+    pl.uw_off = (int)align_up((size_t)s.N * own_rows * s.r * 2, 16);
     pl.idx_off = pl.uw_off + duties * pl.BN * s.k * s.r * 4;
     const size_t epi_bytes = (size_t)pl.idx_off + (size_t)duties * pl.BN * s.k * 4;
     pl.epi_off = (int)align_up((size_t)(2 * 16 + 3) * 8 + 16, 128);

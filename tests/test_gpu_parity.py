@@ -278,10 +278,12 @@ def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
 
 # Adapter counts that change the layout of the stacked shrink: Wg behind A's only tile (N = 4), Wg in a tile of
 # its own (N = 16: A fills its tile), three A tiles with Wg behind 8 rows (N = 33, logits beyond one warp).
-@pytest.mark.parametrize("N,k,T", [(4, 2, 9), (16, 4, 40), (33, 3, 130), (2, 1, 3)])
-def test_single_launch_decode_kernel_adapter_counts(N, k, T):
-    w = workloads.make_workload("fused_n", T=T, d_in=768, d_out=896, N=N, k=k, dtype="bf16", x_kind="normal",
-                                seed=900 + N, b_std=0.3)
+# ... and ranks above 8 (16-byte words per B row: 2, 3, 4), which also change the number of stacked-shrink tiles.
+@pytest.mark.parametrize("N,k,T,r", [(4, 2, 9, 8), (16, 4, 40, 8), (33, 3, 130, 8), (2, 1, 3, 8),
+                                     (28, 2, 20, 16), (28, 2, 128, 32), (10, 3, 64, 24)])
+def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
+    w = workloads.make_workload("fused_n", T=T, d_in=768, d_out=896, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
+                                seed=900 + N + r, b_std=0.3)
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
     assert "fused_decode" in mb.meteora_describe_plan(shape)
     check_forward(w, y_tol=1e-2)
