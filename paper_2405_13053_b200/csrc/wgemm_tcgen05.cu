@@ -1357,6 +1357,9 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     int n_main = std::min(m_max, 6 * fp.row_tiles);
     // (large batches exchange 64 KB and more per partial tile: there even 80 % of the CTAs are the better deal)
     if (m_even > 0 && m_even * 10 >= n_main * (s.T >= 96 ? 8 : 9)) n_main = m_even;
+    // an uneven split makes a CTA finish up to 128 rows: if the B rows of 128 rows of every adapter (large ranks)
+    // would crowd out the ring, stay with whole tiles per CTA group
+    if (m_even > 0 && n_main % fp.row_tiles != 0 && (size_t)s.N * kBM * s.r * 2 > 64 * 1024) n_main = m_even;
     if (tn.splits > 0 && tn.splits * fp.row_tiles <= m_max) n_main = std::min(tn.splits, 8) * fp.row_tiles;
     n_main = (int)std::min<long long>(n_main, units);
     if (n_main < fp.row_tiles || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
