@@ -51,6 +51,7 @@ def _load():
         lib.meteora_oracle_lora_delta.argtypes = [_f32p, _f32p, _f32p, _i32p, _f32p] + [c_int] * 6 + [_f64p]
         lib.meteora_oracle_linear_forward.argtypes = [_f32p] * 5 + [c_int] * 6 + [c_double, _f64p, _i32p, _f64p]
         lib.meteora_oracle_linear_forward_routed.argtypes = [_f32p] * 5 + [_i32p] + [c_int] * 6 + [c_double, _f64p]
+        lib.meteora_oracle_gate_backward.argtypes = [_f32p] * 5 + [_i32p] + [c_int] * 6 + [c_double, _f64p, _f64p]
         _lib = lib
     return _lib
 
@@ -155,3 +156,21 @@ def linear_forward_routed(x, W0, A, B, Wg, topk_idx, temperature=1.0):
                                                         d_out, N, r, k, float(temperature), _p(y, _f64p)),
            "linear_forward_routed")
     return y
+
+
+def gate_backward(x, A, B, Wg, dy, topk_idx, temperature=1.0):
+    """Gradient of the gate weights through Eq. 3 and Eq. 2 for a given selection (Sec. 3.2).
+    Returns (dlogit[T,k] float64, dWg[N,d_in] float64)."""
+    T, d_in = x.shape
+    N, r, _ = A.shape
+    d_out = B.shape[1]
+    k = topk_idx.shape[1]
+    x, A, B = _f32(x, (T, d_in)), _f32(A, (N, r, d_in)), _f32(B, (N, d_out, r))
+    Wg, dy, idx = _f32(Wg, (N, d_in)), _f32(dy, (T, d_out)), _i32(topk_idx, (T, k))
+    dlogit = np.empty((T, k), np.float64)
+    dWg = np.empty((N, d_in), np.float64)
+    _check(_load().meteora_oracle_gate_backward(_p(x, _f32p), _p(A, _f32p), _p(B, _f32p), _p(Wg, _f32p),
+                                                _p(dy, _f32p), _p(idx, _i32p), T, d_in, d_out, N, r, k,
+                                                float(temperature), _p(dlogit, _f64p), _p(dWg, _f64p)),
+           "gate_backward")
+    return dlogit, dWg

@@ -20,6 +20,8 @@
  *     one group per adapter; the routing function below produces that grouping
  *     as a stable counting sort.
  *   - App. A.5: a temperature divides the selected logits before the softmax.
+ *   - Sec. 3.2: only the gating networks are trained; meteora_oracle_gate_backward is the chain rule of Eq. 2
+ *     and Eq. 3 with respect to the gate weights.
  *
  * Storage convention (row-major, contiguous; transposes of the paper's
  * (n,d,r) / (n,r,h) tensors so that every contraction runs along the
@@ -250,5 +252,67 @@ int meteora_oracle_linear_forward_routed(const float *x, const float *W0, const 
         free(logit);
         free(w);
     }
+    return ORACLE_OK;
+}
+
+/*
+ * Gradient of the gating network's weights (Sec. 3.2: the base model and the adapters stay fixed, only the
+ * gating networks are trained; with top-k > 1 the token loss reaches them through the weights of Eq. 3).
+ * Given dy = dL/dy and a selection, by the chain rule on Eq. 2 and Eq. 3 (temperature of App. A.5):
+ *     v_j        = (x A_{i_j}) B_{i_j}                      the adapter's own output, in R^{d_out}
+ *     g_j        = < dy, v_j >                             = dL/dw_j
+ *     dlogit_j   = w_j (g_j - sum_m w_m g_m) / tau         softmax over the selected logits
+ *     dWg[i_j,:] += dlogit_j * x                           G(x) = Wg x
+ * summed over the tokens.  Unselected adapters get no gradient from this path.  fp64 throughout; the weights
+ * are recomputed from this side's logits for the given selection, as in the routed forward.
+ */
+int meteora_oracle_gate_backward(const float *x, const float *A, const float *B, const float *Wg, const float *dy,
+                                 const int32_t *topk_idx, int T, int d_in, int d_out, int N, int r, int k,
+                                 double tau, double *dlogit, double *dWg) {
+    if (bad_dims(T, d_in, N, k) || d_out <= 0 || r <= 0 || !(tau > 0.0)) return ORACLE_BAD_ARG;
+    for (size_t s = 0; s < (size_t)T * k; ++s)
+        if (topk_idx[s] < 0 || topk_idx[s] >= N) return ORACLE_BAD_ARG;
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        const float *xt = x + (size_t)t * d_in;
+        const float *dyt = dy + (size_t)t * d_out;
+        const int32_t *sel = topk_idx + (size_t)t * k;
+        float *logit = (float *)malloc(sizeof(float) * (size_t)N);
+        double *w = (double *)malloc(sizeof(double) * (size_t)k);
+        double *g = (double *)malloc(sizeof(double) * (size_t)k);
+        double *u = (double *)malloc(sizeof(double) * (size_t)r);
+        token_logits(xt, Wg, d_in, N, logit);
+        token_weights(logit, sel, k, tau, w);
+        for (int j = 0; j < k; ++j) {
+            const float *Ai = A + (size_t)sel[j] * r * d_in;
+            const float *Bi = B + (size_t)sel[j] * d_out * r;
+            for (int p = 0; p < r; ++p) {
+                double acc = 0.0;
+                for (int d = 0; d < d_in; ++d) acc += (double)Ai[(size_t)p * d_in + d] * (double)xt[d];
+                u[p] = acc;
+            }
+            double gj = 0.0;
+            for (int o = 0; o < d_out; ++o) {
+                double v = 0.0;
+                for (int p = 0; p < r; ++p) v += (double)Bi[(size_t)o * r + p] * u[p];
+                gj += (double)dyt[o] * v;
+            }
+            g[j] = gj;
+        }
+        double mean = 0.0;
+        for (int j = 0; j < k; ++j) mean += w[j] * g[j];
+        for (int j = 0; j < k; ++j) dlogit[(size_t)t * k + j] = w[j] * (g[j] - mean) / tau;
+        free(logit);
+        free(w);
+        free(g);
+        free(u);
+    }
+    for (size_t i = 0; i < (size_t)N * d_in; ++i) dWg[i] = 0.0;
+    for (int t = 0; t < T; ++t)                                  /* in token order: one writer per row at a time */
+        for (int j = 0; j < k; ++j) {
+            double *row = dWg + (size_t)topk_idx[(size_t)t * k + j] * d_in;
+            const double dl = dlogit[(size_t)t * k + j];
+            for (int d = 0; d < d_in; ++d) row[d] += dl * (double)x[(size_t)t * d_in + d];
+        }
     return ORACLE_OK;
 }
