@@ -173,6 +173,25 @@ int meteora_linear_forward_group(const void* x, const void* const* W0, const voi
                                  size_t workspace_bytes, void* stream);
 
 /*
+ * Gradient of the gate weights (Sec. 3.2: the base model and the adapters stay fixed, only the gating networks
+ * are trained; with top-k > 1 the token loss reaches them through the weights of Eq. 3).  Given dy = dL/dy
+ * [T,d_out] (shape->dtype) and the routing a forward left (topk_idx, topk_w; meteora_workspace_routing):
+ *   g[t,j]      = < dy[t], B_e (A_e x[t]) >,  e = topk_idx[t,j]
+ *   dlogit[t,j] = topk_w[t,j] * (g[t,j] - sum_m topk_w[t,m] g[t,m]) / temperature
+ *   dWg[e,:]    = sum over the slots (t,j) that picked e of dlogit[t,j] * x[t]          fp32 [N,d_in], overwritten
+ * Adapters nobody picked get a zero row; top-1 gives all zeros (the weight is the constant 1, App. A.1).  The
+ * cross-entropy term of the gate loss (Eq. 4) is the caller's: it needs labels this library does not see.
+ * dlogit: optional fp32 [T,k] output (may be null).  fp32 accumulation, sums in a fixed order (bit-identical
+ * from run to run).  workspace: device scratch of meteora_gate_backward_workspace_bytes(shape) bytes; it may be
+ * the forward's workspace once its routing has been copied out or is passed here as topk_idx / topk_w from a
+ * DIFFERENT buffer (the call overwrites the start of the workspace).
+ */
+size_t meteora_gate_backward_workspace_bytes(const meteora_shape_t* shape);
+int meteora_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
+                          const float* topk_w, const meteora_shape_t* shape, float* dlogit, float* dWg,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same as meteora_linear_forward with the activations in HOST memory: x_host[T,d_in] is copied to
  * the device, the layer runs, y_host[T,d_out] is copied back, all on `stream` (pinned host memory
  * makes the copies asynchronous).  Weights and workspace stay device pointers.  The call does not

@@ -24,7 +24,8 @@ STATUS = {0: "METEORA_OK", -1: "METEORA_ERR_INVALID_ARG", -2: "METEORA_ERR_UNSUP
 
 EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_lora_delta_static",
            "meteora_linear_forward", "meteora_linear_forward_group", "meteora_group_workspace_bytes",
-           "meteora_group_workspace_routing", "meteora_group_plan",
+           "meteora_group_workspace_routing", "meteora_group_plan", "meteora_gate_backward",
+           "meteora_gate_backward_workspace_bytes",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
            "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
            "meteora_describe_plan", "meteora_set_tuning", "meteora_status_string"]
@@ -64,6 +65,9 @@ def load_library() -> ctypes.CDLL:
     ip = ctypes.POINTER(ci)
     lib.meteora_linear_forward_group.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
                                                  ctypes.POINTER(vp), ip, ci, shp, ctypes.POINTER(vp), vp, sz, vp]
+    lib.meteora_gate_backward.argtypes = [vp, vp, vp, vp, vp, vp, shp, vp, vp, vp, sz, vp]
+    lib.meteora_gate_backward_workspace_bytes.argtypes = [shp]
+    lib.meteora_gate_backward_workspace_bytes.restype = sz
     lib.meteora_group_plan.argtypes = [shp, ip, ci]
     lib.meteora_group_workspace_bytes.argtypes = [shp, ip, ci]
     lib.meteora_group_workspace_bytes.restype = sz
@@ -80,7 +84,8 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_status_string.argtypes = [ci]
     lib.meteora_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("meteora_workspace_bytes", "meteora_group_workspace_bytes", "meteora_status_string"):
+        if name not in ("meteora_workspace_bytes", "meteora_group_workspace_bytes",
+                        "meteora_gate_backward_workspace_bytes", "meteora_status_string"):
             getattr(lib, name).restype = ci
     _lib = lib
     return lib
@@ -229,6 +234,29 @@ def meteora_linear_forward(x, W0, A, B, Wg, k: int, temperature: float = 1.0,
         return y
     idx, w = meteora_workspace_routing(shape, workspace)
     return y, idx, w
+
+
+def meteora_gate_backward(x, A, B, dy, topk_idx, topk_w, temperature: float = 1.0):
+    """dWg[N,d_in] (fp32) and dlogit[T,k] (fp32): gradient of the gate through Eq. 3 and Eq. 2 for the routing given."""
+    lib = load_library()
+    T, d_in = x.shape
+    N, r, _ = A.shape
+    d_out = B.shape[1]
+    k = topk_idx.shape[1]
+    shape = make_shape(T, d_in, d_out, N, r, k, x.dtype, temperature)
+    n = lib.meteora_gate_backward_workspace_bytes(ctypes.byref(shape))
+    if n == 0:
+        raise MeteoraError(-1, "meteora_gate_backward_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=x.device)
+    dWg = torch.empty((N, d_in), dtype=torch.float32, device=x.device)
+    dlogit = torch.empty((T, k), dtype=torch.float32, device=x.device)
+    _check(lib.meteora_gate_backward(_dev(x, (T, d_in), x.dtype, "x"), _dev(A, (N, r, d_in), x.dtype, "A"),
+                                     _dev(B, (N, d_out, r), x.dtype, "B"), _dev(dy, (T, d_out), x.dtype, "dy"),
+                                     _dev(topk_idx, (T, k), torch.int32, "topk_idx"),
+                                     _dev(topk_w, (T, k), torch.float32, "topk_w"), ctypes.byref(shape),
+                                     dlogit.data_ptr(), dWg.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "meteora_gate_backward")
+    return dWg, dlogit
 
 
 def meteora_group_plan(T, d_in, d_outs, N, r, k, dtype: torch.dtype) -> int:

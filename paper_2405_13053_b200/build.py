@@ -9,7 +9,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libmeteora.so")
-SOURCES = ["api.cu", "gate_topk.cu", "route.cu", "lora.cu", "gemm_simt.cu", "wgemm_tcgen05.cu", "lora_static.cu"]
+SOURCES = ["api.cu", "gate_topk.cu", "route.cu", "lora.cu", "gemm_simt.cu", "wgemm_tcgen05.cu", "lora_static.cu",
+           "gate_backward.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -291,6 +291,41 @@ int meteora_linear_forward_group(const void* x, const void* const* W0, const voi
     return METEORA_OK;
 }
 
+size_t meteora_gate_backward_workspace_bytes(const meteora_shape_t* shape) {
+    if (check_shape(shape, true, true) != METEORA_OK) return 0;
+    const size_t S = (size_t)shape->T * shape->k;
+    return kHeaderBytes + 3 * align_up(S * 4, 256) + 2 * align_up(((size_t)shape->N + 1) * 4, 256);
+}
+
+int meteora_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
+                          const float* topk_w, const meteora_shape_t* shape, float* dlogit, float* dWg,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (!dWg || !workspace) return METEORA_ERR_INVALID_ARG;
+    if (shape->T > 0 && (!x || !A || !B || !dy || !topk_idx || !topk_w)) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(A) || !aligned16(B) || !aligned16(dy) || !aligned16(workspace))
+        return METEORA_ERR_MISALIGNED;
+    if (workspace_bytes < meteora_gate_backward_workspace_bytes(shape)) return METEORA_ERR_WORKSPACE_TOO_SMALL;
+    const size_t S = (size_t)shape->T * shape->k;
+    uint8_t* p = (uint8_t*)workspace + kHeaderBytes;
+    float* g = (float*)p;
+    p += align_up(S * 4, 256);
+    float* dl = (float*)p;
+    p += align_up(S * 4, 256);
+    int32_t* perm = (int32_t*)p;
+    p += align_up(S * 4, 256);
+    int32_t* counts = (int32_t*)p;
+    p += align_up(((size_t)shape->N + 1) * 4, 256);
+    int32_t* offsets = (int32_t*)p;
+    cudaStream_t st = (cudaStream_t)stream;
+    rc = launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, g, dl, counts, offsets, perm, dWg, st);
+    if (rc != METEORA_OK) return rc;
+    if (dlogit && S > 0)
+        return cuda_status(cudaMemcpyAsync(dlogit, dl, S * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    return METEORA_OK;
+}
+
 int meteora_linear_forward_host(const void* x_host, const void* W0, const void* A, const void* B,
                                 const void* Wg, const meteora_shape_t* shape, void* y_host, void* workspace,
                                 size_t workspace_bytes, void* stream) {
