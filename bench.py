@@ -618,6 +618,47 @@ def run_layer_sweep():
         del mods, graph, groups
 
 
+def run_gate_backward_sweep():
+    """meteora_gate_backward (gradient of the gate weights for a forward's routing) at the q_proj shape."""
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+
+    hbm, _ = measured_peaks()
+    dt, es = torch.bfloat16, 2
+    d_in = d_out = 4096
+    for T in (128, 2048, 8192):
+        g = torch.Generator(device="cuda").manual_seed(13)
+        x = torch.randn(T, d_in, device="cuda", generator=g).to(dt)
+        W0 = (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt)
+        A = ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt)
+        B = (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt)
+        Wg = (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt)
+        dy = torch.randn(T, d_out, device="cuda", generator=g).to(dt)
+        _, idx, w = mb.meteora_linear_forward(x, W0, A, B, Wg, TOPK, return_routing=True)
+        idx, w = idx.clone(), w.clone()
+        for _ in range(3):
+            mb.meteora_gate_backward(x, A, B, dy, idx, w)
+        torch.cuda.synchronize()
+        iters = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            mb.meteora_gate_backward(x, A, B, dy, idx, w)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / iters
+        touched = int(torch.unique(idx).numel())
+        # x is read for the shrink and again, once per pick, for the reduction over tokens; dy once; dWg written in fp32
+        nbytes = ((1 + TOPK) * T * d_in + T * d_out + touched * RANK * (d_in + d_out)) * es + N_ADAPTERS * d_in * 4
+        print(json.dumps({"op": "meteora_gate_backward", "shape": "4096->4096", "T": T, "us_per_call": round(us, 2),
+                          "tokens_per_s": round(T / us * 1e6), "bound": "hbm",
+                          "roofline_us": round(nbytes / hbm / 1e3, 2),
+                          "frac_of_roofline": round(nbytes / hbm / 1e3 / us, 3),
+                          "note": "4 launches (slot gradients, dlogit, bucketing, reduction over tokens); stream timing"}),
+              flush=True)
+
+
 def run_variants():
     """The paper's synthetic sweep axes (App. A.7: k, r, number of adapters; temperature of App. A.5) at the
     LLaMA3-8B q_proj shape, a decode batch (T = 32) and a prefill batch (T = 2048), one axis at a time around
@@ -712,6 +753,7 @@ def main():
     elif args.sweep:
         run_sweep(args)
         run_layer_sweep()
+        run_gate_backward_sweep()
     elif args.impl == "reference":
         run_reference(args)
     else:
