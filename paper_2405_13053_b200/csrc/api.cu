@@ -293,8 +293,10 @@ int meteora_linear_forward_group(const void* x, const void* const* W0, const voi
 
 size_t meteora_gate_backward_workspace_bytes(const meteora_shape_t* shape) {
     if (check_shape(shape, true, true) != METEORA_OK) return 0;
-    const size_t S = (size_t)shape->T * shape->k;
-    return kHeaderBytes + 3 * align_up(S * 4, 256) + 2 * align_up(((size_t)shape->N + 1) * 4, 256);
+    const size_t S = (size_t)shape->T * shape->k, r = (size_t)shape->r;
+    return kHeaderBytes + 2 * align_up(S * 4, 256) + 2 * align_up(S * r * 4, 256) +
+           2 * align_up(((size_t)shape->N + 1) * 4, 256) +
+           align_up((size_t)shape->N * shape->d_out * r * elem_size(shape->dtype), 256);
 }
 
 int meteora_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
@@ -307,19 +309,22 @@ int meteora_gate_backward(const void* x, const void* A, const void* B, const voi
     if (!aligned16(x) || !aligned16(A) || !aligned16(B) || !aligned16(dy) || !aligned16(workspace))
         return METEORA_ERR_MISALIGNED;
     if (workspace_bytes < meteora_gate_backward_workspace_bytes(shape)) return METEORA_ERR_WORKSPACE_TOO_SMALL;
-    const size_t S = (size_t)shape->T * shape->k;
+    const size_t S = (size_t)shape->T * shape->k, r = (size_t)shape->r;
     uint8_t* p = (uint8_t*)workspace + kHeaderBytes;
-    float* g = (float*)p;
-    p += align_up(S * 4, 256);
-    float* dl = (float*)p;
-    p += align_up(S * 4, 256);
-    int32_t* perm = (int32_t*)p;
-    p += align_up(S * 4, 256);
-    int32_t* counts = (int32_t*)p;
-    p += align_up(((size_t)shape->N + 1) * 4, 256);
-    int32_t* offsets = (int32_t*)p;
+    auto take = [&](size_t bytes) {
+        uint8_t* q = p;
+        p += align_up(bytes, 256);
+        return q;
+    };
+    float* dl = (float*)take(S * 4);
+    int32_t* perm = (int32_t*)take(S * 4);
+    float* u = (float*)take(S * r * 4);
+    float* z = (float*)take(S * r * 4);
+    int32_t* counts = (int32_t*)take(((size_t)shape->N + 1) * 4);
+    int32_t* offsets = (int32_t*)take(((size_t)shape->N + 1) * 4);
+    void* Bt = take((size_t)shape->N * shape->d_out * r * elem_size(shape->dtype));
     cudaStream_t st = (cudaStream_t)stream;
-    rc = launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, g, dl, counts, offsets, perm, dWg, st);
+    rc = launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, Bt, u, z, dl, counts, offsets, perm, dWg, st);
     if (rc != METEORA_OK) return rc;
     if (dlogit && S > 0)
         return cuda_status(cudaMemcpyAsync(dlogit, dl, S * sizeof(float), cudaMemcpyDeviceToDevice, st));

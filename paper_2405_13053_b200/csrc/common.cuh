@@ -59,8 +59,8 @@ int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int
                                int32_t* topk_idx, float* topk_w, float* uw, bool pdl, cudaStream_t st);
 // route.cu
 int launch_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
-                         const float* topk_w, const meteora_shape_t& s, float* g, float* dlogit, int32_t* counts,
-                         int32_t* offsets, int32_t* perm, float* dWg, cudaStream_t st);
+                         const float* topk_w, const meteora_shape_t& s, void* Bt, float* u, float* z, float* dlogit,
+                         int32_t* counts, int32_t* offsets, int32_t* perm, float* dWg, cudaStream_t st);
 int launch_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets, int32_t* perm,
                  cudaStream_t st);
 // lora.cu
