@@ -46,21 +46,48 @@ __global__ void k_gate_dlogit(const float* __restrict__ u, const float* __restri
     for (int j = 0; j < k; ++j) dlogit[(size_t)t * k + j] = topk_w[(size_t)t * k + j] * (g[j] - mean) * inv_tau;
 }
 
-// dWg[e, d] = sum over the adapter's bucket, in permutation order, of dlogit[slot] * x[token(slot), d].
+// dWg[e, d] = sum over the adapter's bucket of dlogit[slot] * x[token(slot), d].  A CTA owns 256 columns of one
+// adapter: warp w adds the bucket's entries w, w + 8, w + 16, ... in that order (8 columns per lane, 128-bit
+// loads when the row pitch allows), and the eight partial sums of a column are added in warp order: a fixed
+// order whatever the scheduling.
 template <typename TI>
 __global__ void __launch_bounds__(256)
 k_gate_dwg(const TI* __restrict__ x, const float* __restrict__ dlogit, const int32_t* __restrict__ offsets,
            const int32_t* __restrict__ perm, int d_in, int k, float* __restrict__ dWg) {
+    __shared__ float part[8][256];
     const int e = blockIdx.x;
-    const int d = blockIdx.y * 256 + threadIdx.x;
-    if (d >= d_in) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int d0 = blockIdx.y * 256 + lane * 8;
     const int p0 = offsets[e], p1 = offsets[e + 1];
-    float acc = 0.f;
-    for (int p = p0; p < p1; ++p) {
+    const bool vec = (d_in % 8) == 0;
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int p = p0 + warp; p < p1; p += 8) {
         const int s = perm[p];
-        acc = fmaf(dlogit[s], to_f32(x[(size_t)(s / k) * d_in + d]), acc);
+        const float dl = dlogit[s];
+        const TI* row = x + (size_t)(s / k) * d_in + d0;
+        if (vec && d0 + 8 <= d_in) {
+            float xv[8];
+            load8(row, xv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = fmaf(dl, xv[i], acc[i]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (d0 + i < d_in) acc[i] = fmaf(dl, to_f32(row[i]), acc[i]);
+        }
     }
-    dWg[(size_t)e * d_in + d] = acc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) part[warp][lane * 8 + i] = acc[i];
+    __syncthreads();
+    const int d = blockIdx.y * 256 + threadIdx.x;
+    if (d < d_in) {
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) sum += part[w][threadIdx.x];
+        dWg[(size_t)e * d_in + d] = sum;
+    }
 }
 
 int launch_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
