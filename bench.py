@@ -655,7 +655,7 @@ def run_gate_backward_sweep():
                           "tokens_per_s": round(T / us * 1e6), "bound": "hbm",
                           "roofline_us": round(nbytes / hbm / 1e3, 2),
                           "frac_of_roofline": round(nbytes / hbm / 1e3 / us, 3),
-                          "note": "4 launches (slot gradients, dlogit, bucketing, reduction over tokens); stream timing"}),
+                          "note": "7 launches (bucketing, transpose of B, two grouped shrinks, dlogit, reduction over tokens, copy); stream timing through the Python binding"}),
               flush=True)
 
 
