@@ -89,16 +89,32 @@ k_shrink_segments(const TI* __restrict__ x, const TI* __restrict__ A, const int3
                 if (slot[i] < 0) continue;
                 const TI* xt = x + (size_t)(slot[i] / k) * d_in + d0;
                 if (vec) {
-                    for (int d = lane * 8; d < len; d += 256) {
-                        float xv[8];
-                        load8(xt + d, xv);
+                    // all of the slot's x values of this chunk first (one round trip to memory instead of one
+                    // per 256 columns), then the products against the staged rows
+                    constexpr int NV = DC / 256;
+                    float xv[NV][8];
 #pragma unroll
-                        for (int q = 0; q < kSegRows; ++q) {
-                            if (q < rows) {
-                                float av[8];
-                                load8(&sA[q][d], av);
+                    for (int v = 0; v < NV; ++v) {
+                        const int d = lane * 8 + v * 256;
+                        if (d < len) {
+                            load8(xt + d, xv[v]);
+                        } else {
 #pragma unroll
-                                for (int c = 0; c < 8; ++c) acc[i][q] = fmaf(av[c], xv[c], acc[i][q]);
+                            for (int c = 0; c < 8; ++c) xv[v][c] = 0.f;
+                        }
+                    }
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        const int d = lane * 8 + v * 256;
+                        if (d < len) {
+#pragma unroll
+                            for (int q = 0; q < kSegRows; ++q) {
+                                if (q < rows) {
+                                    float av[8];
+                                    load8(&sA[q][d], av);
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c) acc[i][q] = fmaf(av[c], xv[v][c], acc[i][q]);
+                                }
                             }
                         }
                     }
