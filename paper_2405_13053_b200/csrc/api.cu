@@ -34,11 +34,11 @@ Workspace carve_workspace(const meteora_shape_t& s_in, void* base) {
     ws.topk_w = (float*)take(T * s.k * sizeof(float));
     ws.uw = (float*)take(T * s.k * s.r * sizeof(float));
     ws.u_all = (float*)take(T * ws.ld_u * sizeof(float) * (size_t)stacked_zsplits_bound(s.T));   // one copy per slice of the contraction axis
-    // decode kernel scratch: two partial tiles of 128 x BN fp32 per main CTA, at most 148 main CTAs, at most
-    // 14 per row tile
+    // decode kernel scratch: one partial tile of 128 x BN fp32 per (main CTA, row tile it touches), in slot
+    // row tile + main CTA: fewer than row tiles + 148 slots
     const size_t row_tiles = ((size_t)s.d_out + 127) / 128;
     const size_t bn = (T + 15) / 16 * 16;
-    const size_t part_tiles = s.T <= 256 ? (row_tiles * 28 < 296 ? row_tiles * 28 : 296) : 0;
+    const size_t part_tiles = s.T <= 256 ? row_tiles + 148 : 0;
     ws.part_g = (float*)take(part_tiles * bn * 128 * sizeof(float));
     ws.x_dev = take(T * s.d_in * es);
     ws.y_dev = take(T * s.d_out * es);
@@ -154,7 +154,7 @@ static GroupWorkspace carve_group(const meteora_shape_t& s, const int* d_outs, i
         tiles += ((size_t)d_outs[m] + 127) / 128;
     }
     const size_t bn = ((size_t)s.T + 15) / 16 * 16;
-    const size_t part_tiles = s.T <= 256 ? std::min<size_t>(tiles * 28, 296) : 0;
+    const size_t part_tiles = s.T <= 256 ? tiles + 148 : 0;
     gw.part_g = (float*)(p ? p + off : nullptr);
     off += align_up(part_tiles * bn * 128 * sizeof(float), 256);
     gw.bytes = off;

@@ -22,6 +22,7 @@
 
 namespace meteora {
 
+constexpr int kMaxSeg = 4;     // row tiles a main CTA's unit range may touch (one TMEM accumulator each)
 constexpr int kMaxGroup = kMaxGroupModules;   // modules one launch can serve (they share x: q/k/v, gate/up)
 
 // What differs between the modules of a group: weights come through the tensor maps, the rest is here.
@@ -58,9 +59,10 @@ struct DecodeParams {
     float inv_tau;
     int hold;              // main CTAs start loading only after the aux CTAs have issued their first loads
     int32_t* ctr;          // [0] aux partials written, [1] selections published, [2] CTAs exited, [3] aux loads issued
-    float* part_g;         // [main CTA][segment 0/1][BN][128] fp32 partial accumulator tiles of the base product
+    float* part_g;         // [row tile + main CTA][BN][128] fp32 partial accumulator tiles of the base product
     int32_t* tile_ctr;     // [row tiles] partials delivered per tile
     int row_tiles;         // of all modules together
+    int slab_rows;         // rows of B (of every adapter) the staging buffer of a main CTA holds
     int trace_call;        // trace builds: which record of the trace buffer this launch fills
 };
 
@@ -235,14 +237,11 @@ __device__ __forceinline__ void finish_tile(__nv_bfloat16* y, int d_out, int k, 
                                             size_t part_stride, int units, int M, int upt, int tile, int first_cta, int c,
                                             int q0, int nq, int ntok, const uint4* slab, const float* s_uw,
                                             const int* s_idx, int etid, int nthr, bool& routing_pending) {
-    // partial of contributor q: CTA first_cta + q, its segment 0 if its range starts in this tile, else 1
+    // The partial of main CTA i for row tile t sits in slot t + i: unit ranges are ordered, so no two (CTA, tile)
+    // pairs share a slot, and at most row tiles + main CTAs slots are in use.
     const float* parts[C];
 #pragma unroll
-    for (int q = 0; q < C; ++q) {
-        const int cta = first_cta + min(q, c - 1);
-        const int seg = (int)((unsigned)units * (unsigned)cta / (unsigned)M) / upt == tile ? 0 : 1;
-        parts[q] = part_g + ((size_t)cta * 2 + seg) * part_stride;
-    }
+    for (int q = 0; q < C; ++q) parts[q] = part_g + (size_t)(tile + first_cta + min(q, c - 1)) * part_stride;
     finish_rows<C, U>(y, d_out, k, cpa, parts, c, tile_row0, q0, nq, ntok, slab, s_uw, s_idx, etid, nthr, routing_pending);
 }
 
@@ -339,7 +338,7 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
     const uint32_t stage_bytes = p.kc * (kWTileBytes + x_tile_bytes);
     const uint32_t ring_bytes = p.stages * stage_bytes;
     const uint32_t bar_base = ring + ring_bytes;
-    const int nbar = 2 * d.bar_stages + 3;           // sized for the deeper of the two rings
+    const int nbar = 2 * d.bar_stages + kMaxSeg + 1;  // full / empty for the deeper of the two rings, one per segment
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ring_ptr + ring_bytes + nbar * 8);
     uint8_t* epi = ring_ptr + ring_bytes + p.epi_off;
 
@@ -468,10 +467,9 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
         const int u1 = (int)(U * (unsigned)(main_id + 1) / (unsigned)M);
         const int n_it = u1 - u0;
         const int tile_a = u0 / upt, tile_b = (u1 - 1) / upt;
-        const int nseg = tile_b - tile_a + 1;                                        // 1 or 2
-        const int it_switch = nseg > 1 ? (tile_a + 1) * upt - u0 : n_it;             // iterations of segment 0
+        const int nseg = tile_b - tile_a + 1;                                        // 1 .. kMaxSeg (host-checked)
         const RingGeom geom = {ring, bar_base, x_tile_bytes, stage_bytes, p.stages, p.kc, p.maps3d};
-        const uint32_t bar_acc = bar_base + 2 * p.stages * 8;                        // [0], [1]: one per segment
+        const uint32_t bar_acc = bar_base + 2 * p.stages * 8;                        // [0 .. kMaxSeg): one per segment
         const size_t part_stride = (size_t)p.BN * kBM;                               // floats per partial tile
         if (warp == 0) {
             if (lane == 0) {
@@ -527,15 +525,16 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             }
         } else if (warp == 1) {
             if (lane == 0) {
-                bool ok = true, seg0_done = false;
+                bool ok = true;
+                int committed = 0;                                                  // segments announced so far
                 for (int it = 0; it < n_it; ++it) {
                     const int st = it % geom.stages, round = it / geom.stages;
                     ok = mbar_wait(bar_base + st * 8, round & 1);
                     if (!ok) break;
                     tc_fence_after();
-                    const bool second = it >= it_switch;
-                    const bool fresh = it == 0 || it == it_switch;                  // first MMA of a segment overwrites
-                    const uint32_t acc = tmem_base + (second ? (uint32_t)p.BN : 0u);
+                    const int unit = u0 + it, sg = unit / upt - tile_a;
+                    const bool fresh = it == 0 || unit % upt == 0;                  // first MMA of a segment overwrites
+                    const uint32_t acc = tmem_base + (uint32_t)(sg * p.BN);
                     const uint32_t wa = ring + st * stage_bytes, xa = wa + p.kc * kWTileBytes;
                     for (int c = 0; c < p.kc; ++c) {
                         const uint64_t da = smem_desc_sw128(wa + c * kWTileBytes);
@@ -545,23 +544,24 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                             umma_bf16(acc, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, !fresh || (c | kk) != 0);
                     }
                     umma_commit(bar_base + (geom.stages + st) * 8);
-                    if (it == it_switch - 1) {                                      // segment 0 complete
-                        umma_commit(bar_acc);
-                        seg0_done = true;
+                    if (it + 1 == n_it || (unit + 1) % upt == 0) {                  // the segment is complete
+                        umma_commit(bar_acc + 8 * sg);
+                        committed = sg + 1;
                     }
                 }
                 if (tr_main) FUSED_STAMP(p, 32, 2);
-                if (!seg0_done) umma_commit(bar_acc);                               // only after a failed wait
-                if (nseg > 1) umma_commit(bar_acc + 8);
+                for (int sg = committed; sg < nseg; ++sg) umma_commit(bar_acc + 8 * sg);   // only after a failed wait
                 if (!ok) flag_error(p, 2, 200);
             }
         } else {
             // Which rows of which tile this CTA finishes: tile `t` is shared by the CTAs owner(first unit) ..
             // owner(last unit), in that order; contributor j of c takes the groups of 4 rows [32j/c, 32(j+1)/c).
-            int d_tile[2], d_first[2], d_c[2], d_q0[2], d_nq[2], d_mod[2], d_row0[2];
+            int d_tile[kMaxSeg], d_first[kMaxSeg], d_c[kMaxSeg], d_q0[kMaxSeg], d_nq[kMaxSeg], d_mod[kMaxSeg],
+                d_row0[kMaxSeg];
+            bool side_by_side = nseg <= 2;         // else the tiles are finished one after the other, B rows staged each time
             const int cpa = p.r >> 3;                                        // 16-byte words per B row
             uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
-            uint4* d_slab[2];
+            uint4* d_slab[kMaxSeg];
             int slab_words = 0;
             for (int sg = 0; sg < nseg; ++sg) {
                 const int tile = tile_a + sg;
@@ -577,10 +577,16 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 d_slab[sg] = slab + slab_words;
                 d_mod[sg] = module_of_tile(d.mod, d.n_mod, tile);
                 d_row0[sg] = (tile - d.mod[d_mod[sg]].tile0) * kBM;          // the tile's first row inside its module
-                // B rows of that slice for every adapter: no routing needed yet
-                stage_slab_rows(d.mod[d_mod[sg]].B, d.mod[d_mod[sg]].d_out, p.N, cpa, d_slab[sg],
-                                d_row0[sg] + 4 * d_q0[sg], 4 * d_nq[sg], etid);
                 slab_words += p.N * cpa * 4 * d_nq[sg];
+            }
+            // side by side only if both tiles' rows fit the staging buffer together (a range longer than a
+            // tile's units can own one tile entirely and share another)
+            if (slab_words > p.N * cpa * d.slab_rows) side_by_side = false;
+            if (side_by_side) {
+                // B rows of the CTA's slices for every adapter: no routing needed yet
+                for (int sg = 0; sg < nseg; ++sg)
+                    stage_slab_rows(d.mod[d_mod[sg]].B, d.mod[d_mod[sg]].d_out, p.N, cpa, d_slab[sg],
+                                    d_row0[sg] + 4 * d_q0[sg], 4 * d_nq[sg], etid);
             }
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 3);
             // Accumulators out of TMEM to the fp32 scratch, segment by segment (lane = row, a warp writes 128
@@ -592,7 +598,7 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
                 tc_fence_after();
                 if (etid == 0 && tr_main && sg == nseg - 1) FUSED_STAMP(p, 32, 5);
-                float* part = d.part_g + ((size_t)main_id * 2 + sg) * part_stride;
+                float* part = d.part_g + (size_t)(d_tile[sg] + main_id) * part_stride;
                 for (int c = c_begin; c < c_end; c += 16) {
                     float v[16];
                     if (acc_ok) {
@@ -613,7 +619,7 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             }
             // Two tiles to finish: half of the epilogue threads each, side by side (one round trip to L2 for both).
             bool routing_pending = true;
-            {
+            if (side_by_side) {
                 const int nthr = nseg > 1 ? kEpiThreads / 2 : kEpiThreads;
                 const int sg = nseg > 1 ? etid / nthr : 0, gtid = etid - sg * nthr;
                 if (gtid == 0) {
@@ -635,6 +641,32 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                     finish_tile<8, 2>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
                 else
                     finish_tile<16, 1>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, d_slab[sg], s_uw, s_idx, gtid, nthr, routing_pending);
+            } else {
+                // More than two tiles (a range longer than a tile's units): one after the other with all epilogue
+                // threads, the single staging buffer refilled with each tile's B rows.
+                for (int sg = 0; sg < nseg; ++sg) {
+                    const DecodeModule& mo = d.mod[d_mod[sg]];
+                    epi_barrier();                                                   // the buffer's previous readers are done
+                    stage_slab_rows(mo.B, mo.d_out, p.N, cpa, slab, d_row0[sg] + 4 * d_q0[sg], 4 * d_nq[sg], etid);
+                    if (etid == 0) {
+                        if (!wait_counter(d.tile_ctr + d_tile[sg], d_c[sg])) flag_error(p, 4, 900);
+                        if (tr_main && sg == nseg - 1) FUSED_STAMP(p, 32, 6);
+                    }
+                    epi_barrier();
+                    const int c = d_c[sg];
+                    const float* s_uw = reinterpret_cast<const float*>(epi + p.uw_off) + sg * p.BN * p.k * p.r;
+                    const int* s_idx = reinterpret_cast<const int*>(epi + p.idx_off) + sg * p.BN * p.k;
+                    if (c <= 1)
+                        finish_tile<1, 4>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, slab, s_uw, s_idx, etid, kEpiThreads, routing_pending);
+                    else if (c <= 2)
+                        finish_tile<2, 4>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, slab, s_uw, s_idx, etid, kEpiThreads, routing_pending);
+                    else if (c <= 4)
+                        finish_tile<4, 4>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, slab, s_uw, s_idx, etid, kEpiThreads, routing_pending);
+                    else if (c <= 8)
+                        finish_tile<8, 2>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, slab, s_uw, s_idx, etid, kEpiThreads, routing_pending);
+                    else
+                        finish_tile<16, 1>(mo.y, mo.d_out, p.k, cpa, d_row0[sg], d.part_g, part_stride, d.units, M, upt, d_tile[sg], d_first[sg], c, d_q0[sg], d_nq[sg], ntok, slab, s_uw, s_idx, etid, kEpiThreads, routing_pending);
+                }
             }
             if (routing_pending) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
             if (etid == 0 && tr_main) FUSED_STAMP(p, 32, 10);

@@ -1289,7 +1289,7 @@ struct FusedPlan {
     bool ok;
     int why;   // why not: 1 knob/shape, 2 more row tiles than main CTAs, 4 residency, 5 shared memory
     Plan main; // BN, stages, kc, maps3d, tmem_cols, staging offsets, smem of the decode kernel
-    int row_tiles, n_main, upt, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages;
+    int row_tiles, n_main, upt, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages, slab_rows;
     size_t w0_bytes;
 };
 
@@ -1343,8 +1343,8 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     fp.gate_row0 = merged ? tail_rows : 0;
     fp.why = 2;
     const int group_tiles = G * fp.aux_tiles;                    // every module has its own stacked shrink
-    if (group_tiles + fp.row_tiles > sms) return fp;
-    const int aux_budget = std::min(std::max(std::max(20, 4 * group_tiles), group_tiles), sms - fp.row_tiles);
+    if (group_tiles + 8 > sms) return fp;
+    const int aux_budget = std::min(std::max(std::max(20, 4 * group_tiles), group_tiles), sms - 8);
     fp.aux_slices = std::min(std::min(aux_budget / group_tiles, ksteps), 16);   // 16: the selection reads all slices at once
     if (fp.aux_slices < 1) return fp;
     fp.n_aux = group_tiles * fp.aux_slices;
@@ -1353,6 +1353,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     // every CTA inside one tile (one accumulator, one finishing duty); it is taken unless it idles more than a
     // tenth of the CTAs an uneven split would use (6 per tile keep any tile within 8 unit ranges).
     const int m_max = sms - fp.n_aux;
+    if (m_max < 1) return fp;
     const int m_even = fp.row_tiles * std::min(8, m_max / fp.row_tiles);
     int n_main = std::min(m_max, 6 * fp.row_tiles);
     // (large batches exchange 64 KB and more per partial tile: there even 80 % of the CTAs are the better deal)
@@ -1362,7 +1363,12 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     if (m_even > 0 && n_main % fp.row_tiles != 0 && (size_t)s.N * kBM * s.r * 2 > 64 * 1024) n_main = m_even;
     if (tn.splits > 0 && tn.splits * fp.row_tiles <= m_max) n_main = std::min(tn.splits, 8) * fp.row_tiles;
     n_main = (int)std::min<long long>(n_main, units);
-    if (n_main < fp.row_tiles || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
+    if (n_main < 1 || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
+    // Row tiles a CTA's unit range can touch: 1 for whole tiles per CTA group, 2 while a range is no longer than a
+    // tile's units, more beyond that (one TMEM accumulator of BN columns each: at most 4, and 512 columns in all).
+    const long long range = (units + n_main - 1) / n_main;
+    const int segs = n_main % fp.row_tiles == 0 ? 1 : (int)std::max<long long>(2, (range - 2) / fp.upt + 2);
+    if (segs > kMaxSeg || segs * pl.BN > 512) return fp;
     fp.n_main = n_main;
     // shared memory: staged B rows (at most 128 rows of every adapter), routing, barriers, ring
     fp.why = 5;
@@ -1371,11 +1377,12 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     const bool whole = n_main % fp.row_tiles == 0;
     const int own_rows = whole ? 4 * ((32 + n_main / fp.row_tiles - 1) / (n_main / fp.row_tiles)) : kBM;
     // the routing once per tile a CTA finishes rows of (one tile, or two that may belong to two modules)
-    const int duties = whole ? 1 : 2;
+    const int duties = segs;
+    fp.slab_rows = own_rows;
     pl.uw_off = (int)align_up((size_t)s.N * own_rows * s.r * 2, 16);
     pl.idx_off = pl.uw_off + duties * pl.BN * s.k * s.r * 4;
     const size_t epi_bytes = (size_t)pl.idx_off + (size_t)duties * pl.BN * s.k * 4;
-    pl.epi_off = (int)align_up((size_t)(2 * 16 + 3) * 8 + 16, 128);
+    pl.epi_off = (int)align_up((size_t)(2 * 16 + kMaxSeg + 1) * 8 + 16, 128);
     const size_t fixed = 1024 + pl.epi_off + epi_bytes;
     if (fixed + 48 * 1024 > 226 * 1024) return fp;
     const size_t chunk = kWTileBytes + (size_t)pl.BN * 128;      // one k-step of both operands
@@ -1390,7 +1397,7 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     int col_logits = 0;
     if (ring_bytes < (size_t)(kThreads / 32) * tc_stacked_pitch(s, &col_logits) * sizeof(float)) return fp;
     int cols = 32;
-    while (cols < 2 * pl.BN) cols *= 2;                           // two accumulators: one per segment of a unit range
+    while (cols < std::max(2, segs) * pl.BN) cols *= 2;           // one accumulator per row tile a unit range can touch
     pl.tmem_cols = cols;
     pl.smem = 1024 + ring_bytes + pl.epi_off + epi_bytes;
     const int nks_aux = (ksteps + fp.aux_slices - 1) / fp.aux_slices;
@@ -1499,6 +1506,7 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
     d.part_g = part_g;
     d.tile_ctr = tile_ctr;
     d.row_tiles = fp.row_tiles;
+    d.slab_rows = fp.slab_rows;
     if (pl.smem > 227 * 1024) return METEORA_ERR_UNSUPPORTED_SHAPE;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(fp.n_main + fp.n_aux);

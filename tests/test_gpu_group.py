@@ -52,6 +52,7 @@ def check_group(ws, y_tol):
 @pytest.mark.parametrize("d_in,d_outs,T", [
     (1024, (640, 256, 384), 1), (1024, (640, 256, 384), 37), (1024, (640, 256, 384), 128),
     (1536, (1000, 128), 200), (512, (256, 256, 128, 384), 16), (1096, (384, 640), 64), (1024, (2304, 768), 256),
+    (256, (14336, 14336), 64),                   # gate/up of LLaMA3-8B: 224 row tiles on 128 CTAs, three tiles per CTA
 ])
 def test_group_of_decode_modules_matches_oracle(d_in, d_outs, T):
     ws = make_group(T, d_in, d_outs, seed=6000 + T)

@@ -253,11 +253,13 @@ def test_split_k_cluster_sizes_agree_with_oracle(splits, stages):
 # (d_in, d_out) chosen so that the unit ranges of the main CTAs fall every way they can: many CTAs per row tile
 # (640), a ragged last tile (1000), a contraction length that is no multiple of 64 (1096: plain 2-D tensor
 # maps, one k-step per stage), ranges that straddle two tiles (4224 = 33 tiles over 128 CTAs), more tiles than
-# half the CTAs (9000 = 71 tiles) and, with the "splits" knob capping the CTAs per tile, one CTA per tile.
+# half the CTAs (9000 = 71 tiles), with the "splits" knob capping the CTAs per tile, one CTA per tile, and layers
+# with several row tiles per CTA (40000 and 60000 rows: 313 and 469 tiles on 128 CTAs).
 @pytest.mark.parametrize("d_in,d_out,T,per_tile", [
     (1024, 640, 1, 0), (1024, 640, 8, 0), (1024, 640, 100, 0), (1024, 640, 256, 0),
     (1536, 1000, 37, 0), (1096, 768, 16, 0), (2048, 4224, 5, 0), (2048, 4224, 128, 0),
     (512, 9000, 24, 0), (1024, 1280, 64, 1), (1024, 1280, 200, 3),
+    (128, 40000, 4, 0), (128, 60000, 70, 0),     # more row tiles than CTAs: unit ranges over three and four tiles
 ])
 def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
     # one kernel per call: base product + stacked shrink + selection + LoRA expand
