@@ -478,12 +478,12 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 if (tr_main) FUSED_STAMP(p, 32, 1);
                 int cur_tile = -1, row0 = 0;
                 const CUtensorMap* tmW0 = &maps.W0[0];
+                int tile = tile_a, kpos = u0 - tile_a * upt, st = 0, round = 0;
                 for (int it = 0; it < n_it && ok; ++it) {
-                    const int st = it % geom.stages, round = it / geom.stages;
                     if (round > 0) ok = mbar_wait(bar_base + (geom.stages + st) * 8, (round & 1) ^ 1);
                     if (!ok) break;
                     const uint32_t full = bar_base + st * 8, dst = ring + st * stage_bytes;
-                    const int unit = u0 + it, tile = unit / upt, kstep = (unit - tile * upt) * p.kc;
+                    const int kstep = kpos * p.kc;
                     if (tile != cur_tile) {                      // rows of which module's W0
                         const int wm = module_of_tile(d.mod, d.n_mod, tile);
                         cur_tile = tile;
@@ -497,6 +497,14 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                     } else {
                         tma_load_2d(dst, tmW0, kstep * kBK, row0, full);
                         tma_load_2d(dst + kWTileBytes, &tmX, kstep * kBK, 0, full);
+                    }
+                    if (++kpos == upt) {
+                        kpos = 0;
+                        ++tile;
+                    }
+                    if (++st == geom.stages) {
+                        st = 0;
+                        ++round;
                     }
                 }
                 if (!ok) flag_error(p, 1, 100);
@@ -527,13 +535,12 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             if (lane == 0) {
                 bool ok = true;
                 int committed = 0;                                                  // segments announced so far
+                int sg = 0, kpos = u0 - tile_a * upt, st = 0, round = 0;            // no divisions in this loop: it paces the tensor cores
                 for (int it = 0; it < n_it; ++it) {
-                    const int st = it % geom.stages, round = it / geom.stages;
                     ok = mbar_wait(bar_base + st * 8, round & 1);
                     if (!ok) break;
                     tc_fence_after();
-                    const int unit = u0 + it, sg = unit / upt - tile_a;
-                    const bool fresh = it == 0 || unit % upt == 0;                  // first MMA of a segment overwrites
+                    const bool fresh = it == 0 || kpos == 0;                        // first MMA of a segment overwrites
                     const uint32_t acc = tmem_base + (uint32_t)(sg * p.BN);
                     const uint32_t wa = ring + st * stage_bytes, xa = wa + p.kc * kWTileBytes;
                     for (int c = 0; c < p.kc; ++c) {
@@ -544,9 +551,18 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                             umma_bf16(acc, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, !fresh || (c | kk) != 0);
                     }
                     umma_commit(bar_base + (geom.stages + st) * 8);
-                    if (it + 1 == n_it || (unit + 1) % upt == 0) {                  // the segment is complete
+                    ++kpos;
+                    if (it + 1 == n_it || kpos == upt) {                            // the segment is complete
                         umma_commit(bar_acc + 8 * sg);
                         committed = sg + 1;
+                    }
+                    if (kpos == upt) {
+                        kpos = 0;
+                        ++sg;
+                    }
+                    if (++st == geom.stages) {
+                        st = 0;
+                        ++round;
                     }
                 }
                 if (tr_main) FUSED_STAMP(p, 32, 2);
