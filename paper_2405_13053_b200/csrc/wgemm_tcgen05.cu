@@ -1289,7 +1289,7 @@ struct FusedPlan {
     bool ok;
     int why;   // why not: 1 knob/shape, 2 more row tiles than main CTAs, 4 residency, 5 shared memory
     Plan main; // BN, stages, kc, maps3d, tmem_cols, staging offsets, smem of the decode kernel
-    int row_tiles, n_main, upt, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages, slab_rows;
+    int row_tiles, n_main, upt, n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices, aux_stages, slab_rows, segs;
     size_t w0_bytes;
 };
 
@@ -1369,6 +1369,10 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     const long long range = (units + n_main - 1) / n_main;
     const int segs = n_main % fp.row_tiles == 0 ? 1 : (int)std::max<long long>(2, (range - 2) / fp.upt + 2);
     if (segs > kMaxSeg || segs * pl.BN > 512) return fp;
+    // Measured (gate/up of LLaMA3-8B, 224 row tiles, T = 64): a group whose CTAs finish three tiles one after the
+    // other takes 83 us in one launch against 2 x 36 us as two calls, so groups stay within two tiles per CTA.
+    if (G > 1 && segs > 2) return fp;
+    fp.segs = segs;
     fp.n_main = n_main;
     // shared memory: staged B rows (at most 128 rows of every adapter), routing, barriers, ring
     fp.why = 5;

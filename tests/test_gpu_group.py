@@ -52,7 +52,6 @@ def check_group(ws, y_tol):
 @pytest.mark.parametrize("d_in,d_outs,T", [
     (1024, (640, 256, 384), 1), (1024, (640, 256, 384), 37), (1024, (640, 256, 384), 128),
     (1536, (1000, 128), 200), (512, (256, 256, 128, 384), 16), (1096, (384, 640), 64), (1024, (2304, 768), 256),
-    (256, (14336, 14336), 64),                   # gate/up of LLaMA3-8B: 224 row tiles on 128 CTAs, three tiles per CTA
 ])
 def test_group_of_decode_modules_matches_oracle(d_in, d_outs, T):
     ws = make_group(T, d_in, d_outs, seed=6000 + T)
@@ -91,12 +90,14 @@ def test_group_workspace_reused_across_calls():
     assert mb.meteora_workspace_status(workspace) == 0
 
 
-# What the one-launch kernel does not take runs module by module: a prefill batch, fp32 modules.
-@pytest.mark.parametrize("T,dtype,r,tol", [(300, "bf16", 8, 1e-2), (20, "f32", 8, 1e-4)])
-def test_group_falls_back_module_by_module(T, dtype, r, tol):
+# What the one-launch kernel does not take runs module by module: a prefill batch, fp32 modules, and groups with
+# so many row tiles that a CTA would finish more than two (gate/up of LLaMA3-8B: 224 tiles on 128 CTAs).
+@pytest.mark.parametrize("T,dtype,d_outs,tol", [(300, "bf16", (128, 200), 1e-2), (20, "f32", (128, 200), 1e-4),
+                                                (64, "bf16", (14336, 14336), 1e-2)])
+def test_group_falls_back_module_by_module(T, dtype, d_outs, tol):
     N = 6 if dtype == "f32" else 28
-    ws = make_group(T, 256, (128, 200), seed=6300 + T, dtype=dtype, N=N)
-    assert mb.meteora_group_plan(T, 256, [128, 200], N, 8, 2, torch.float32 if dtype == "f32" else torch.bfloat16) == 0
+    ws = make_group(T, 256, d_outs, seed=6300 + T, dtype=dtype, N=N)
+    assert mb.meteora_group_plan(T, 256, list(d_outs), N, 8, 2, torch.float32 if dtype == "f32" else torch.bfloat16) == 0
     check_group(ws, y_tol=tol)
 
 
