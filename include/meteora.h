@@ -259,7 +259,8 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "no_tma_store"   1 = plain stores of y where the TMA store would apply
  *   "force_simt"     1 = never take a tensor-core path
  *   "pdl"            default 1 = the three launches of a call overlap by programmatic dependent launch
- *   "fused"          default 1; 0 = never use the single-launch decode kernel
+ *   "fused"          default 1; 0 = never use the single-launch decode kernel; 2 = also where the planner
+ *                    prefers the three launches (layers with several row tiles per CTA below 32 tokens)
  *   "coop"           default 1; 0 = launch the decode kernel without the co-residency guarantee
  *   "no_hold"        1 = the decode kernel's main CTAs do not wait for the aux CTAs' first loads
  *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)

@@ -1372,6 +1372,9 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     // Measured (gate/up of LLaMA3-8B, 224 row tiles, T = 64): a group whose CTAs finish three tiles one after the
     // other takes 83 us in one launch against 2 x 36 us as two calls, so groups stay within two tiles per CTA.
     if (G > 1 && segs > 2) return fp;
+    // A single layer with more row tiles than CTAs (4096 -> 32000, three tiles per CTA): 75 us here against 61 us
+    // for the three launches at T = 1, 89 against 96 us at T = 64: taken from 32 tokens up.
+    if (segs > 2 && s.T < 32 && tn.fused != 2) return fp;
     fp.segs = segs;
     fp.n_main = n_main;
     // shared memory: staged B rows (at most 128 rows of every adapter), routing, barriers, ring

@@ -266,6 +266,7 @@ def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
     w = workloads.make_workload("fused", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="rms",
                                 seed=50 + T + d_out, b_std=0.3)
     mb.meteora_set_tuning("splits", per_tile)
+    mb.meteora_set_tuning("fused", 2)                                # 2: also where the three launches are the default
     try:
         shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
         assert "fused_decode" in mb.meteora_describe_plan(shape)
@@ -276,6 +277,7 @@ def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
         np.testing.assert_array_equal(i1, i2)
     finally:
         mb.meteora_set_tuning("splits", 0)
+        mb.meteora_set_tuning("fused", 1)
 
 
 # Adapter counts that change the layout of the stacked shrink: Wg behind A's only tile (N = 4), Wg in a tile of
