@@ -1356,11 +1356,14 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     if (m_max < 1) return fp;
     const int m_even = fp.row_tiles * std::min(8, m_max / fp.row_tiles);
     int n_main = std::min(m_max, 6 * fp.row_tiles);
-    // (large batches exchange 64 KB and more per partial tile: there even 80 % of the CTAs are the better deal)
-    if (m_even > 0 && m_even * 10 >= n_main * (s.T >= 96 ? 8 : 9)) n_main = m_even;
+    // (measured at 5120 -> 13824 and 4096 -> 14336, 84 % and 88 %: the even unit ranges win by 4 - 8 % up to 192
+    // tokens; with 256-token tiles, whose partial tiles are 128 KB each, the whole tiles win by 11 %)
+    if (m_even > 0 && m_even * 10 >= n_main * (s.T > 192 ? 8 : 9)) n_main = m_even;
     // an uneven split makes a CTA finish up to 128 rows: if the B rows of 128 rows of every adapter (large ranks)
     // would crowd out the ring, stay with whole tiles per CTA group
     if (m_even > 0 && n_main % fp.row_tiles != 0 && (size_t)s.N * kBM * s.r * 2 > 64 * 1024) n_main = m_even;
+    if (tn.unit_split == 1) n_main = std::min(m_max, 6 * fp.row_tiles);
+    if (tn.unit_split == 2 && m_even > 0) n_main = m_even;
     if (tn.splits > 0 && tn.splits * fp.row_tiles <= m_max) n_main = std::min(tn.splits, 8) * fp.row_tiles;
     n_main = (int)std::min<long long>(n_main, units);
     if (n_main < 1 || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
