@@ -294,7 +294,7 @@ int meteora_linear_forward_group(const void* x, const void* const* W0, const voi
 size_t meteora_gate_backward_workspace_bytes(const meteora_shape_t* shape) {
     if (check_shape(shape, true, true) != METEORA_OK) return 0;
     const size_t S = (size_t)shape->T * shape->k, r = (size_t)shape->r;
-    return kHeaderBytes + 2 * align_up(S * 4, 256) + 2 * align_up(S * r * 4, 256) +
+    return kHeaderBytes + 2 * align_up(S * 4, 256) + 2 * align_up(gate_backward_shrink_floats(*shape) * 4, 256) +
            2 * align_up(((size_t)shape->N + 1) * 4, 256) +
            align_up((size_t)shape->N * shape->d_out * r * elem_size(shape->dtype), 256);
 }
@@ -318,13 +318,17 @@ int meteora_gate_backward(const void* x, const void* A, const void* B, const voi
     };
     float* dl = (float*)take(S * 4);
     int32_t* perm = (int32_t*)take(S * 4);
-    float* u = (float*)take(S * r * 4);
-    float* z = (float*)take(S * r * 4);
+    const size_t shrink_bytes = gate_backward_shrink_floats(*shape) * 4;
+    float* u = (float*)take(shrink_bytes);
+    float* z = (float*)take(shrink_bytes);
     int32_t* counts = (int32_t*)take(((size_t)shape->N + 1) * 4);
     int32_t* offsets = (int32_t*)take(((size_t)shape->N + 1) * 4);
     void* Bt = take((size_t)shape->N * shape->d_out * r * elem_size(shape->dtype));
     cudaStream_t st = (cudaStream_t)stream;
-    rc = launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, Bt, u, z, dl, counts, offsets, perm, dWg, st);
+    // the header's first words take the error flags of the tensor-core kernels
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) return METEORA_ERR_CUDA;
+    rc = launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, Bt, u, z, dl, counts, offsets, perm,
+                              (int32_t*)workspace, dWg, st);
     if (rc != METEORA_OK) return rc;
     if (dlogit && S > 0)
         return cuda_status(cudaMemcpyAsync(dlogit, dl, S * sizeof(float), cudaMemcpyDeviceToDevice, st));

@@ -60,7 +60,10 @@ int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int
 // route.cu
 int launch_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
                          const float* topk_w, const meteora_shape_t& s, void* Bt, float* u, float* z, float* dlogit,
-                         int32_t* counts, int32_t* offsets, int32_t* perm, float* dWg, cudaStream_t st);
+                         int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* status, float* dWg,
+                         cudaStream_t st);
+bool gate_backward_dense(const meteora_shape_t& s);            // both shrinks as dense products on the tensor cores
+size_t gate_backward_shrink_floats(const meteora_shape_t& s);  // floats of each of the two shrink outputs
 int launch_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets, int32_t* perm,
                  cudaStream_t st);
 // lora.cu

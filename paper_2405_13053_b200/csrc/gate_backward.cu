@@ -5,12 +5,19 @@
 //   dlogit[t,j] = w[t,j] * (g[t,j] - sum_m w[t,m] g[t,m]) / tau
 //   dWg[e,:]    = sum over the slots (t,j) that picked e of dlogit[t,j] * x_t
 //
-// The slots are bucketed by adapter first (meteora_route's stable permutation, Sec. 3.3).  Both rank-r vectors
-// then come from the grouped shrink kernel of the LoRA term (a CTA stages one adapter's rows in shared memory
-// for up to 32 of its slots): A_e x_t as it is, B_e^T dy_t on a transposed copy of B.  A thread per token applies
-// the softmax Jacobian, and a CTA per (adapter, 256 columns of d_in) adds its bucket in permutation order, so
-// the result does not depend on scheduling and needs no atomics.
+// The slots are bucketed by adapter first (meteora_route's stable permutation, Sec. 3.3).  With B transposed,
+// B_e^T dy_t is the same product as the shrink A_e x_t, so both rank-r vectors come from one kernel run twice:
+//   - bf16 layers the tensor cores take: the stacked shrink of the forward pass ([A_0..A_{N-1}] x for ALL adapters
+//     as one dense product, Sec. 3.3), once on (x, A) and once on (dy, B^T); the slots then read their adapter's
+//     r columns.  The dense product does N / k times the needed flops and is still several times faster than
+//     gathering, as in the forward pass;
+//   - otherwise the grouped shrink kernel of the LoRA term (a CTA stages one adapter's rows in shared memory for
+//     up to 32 of its slots).
+// A warp per token applies the softmax Jacobian, and a CTA per (adapter, 256 columns of d_in) adds its bucket in
+// permutation order, so the result does not depend on scheduling and needs no atomics.
 #include "common.cuh"
+
+#include <algorithm>
 
 namespace meteora {
 
@@ -27,23 +34,33 @@ __global__ void k_transpose_b(const TI* __restrict__ B, TI* __restrict__ Bt, int
 }
 
 // g[t,j] = < B_e^T dy_t, A_e x_t > from the two shrink outputs, then
-// dlogit[t,j] = w_j (g_j - sum_m w_m g_m) / tau; one thread per token.
-__global__ void k_gate_dlogit(const float* __restrict__ u, const float* __restrict__ z,
-                              const float* __restrict__ topk_w, int T, int k, int r, float inv_tau,
-                              float* __restrict__ dlogit) {
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+// dlogit[t,j] = w_j (g_j - sum_m w_m g_m) / tau; one warp per token.  The shrink outputs are either per slot
+// (`dense` = 0: u[(t*k + j)*r + p]) or the stacked shrink's rows (`dense` = 1: u[z][t][e*r + p], `zsplits` partial
+// copies `zstride` floats apart that are added in slice order, row pitch `ld`).
+__global__ void __launch_bounds__(256)
+k_gate_dlogit(const float* __restrict__ u, const float* __restrict__ z, const int32_t* __restrict__ topk_idx,
+              const float* __restrict__ topk_w, int T, int N, int k, int r, float inv_tau, int dense, int ld,
+              int zsplits_u, int zsplits_z, size_t zstride, float* __restrict__ dlogit) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (t >= T) return;
     float g[METEORA_MAX_K];
     float mean = 0.f;
     for (int j = 0; j < k; ++j) {
-        const float* us = u + ((size_t)t * k + j) * r;
-        const float* zs = z + ((size_t)t * k + j) * r;
+        const int e = min(max(topk_idx[(size_t)t * k + j], 0), N - 1);
+        const size_t row = dense ? (size_t)t * ld + (size_t)e * r : ((size_t)t * k + j) * r;
         float acc = 0.f;
-        for (int p = 0; p < r; ++p) acc = fmaf(us[p], zs[p], acc);
-        g[j] = acc;
-        mean = fmaf(topk_w[(size_t)t * k + j], acc, mean);
+        for (int p = lane; p < r; p += 32) {
+            float uv = 0.f, zv = 0.f;
+            for (int q = 0; q < zsplits_u; ++q) uv += u[q * zstride + row + p];
+            for (int q = 0; q < zsplits_z; ++q) zv += z[q * zstride + row + p];
+            acc = fmaf(uv, zv, acc);
+        }
+        g[j] = warp_sum(acc);
+        mean = fmaf(topk_w[(size_t)t * k + j], g[j], mean);
     }
-    for (int j = 0; j < k; ++j) dlogit[(size_t)t * k + j] = topk_w[(size_t)t * k + j] * (g[j] - mean) * inv_tau;
+    if (lane == 0)
+        for (int j = 0; j < k; ++j) dlogit[(size_t)t * k + j] = topk_w[(size_t)t * k + j] * (g[j] - mean) * inv_tau;
 }
 
 // dWg[e, d] = sum over the adapter's bucket of dlogit[slot] * x[token(slot), d].  A CTA owns 256 columns of one
@@ -92,7 +109,8 @@ k_gate_dwg(const TI* __restrict__ x, const float* __restrict__ dlogit, const int
 
 int launch_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
                          const float* topk_w, const meteora_shape_t& s, void* Bt, float* u, float* z, float* dlogit,
-                         int32_t* counts, int32_t* offsets, int32_t* perm, float* dWg, cudaStream_t st) {
+                         int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* status, float* dWg,
+                         cudaStream_t st) {
     int rc;
     if (s.T == 0) return cuda_status(cudaMemsetAsync(dWg, 0, (size_t)s.N * s.d_in * sizeof(float), st));
     if ((rc = launch_route(topk_idx, s.T, s.k, s.N, counts, offsets, perm, st)) != METEORA_OK) return rc;
@@ -101,12 +119,31 @@ int launch_gate_backward(const void* x, const void* A, const void* B, const void
     else
         k_transpose_b<float><<<296, 256, 0, st>>>((const float*)B, (float*)Bt, s.N, s.d_out, s.r);
     if ((rc = last_launch_status()) != METEORA_OK) return rc;
-    // u = A_e x_t and z = B_e^T dy_t for every slot, adapter by adapter over the bucketed slots
-    if ((rc = launch_shrink_segments(x, A, offsets, perm, s, u, st)) != METEORA_OK) return rc;
     meteora_shape_t sb = s;
-    sb.d_in = s.d_out;                                           // the contraction runs over d_out here
-    if ((rc = launch_shrink_segments(dy, Bt, offsets, perm, sb, z, st)) != METEORA_OK) return rc;
-    k_gate_dlogit<<<(s.T + 255) / 256, 256, 0, st>>>(u, z, topk_w, s.T, s.k, s.r, 1.0f / s.temperature, dlogit);
+    sb.d_in = s.d_out;                                           // the contraction of B_e^T dy runs over d_out
+    const bool dense = gate_backward_dense(s);
+    int ld = 0, zs_u = 1, zs_z = 1;
+    if (dense) {
+        // u = [A_0; ..; A_{N-1}] x and z = [B_0^T; ..; B_{N-1}^T] dy for every adapter on the tensor cores.  The
+        // kernel also wants a gate matrix of N rows: the first N rows of the stacked operand stand in, and
+        // the N columns they produce are not read.
+        Workspace wu = {}, wz = {};
+        wu.status = wz.status = status;
+        wu.ld_u = wz.ld_u = ld = tc_stacked_pitch(s, &wu.col_logits);
+        wz.col_logits = wu.col_logits;
+        wu.u_all = u;
+        wz.u_all = z;
+        if ((rc = launch_stacked_shrink_tc(x, A, A, s, wu, st)) != METEORA_OK) return rc;
+        if ((rc = launch_stacked_shrink_tc(dy, Bt, Bt, sb, wz, st)) != METEORA_OK) return rc;
+        zs_u = tc_stacked_zsplits(s);
+        zs_z = tc_stacked_zsplits(sb);
+    } else {
+        // adapter by adapter over the bucketed slots
+        if ((rc = launch_shrink_segments(x, A, offsets, perm, s, u, st)) != METEORA_OK) return rc;
+        if ((rc = launch_shrink_segments(dy, Bt, offsets, perm, sb, z, st)) != METEORA_OK) return rc;
+    }
+    k_gate_dlogit<<<(s.T + 7) / 8, 256, 0, st>>>(u, z, topk_idx, topk_w, s.T, s.N, s.k, s.r, 1.0f / s.temperature,
+                                                 dense ? 1 : 0, ld, zs_u, zs_z, (size_t)s.T * ld, dlogit);
     if ((rc = last_launch_status()) != METEORA_OK) return rc;
     const dim3 grid(s.N, (s.d_in + 255) / 256);
     if (s.dtype == METEORA_BF16)
@@ -114,6 +151,20 @@ int launch_gate_backward(const void* x, const void* A, const void* B, const void
     else
         k_gate_dwg<float><<<grid, 256, 0, st>>>((const float*)x, dlogit, offsets, perm, s.d_in, s.k, dWg);
     return last_launch_status();
+}
+
+// Both products of the gate gradient as dense stacked shrinks on the tensor cores?
+bool gate_backward_dense(const meteora_shape_t& s) {
+    meteora_shape_t sb = s;
+    sb.d_in = s.d_out;
+    return tc_path_supported(s) && tc_path_supported(sb);
+}
+
+// Floats of each of the two shrink outputs: per slot, or the stacked shrink's partial copies.
+size_t gate_backward_shrink_floats(const meteora_shape_t& s) {
+    const size_t slots = (size_t)s.T * s.k * s.r;
+    if (!gate_backward_dense(s)) return slots;
+    return std::max(slots, (size_t)s.T * tc_stacked_pitch(s, nullptr) * stacked_zsplits_bound(s.T));
 }
 
 }  // namespace meteora

@@ -30,6 +30,9 @@ def dy_like(w, seed):
     dict(T=50, d_in=100, d_out=70, N=6, r=3, k=3, dtype="f32"),                  # nothing aligned, odd rank
     dict(T=40, d_in=128, d_out=96, N=64, r=8, k=8, dtype="f32"),                 # most adapters, most picks
     dict(T=20, d_in=64, d_out=64, N=5, r=8, k=1, dtype="bf16"),                  # top-1: zero gradient
+    dict(T=1100, d_in=512, d_out=640, N=28, r=8, k=2, dtype="bf16"),             # dense shrinks on pairs of SMs
+    dict(T=33, d_in=128, d_out=100, N=10, r=8, k=2, dtype="bf16"),               # d_out no multiple of 8: grouped shrink
+    dict(T=130, d_in=1024, d_out=256, N=64, r=24, k=4, dtype="bf16"),            # 1536 stacked rows, rank 24
 ])
 def test_gate_backward_matches_oracle(case):
     kw = dict(case)
