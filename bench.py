@@ -56,6 +56,9 @@ def parse_args():
     ap.add_argument("--variants", action="store_true",
                     help="time the variants of the method at 4096 -> 4096 (top-k, rank, adapter count, temperature), "
                          "the axes of the paper's synthetic sweep (App. A.7); one JSON line each")
+    ap.add_argument("--decode-loop", action="store_true",
+                    help="time one autoregressive decode step over the 224 MeteoRA linears of a LLaMA3-8B-shaped "
+                         "stack (ms per generated token, the unit of App. A.7); also part of --sweep")
     return ap.parse_args()
 
 
@@ -618,6 +621,96 @@ def run_layer_sweep():
         del mods, graph, groups
 
 
+def run_decode_loop():
+    """One autoregressive decode step over all 224 MeteoRA linears of a LLaMA3-8B-shaped stack (32 decoder layers
+    x 7 linears, each with its own gate and adapters, Sec. 3.2), in the unit of the paper's App. A.7 figures:
+    milliseconds per generated token.  A batch of b sequences generates b tokens per step (T = b).  Only the
+    MeteoRA linears run (no attention, norms or sampling: those are not part of the method), every linear on its
+    own synthetic input, the ones that share their input in a real block (q/k/v, gate/up) as group calls; one CUDA
+    graph per step."""
+    import ctypes
+
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import workloads
+
+    lib = mb.load_library()
+    hbm, _ = measured_peaks()
+    dt, es, n_layers = torch.bfloat16, 2, 32
+    g = torch.Generator(device="cuda").manual_seed(17)
+    weights = []                                                   # 32 layers x 7 linears: 14 GB of W0
+    for _ in range(n_layers):
+        layer = {}
+        for name, (d_in, d_out) in workloads.CONFIG4_LINEARS.items():
+            layer[name] = {"W0": (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt),
+                           "A": ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt),
+                           "B": (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt),
+                           "Wg": (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt)}
+        weights.append(layer)
+    vpa = lambda ts: (ctypes.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+    for T in (1, 16, 64):
+        xs = {d: torch.from_numpy(workloads.make_x(T, d, "rms", 60 + i, "bf16")).to(dt).cuda()
+              for i, d in enumerate(sorted({di for di, _ in workloads.CONFIG4_LINEARS.values()}))}
+        calls, nbytes, launches = [], 0.0, 0
+        for layer in weights:
+            for names in (("q", "k", "v"), ("o",), ("gate", "up"), ("down",)):
+                d_in = workloads.CONFIG4_LINEARS[names[0]][0]
+                d_out_list = [workloads.CONFIG4_LINEARS[n][1] for n in names]
+                shape = mb.make_shape(T, d_in, d_out_list[0], N_ADAPTERS, RANK, TOPK, dt)
+                d_outs = (ctypes.c_int * len(names))(*d_out_list)
+                n = lib.meteora_group_workspace_bytes(ctypes.byref(shape), d_outs, len(names))
+                ys = [torch.empty(T, d, device="cuda", dtype=dt) for d in d_out_list]
+                calls.append({"x": xs[d_in], "G": len(names), "d_outs": d_outs, "shape": shape, "ys": ys,
+                              "W0": vpa([layer[n_]["W0"] for n_ in names]), "A": vpa([layer[n_]["A"] for n_ in names]),
+                              "B": vpa([layer[n_]["B"] for n_ in names]), "Wg": vpa([layer[n_]["Wg"] for n_ in names]),
+                              "y": vpa(ys), "ws": torch.zeros(n, dtype=torch.uint8, device="cuda")})
+                launches += 1 if lib.meteora_group_plan(ctypes.byref(shape), d_outs, len(names)) else len(names)
+                touched = min(N_ADAPTERS, T * TOPK)
+                for d_out in d_out_list:
+                    nbytes += (d_in * d_out + N_ADAPTERS * d_in + touched * RANK * (d_in + d_out) + T * (d_in + d_out)) * es
+
+        def step():
+            st = torch.cuda.current_stream().cuda_stream
+            for c in calls:
+                rc = lib.meteora_linear_forward_group(c["x"].data_ptr(), c["W0"], c["A"], c["B"], c["Wg"], c["d_outs"],
+                                                      c["G"], ctypes.byref(c["shape"]), c["y"], c["ws"].data_ptr(),
+                                                      c["ws"].numel(), st)
+                if rc != 0:
+                    raise mb.MeteoraError(rc, "meteora_linear_forward_group")
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        iters = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        for c in calls:
+            st = mb.meteora_workspace_status(c["ws"])
+            if st != 0:
+                raise mb.MeteoraError(st, "device status")
+        ms = e0.elapsed_time(e1) / iters
+        print(json.dumps({"op": "decode_step", "shape": "LLaMA3-8B stack: 32 layers x (q k v o gate up down), MeteoRA linears only",
+                          "batch": T, "ms_per_generated_token": round(ms, 3), "tokens_per_s": round(T / ms * 1e3),
+                          "launches_per_step": launches, "bound": "hbm", "roofline_ms": round(nbytes / hbm / 1e6, 3),
+                          "frac_of_roofline": round(nbytes / hbm / 1e6 / ms, 3),
+                          "modules": n_layers * len(workloads.CONFIG4_LINEARS)}), flush=True)
+        del calls, graph
+
+
 def run_gate_backward_sweep():
     """meteora_gate_backward (gradient of the gate weights for a forward's routing) at the q_proj shape."""
     import torch
@@ -655,7 +748,7 @@ def run_gate_backward_sweep():
                           "tokens_per_s": round(T / us * 1e6), "bound": "hbm",
                           "roofline_us": round(nbytes / hbm / 1e3, 2),
                           "frac_of_roofline": round(nbytes / hbm / 1e3 / us, 3),
-                          "note": "7 launches (bucketing, transpose of B, two grouped shrinks, dlogit, reduction over tokens, copy); stream timing through the Python binding"}),
+                          "note": "bucketing, transpose of B, two stacked shrinks on the tensor cores, dlogit, reduction over tokens, copy; stream timing through the Python binding"}),
               flush=True)
 
 
@@ -750,10 +843,13 @@ def main():
     args = parse_args()
     if args.variants:
         run_variants()
+    elif args.decode_loop:
+        run_decode_loop()
     elif args.sweep:
         run_sweep(args)
         run_layer_sweep()
         run_gate_backward_sweep()
+        run_decode_loop()
     elif args.impl == "reference":
         run_reference(args)
     else:

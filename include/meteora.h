@@ -264,6 +264,7 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "coop"           default 1; 0 = launch the decode kernel without the co-residency guarantee
  *   "unit_split"     decode kernel's main CTAs: 0 = planner's choice, 1 = even unit ranges over all free SMs,
  *                    2 = whole row tiles per group of CTAs (falls back to the choice that fits)
+ *   "aux_ctas"       > 0 = how many CTAs of the decode kernel the stacked shrink and the selection may take
  *   "no_hold"        1 = the decode kernel's main CTAs do not wait for the aux CTAs' first loads
  *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)
  *                    where the pairs cover a quarter of the SMs; 0 = never; 2 = wherever the shape allows

@@ -453,6 +453,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "coop")) t.coop = value;
     else if (!strcmp(name, "no_hold")) t.no_hold = value;
     else if (!strcmp(name, "unit_split")) t.unit_split = value;
+    else if (!strcmp(name, "aux_ctas")) t.aux_ctas = value;
     else if (!strcmp(name, "pair")) t.pair = value;
     else return METEORA_ERR_INVALID_ARG;
     return METEORA_OK;

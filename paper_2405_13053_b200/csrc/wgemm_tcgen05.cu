@@ -1344,7 +1344,8 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     fp.why = 2;
     const int group_tiles = G * fp.aux_tiles;                    // every module has its own stacked shrink
     if (group_tiles + 8 > sms) return fp;
-    const int aux_budget = std::min(std::max(std::max(20, 4 * group_tiles), group_tiles), sms - 8);
+    int aux_budget = std::min(std::max(std::max(20, 4 * group_tiles), group_tiles), sms - 8);
+    if (tn.aux_ctas > 0) aux_budget = std::min(std::max(tn.aux_ctas, group_tiles), sms - 8);
     fp.aux_slices = std::min(std::min(aux_budget / group_tiles, ksteps), 16);   // 16: the selection reads all slices at once
     if (fp.aux_slices < 1) return fp;
     fp.n_aux = group_tiles * fp.aux_slices;
