@@ -38,7 +38,7 @@
 extern "C" {
 #endif
 
-#define METEORA_MAX_N 64
+#define METEORA_MAX_N 128
 #define METEORA_MAX_K 8
 #define METEORA_MAX_R 64
 #define METEORA_STATIC_SCRATCH_FLOATS 65536 /* capacity of meteora_lora_delta_static: T * k * r may not exceed it */

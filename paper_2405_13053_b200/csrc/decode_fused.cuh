@@ -120,11 +120,12 @@ __device__ __forceinline__ void select_token_wide(const float* u_part, int ld_u,
         }
     }
     __syncwarp();
-    const float v0 = lane < N ? wbuf[col_logits + lane] : 0.f;
-    const float v1 = lane + 32 < N ? wbuf[col_logits + lane + 32] : 0.f;
+    float v[kSelVals];
+#pragma unroll
+    for (int i = 0; i < kSelVals; ++i) v[i] = lane + 32 * i < N ? wbuf[col_logits + lane + 32 * i] : 0.f;
     int idx;
     float w;
-    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
     if (lane < k) {
         topk_idx[(size_t)t * k + lane] = idx;
         topk_w[(size_t)t * k + lane] = w;

@@ -1,6 +1,6 @@
 // Gate logits, top-k selection and softmax over the selected logits (Sec. 3.1, Eq. 3; temperature App. A.5).
 //
-// One warp owns one token.  Lane n (and lane n-32 for n >= 32) holds logit n; the k picks are
+// One warp owns one token.  Lane l holds the logits l, l + 32, l + 64, l + 96; the k picks are
 // taken by k rounds of a warp-wide arg-max whose ordering is (logit descending, index ascending),
 // so equal logits always resolve to the lower adapter index.
 #include <math_constants.h>
@@ -21,19 +21,23 @@ k_gate_topk(const TI* __restrict__ x, const TI* __restrict__ Wg, int T, int d_in
     if (t >= T) return;
     const bool vec = (d_in % 8) == 0;
     const TI* xt = x + (size_t)t * d_in;
-    float v0 = 0.f, v1 = 0.f;
+    float v[kSelVals];
+#pragma unroll
+    for (int i = 0; i < kSelVals; ++i) v[i] = 0.f;
     for (int n = 0; n < N; ++n) {
         const float l = warp_dot(xt, Wg + (size_t)n * d_in, d_in, lane, vec);
-        if (n == lane) v0 = l;
-        if (n == lane + 32) v1 = l;
+#pragma unroll
+        for (int i = 0; i < kSelVals; ++i)
+            if (n == lane + 32 * i) v[i] = l;
     }
     if (logits) {
-        if (lane < N) logits[(size_t)t * N + lane] = v0;
-        if (lane + 32 < N) logits[(size_t)t * N + lane + 32] = v1;
+#pragma unroll
+        for (int i = 0; i < kSelVals; ++i)
+            if (lane + 32 * i < N) logits[(size_t)t * N + lane + 32 * i] = v[i];
     }
     int idx;
     float w;
-    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
     if (lane < k) {
         topk_idx[(size_t)t * k + lane] = idx;
         topk_w[(size_t)t * k + lane] = w;

@@ -8,20 +8,27 @@
 
 namespace meteora {
 
-// v0 = logit[lane], v1 = logit[lane + 32]; entries at or beyond N are ignored.
+// Logits per lane: lane l holds logit l, l + 32, l + 64, l + 96 (METEORA_MAX_N = 128 adapters).
+constexpr int kSelVals = METEORA_MAX_N / 32;
+
+// v[i] = logit[lane + 32 i]; entries at or beyond N are ignored.
 // On return lane j < k holds pick j (index and softmax weight).  Every lane runs the same code.
-__device__ __forceinline__ void warp_topk_softmax(float v0, float v1, int N, int k, float inv_tau, int lane,
+__device__ __forceinline__ void warp_topk_softmax(float (&v)[kSelVals], int N, int k, float inv_tau, int lane,
                                                   int& my_idx, float& my_w) {
-    bool taken0 = lane >= N, taken1 = lane + 32 >= N;
-    if (!(v0 > -CUDART_INF_F)) v0 = -CUDART_INF_F;  // NaN never wins a comparison; treat it as -inf
-    if (!(v1 > -CUDART_INF_F)) v1 = -CUDART_INF_F;
+    bool taken[kSelVals];
+#pragma unroll
+    for (int i = 0; i < kSelVals; ++i) {
+        taken[i] = lane + 32 * i >= N;
+        if (!(v[i] > -CUDART_INF_F)) v[i] = -CUDART_INF_F;  // NaN never wins a comparison; treat it as -inf
+    }
     float first = 0.f, sum = 0.f, my_e = 0.f;
     my_idx = 0;
     for (int j = 0; j < k; ++j) {
         float bv = -CUDART_INF_F;
         int bi = 0x7FFFFFFF;
-        if (!taken0) { bv = v0; bi = lane; }
-        if (!taken1 && (bi == 0x7FFFFFFF || v1 > bv)) { bv = v1; bi = lane + 32; }
+#pragma unroll
+        for (int i = 0; i < kSelVals; ++i)                   // ascending index: a later equal value does not replace
+            if (!taken[i] && (bi == 0x7FFFFFFF || v[i] > bv)) { bv = v[i]; bi = lane + 32 * i; }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
@@ -29,8 +36,9 @@ __device__ __forceinline__ void warp_topk_softmax(float v0, float v1, int N, int
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
         bi = min(bi, N - 1);
-        if (bi == lane) taken0 = true;
-        if (bi == lane + 32) taken1 = true;
+#pragma unroll
+        for (int i = 0; i < kSelVals; ++i)
+            if (bi == lane + 32 * i) taken[i] = true;
         if (j == 0) first = bv;
         const float e = expf((bv - first) * inv_tau);
         sum += e;
@@ -52,22 +60,22 @@ template <bool kCoherent, int ZMAX>
 __device__ __forceinline__ void select_token_few(const float* row, int col_logits, int zsplits, size_t zstride,
                                                  int t, int N, int r, int k, float inv_tau, int lane,
                                                  int32_t* topk_idx, float* topk_w, float* uw) {
-    float part0[ZMAX], part1[ZMAX];
+    float v[kSelVals];
 #pragma unroll
-    for (int z = 0; z < ZMAX; ++z) {
-        const bool on = z < zsplits;
-        part0[z] = (on && lane < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane) : 0.f;
-        part1[z] = (on && lane + 32 < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32) : 0.f;
-    }
-    float v0 = 0.f, v1 = 0.f;
+    for (int i = 0; i < kSelVals; ++i) {
+        v[i] = 0.f;
+        if (32 * i < N) {                                   // uniform across the warp
+            float part[ZMAX];
 #pragma unroll
-    for (int z = 0; z < ZMAX; ++z) {
-        v0 += part0[z];
-        v1 += part1[z];
+            for (int z = 0; z < ZMAX; ++z)
+                part[z] = (z < zsplits && lane + 32 * i < N) ? ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32 * i) : 0.f;
+#pragma unroll
+            for (int z = 0; z < ZMAX; ++z) v[i] += part[z];
+        }
     }
     int idx;
     float w;
-    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
     if (lane < k) {
         topk_idx[(size_t)t * k + lane] = idx;
         topk_w[(size_t)t * k + lane] = w;
@@ -110,8 +118,12 @@ __device__ __forceinline__ void select_token(const float* u_all, int ld_u, int c
         // butterfly, the same order for every token and every run.
         const float* mine = row + (size_t)min(lane, zsplits - 1) * zstride;
         const bool live = lane < zsplits;
-        float v0 = 0.f, v1 = 0.f;
-        for (int n0 = 0; n0 < N; n0 += 32) {
+        float v[kSelVals];
+#pragma unroll
+        for (int i = 0; i < kSelVals; ++i) v[i] = 0.f;
+#pragma unroll
+        for (int n0 = 0; n0 < 32 * kSelVals; n0 += 32) {
+            if (n0 >= N) break;
             float vals[32];
 #pragma unroll
             for (int n = 0; n < 32; ++n) vals[n] = (live && n0 + n < N) ? ld_part<kCoherent>(mine + col_logits + n0 + n) : 0.f;
@@ -119,13 +131,13 @@ __device__ __forceinline__ void select_token(const float* u_all, int ld_u, int c
             for (int n = 0; n < 32; ++n) {
                 if (n0 + n < N) {                       // uniform across the warp
                     const float sum = warp_sum(vals[n]);
-                    if (lane == n) { if (n0 == 0) v0 = sum; else v1 = sum; }
+                    if (lane == n) v[n0 / 32] = sum;
                 }
             }
         }
         int idx;
         float w;
-        warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+        warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
         if (lane < k) {
             topk_idx[(size_t)t * k + lane] = idx;
             topk_w[(size_t)t * k + lane] = w;
@@ -156,14 +168,17 @@ __device__ __forceinline__ void select_token(const float* u_all, int ld_u, int c
         if (lane < k * 8) uw[(size_t)t * k * 8 + lane] = out;
         return;
     }
-    float v0 = 0.f, v1 = 0.f;
+    float v[kSelVals];
+#pragma unroll
+    for (int i = 0; i < kSelVals; ++i) v[i] = 0.f;
     for (int z = 0; z < zsplits; ++z) {
-        if (lane < N) v0 += ld_part<kCoherent>(row + z * zstride + col_logits + lane);
-        if (lane + 32 < N) v1 += ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32);
+#pragma unroll
+        for (int i = 0; i < kSelVals; ++i)
+            if (lane + 32 * i < N) v[i] += ld_part<kCoherent>(row + z * zstride + col_logits + lane + 32 * i);
     }
     int idx;
     float w;
-    warp_topk_softmax(v0, v1, N, k, inv_tau, lane, idx, w);
+    warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
     if (lane < k) {
         topk_idx[(size_t)t * k + lane] = idx;
         topk_w[(size_t)t * k + lane] = w;

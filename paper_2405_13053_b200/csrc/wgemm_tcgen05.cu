@@ -819,7 +819,7 @@ int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits) {
 
 struct Plan;
 static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi = false,
-                      int bn_force = 0);
+                      int bn_force = 0, bool no_mma_expand = false);
 
 struct Plan {
     int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
@@ -841,7 +841,8 @@ int stacked_zsplits_bound(int T) {
     return std::min(kMaxZSplits, std::max(1, 148 / tiles));
 }
 
-static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi, int bn_force) {
+static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi, int bn_force,
+                      bool no_mma_expand) {
     const Tuning& tn = tuning();
     Plan pl = {};
     const int ksteps = (K + kBK - 1) / kBK;
@@ -903,7 +904,7 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
         pl.uw_off = (int)align_up((size_t)N * (kBM / splits) * 16, 16);
         pl.idx_off = pl.uw_off + bn * k * r * 4;
         epi_bytes = (size_t)pl.idx_off + (size_t)bn * k * 4;
-    } else if (lora && r == 8 && !tn.simt_expand) {
+    } else if (lora && r == 8 && !tn.simt_expand && !no_mma_expand) {
         // expand on the tensor cores: B rows of this split's adapters for all 128 rows, and the masked,
         // gate-weighted shrink outputs of the tile's tokens as the other operand
         pl.lora_mma = 1;
@@ -966,10 +967,14 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     if (pl.smem > 227 * 1024 && bn_force == 0 && tn.tile_tokens == 0) {
         for (int cand = 128; cand >= 16; cand /= 2) {
             if (cand >= bn) continue;
-            const Plan q = make_plan(row_tiles, T, K, lora, N, r, k, fused_epi, cand);
+            const Plan q = make_plan(row_tiles, T, K, lora, N, r, k, fused_epi, cand, no_mma_expand);
             if (q.smem <= 227 * 1024) return q;
         }
     }
+    // Many adapters (from about 100 at rank 8): the B rows of all of them for 128 output rows no longer fit
+    // beside the ring, so the expand of this kernel runs on CUDA cores, B rows read through L1.
+    if (pl.smem > 227 * 1024 && pl.lora_mma && bn_force == 0)
+        return make_plan(row_tiles, T, K, lora, N, r, k, fused_epi, 0, true);
     return pl;
 }
 

@@ -42,7 +42,7 @@ def test_status_strings(lib):
 def test_shape_validation_needs_no_gpu(lib):
     good = binding.make_shape(64, 256, 256, 4, 8, 2, __import__("torch").float32)
     assert binding.meteora_workspace_bytes(good) > 0
-    for field, value in (("k", 0), ("k", 5), ("N", 65), ("r", 65), ("d_in", 0), ("T", -1), ("temperature", 0.0)):
+    for field, value in (("k", 0), ("k", 5), ("N", 129), ("r", 65), ("d_in", 0), ("T", -1), ("temperature", 0.0)):
         bad = binding.make_shape(64, 256, 256, 4, 8, 2, __import__("torch").float32)
         setattr(bad, field, value)
         assert binding.meteora_workspace_bytes(bad) == 0, field

@@ -33,6 +33,7 @@ def dy_like(w, seed):
     dict(T=1100, d_in=512, d_out=640, N=28, r=8, k=2, dtype="bf16"),             # dense shrinks on pairs of SMs
     dict(T=33, d_in=128, d_out=100, N=10, r=8, k=2, dtype="bf16"),               # d_out no multiple of 8: grouped shrink
     dict(T=130, d_in=1024, d_out=256, N=64, r=24, k=4, dtype="bf16"),            # 1536 stacked rows, rank 24
+    dict(T=90, d_in=256, d_out=512, N=128, r=8, k=3, dtype="bf16"),              # 128 adapters
 ])
 def test_gate_backward_matches_oracle(case):
     kw = dict(case)

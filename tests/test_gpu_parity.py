@@ -31,6 +31,8 @@ GATE_CASES = [
     dict(T=19, d_in=72, d_out=8, N=40, k=8, dtype="bf16"),       # more than 32 adapters, k = 8
     dict(T=9, d_in=64, d_out=8, N=64, k=1, dtype="f32"),         # top-1
     dict(T=11, d_in=48, d_out=8, N=6, k=6, dtype="bf16"),        # k = N
+    dict(T=21, d_in=128, d_out=8, N=128, k=8, dtype="f32"),      # the most adapters: four logits per lane
+    dict(T=17, d_in=256, d_out=8, N=100, k=4, dtype="bf16"),     # the last lanes' fourth logit is out of range
     dict(T=1, d_in=4096, d_out=8, N=28, k=2, dtype="bf16"),
     dict(T=300, d_in=512, d_out=8, N=28, k=2, dtype="bf16", temperature=15.0),
 ]
@@ -182,6 +184,8 @@ FORWARD_CASES = [
     dict(T=300, d_in=256, d_out=256, N=12, r=12, k=3, dtype="bf16"),              # rank 12 -> 16, prefill batch
     dict(T=600, d_in=512, d_out=200, N=28, r=64, k=2, dtype="bf16"),              # rank 64 prefill, d_out % 8 == 0 only
     dict(T=24, d_in=256, d_out=136, N=4, r=8, k=4, dtype="bf16", temperature=20.0),  # k = N with temperature
+    dict(T=26, d_in=96, d_out=72, N=128, r=4, k=8, dtype="f32"),                  # 128 adapters on the plain path
+    dict(T=300, d_in=512, d_out=256, N=128, r=8, k=2, dtype="bf16"),              # 128 adapters: 1024 stacked rows + a gate tile
 ]
 
 
@@ -284,7 +288,8 @@ def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
 # its own (N = 16: A fills its tile), three A tiles with Wg behind 8 rows (N = 33, logits beyond one warp).
 # ... and ranks above 8 (16-byte words per B row: 2, 3, 4), which also change the number of stacked-shrink tiles.
 @pytest.mark.parametrize("N,k,T,r", [(4, 2, 9, 8), (16, 4, 40, 8), (33, 3, 130, 8), (2, 1, 3, 8),
-                                     (28, 2, 20, 16), (28, 2, 128, 32), (10, 3, 64, 24)])
+                                     (28, 2, 20, 16), (28, 2, 128, 32), (10, 3, 64, 24),
+                                     (128, 2, 64, 8), (100, 8, 7, 8), (72, 4, 128, 16)])   # more than 64 adapters
 def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
     w = workloads.make_workload("fused_n", T=T, d_in=768, d_out=896, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
                                 seed=900 + N + r, b_std=0.3)
@@ -301,6 +306,7 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
     (1024, 640, 600, 28, 2, 8), (512, 256, 257, 28, 2, 8), (1096, 512, 300, 28, 2, 8), (768, 1024, 1024, 7, 3, 8),
     (512, 512, 520, 16, 4, 8), (512, 384, 300, 33, 3, 8),      # Wg in a tile of its own; three tiles of stacked rows
     (512, 384, 700, 28, 2, 16), (512, 256, 300, 28, 4, 64), (512, 256, 520, 5, 2, 24),   # ranks 16, 64, 24: 2, 8, 1 rounds
+    (512, 512, 600, 128, 2, 8), (768, 256, 1100, 100, 4, 8),   # 128 and 100 adapters: 5 and 4 rounds of expand columns
 ])
 def test_prefill_on_pairs_of_sms_matches_oracle(d_in, d_out, T, N, k, r):
     w = workloads.make_workload("pairs", T=T, d_in=d_in, d_out=d_out, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
