@@ -774,7 +774,7 @@ def run_variants():
     points = [dict(base)]
     points += [dict(base, k=k) for k in (1, 4)]
     points += [dict(base, r=r) for r in (4, 16, 32, 64)]
-    points += [dict(base, N=N) for N in (8, 64)]
+    points += [dict(base, N=N) for N in (8, 64, 128)]
     points += [dict(base, tau=20.0)]
     for T in (32, 2048):
         for pt in points:
