@@ -14,8 +14,10 @@
 //     [A_0..A_{N-1}; Wg] x (every adapter's A_i x and the gate logits, Sec. 3.1) on the same main loop and
 //     writes it as an fp32 partial; once all partials are in, the aux CTAs share the tokens and run the
 //     top-k selection and the softmax over the selected logits (Eq. 3), publishing topk_idx, topk_w, uw.
-// The main CTAs hold their first loads back until the aux CTAs have issued theirs, so the 2 MB of the shrink
-// are ahead of W0 in the memory queues; they need the routing only after their main loop and the exchange
+// While the base product is short (W0 below about 50 MB) the main CTAs give the aux CTAs a head start of two
+// microseconds, so the 2 MB of the shrink are ahead of W0 in the memory queues (measured: a fixed delay does
+// as well as waiting for a counter the aux CTAs bump, without the round trip); they need the routing only after
+// their main loop and the exchange
 // of the partial tiles.  Every wait is bounded; on expiry the status word is set and the kernel drains.  The
 // counters live in the workspace header and are re-armed by the last CTA to exit.
 #pragma once
@@ -57,7 +59,7 @@ struct DecodeParams {
     int bar_stages;        // barriers are laid out for max(main stages, aux stages) ring slots
     int ld_u, col_logits;
     float inv_tau;
-    int hold;              // main CTAs start loading only after the aux CTAs have issued their first loads
+    int hold;              // 1: main CTAs start loading only after the aux CTAs have issued their first loads; > 1: after that many nanoseconds
     int32_t* ctr;          // [0] aux partials written, [1] selections published, [2] CTAs exited, [3] aux loads issued
     float* part_g;         // [row tile + main CTA][BN][128] fp32 partial accumulator tiles of the base product
     int32_t* tile_ctr;     // [row tiles] partials delivered per tile
@@ -475,7 +477,17 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
         if (warp == 0) {
             if (lane == 0) {
                 // let the stacked shrink get its loads into the memory queues first
-                bool ok = d.hold ? wait_counter(d.ctr + 3, n_active) : true;
+                bool ok = true;
+                if (d.hold == 1) {
+                    ok = wait_counter(d.ctr + 3, n_active);
+                } else if (d.hold > 1) {                         // a fixed head start for the aux CTAs, in nanoseconds
+                    unsigned long long t0, t1;
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+                    do {
+                        __nanosleep(64);
+                        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+                    } while (t1 - t0 < (unsigned long long)d.hold);
+                }
                 if (tr_main) FUSED_STAMP(p, 32, 1);
                 int cur_tile = -1, row0 = 0;
                 const CUtensorMap* tmW0 = &maps.W0[0];

@@ -1515,9 +1515,15 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
     d.ld_u = mods[0].ws.ld_u;
     d.col_logits = mods[0].ws.col_logits;
     d.inv_tau = 1.0f / s.temperature;
-    // Holding the main CTAs back until the aux CTAs have issued their loads pays only while the base product is
-    // short: from about 64 MB of W0 on the routing is ready long before it is needed either way.
-    d.hold = (tuning().no_hold || fp.w0_bytes > ((size_t)64 << 20)) ? 0 : 1;
+    // A head start for the aux CTAs' loads pays only while the base product is short: measured, 4096 -> 4096
+    // (34 MB) loses 0.5 - 1.4 us without it, 5120 -> 5120 (52 MB) gains 0.6 - 1.5 us without it (the routing is
+    // ready long before it is needed either way).  Knob no_hold: 1 = none, 64 = wait for the aux CTAs' counter,
+    // any other value = that many nanoseconds.
+    {
+        const int nh = tuning().no_hold;
+        const bool is_short = fp.w0_bytes < ((size_t)52 << 20);
+        d.hold = nh == 1 ? 0 : nh == 64 ? 1 : nh > 1 ? nh : is_short ? 2100 : 0;
+    }
     d.ctr = status + 16;
     d.part_g = part_g;
     d.tile_ctr = tile_ctr;
