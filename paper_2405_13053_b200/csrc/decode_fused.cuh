@@ -399,11 +399,17 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 // A's last tile has its own map (its box stops at A's last row when Wg follows in the same tile)
                 const CUtensorMap* mA = tile >= d.a_tiles ? nullptr : tile == d.a_tiles - 1 ? &maps.At[am] : &maps.A[am];
                 const CUtensorMap* mG = tile == d.gate_tile ? &maps.G[am] : nullptr;
+                if (tr_aux) FUSED_STAMP(p, 48, 6);
                 if (!fused_producer(geom, mA, &tmX1, tile * kBM, ks0, niter, d.ctr + 3, mG, (uint32_t)d.gate_row0 * 128u))
                     flag_error(p, 1, 400);
+                if (tr_aux) FUSED_STAMP(p, 48, 7);
             }
         } else if (warp == 1) {
             if (lane == 0 && active) {
+#ifdef METEORA_TRACE
+                if (niter > 0) mbar_wait(bar_base, 0);                          // first stage landed
+                FUSED_STAMP(p, 48, 8);
+#endif
                 if (!fused_mma(geom, tmem_base, idesc, niter)) flag_error(p, 2, 500);
                 umma_commit(bar_acc);
                 if (tr_aux) FUSED_STAMP(p, 48, 1);
