@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "5390547325db34e9", "bytes_per_launch": {"128": 38646357 + 159061}}
+NCU_TRAFFIC = {"kernel_sha": "f0594772e4287990", "bytes_per_launch": {"128": 38646699 + 172544}}
 
 
 def parse_args():
