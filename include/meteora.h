@@ -136,10 +136,10 @@ int meteora_lora_delta_static(const void* x, const void* A, const void* B, const
  *   meteora_workspace_bytes(shape); calls that share a workspace must not overlap in time.
  * After the call the workspace holds the routing that was used (meteora_workspace_routing).
  * bf16 shapes with d_in % 8 == 0 and r % 8 == 0 run on the tensor-core paths (TMA + tcgen05):
- * decode batches (T <= 256, rank 8, d_out <= 16384) as ONE cooperative kernel launch in which
- * the CTAs exchange partial results through the workspace, everything else as three launches
+ * decode batches (T <= 256, rank a multiple of 8 whose staged rows of B fit shared memory) as ONE cooperative
+ * kernel launch in which the CTAs exchange partial results through the workspace, everything else as three launches
  * (stacked shrink [A; Wg] x, selection, base product with the LoRA expand; for prefill batches of
- * rank 8 on pairs of SMs with two-CTA MMAs).  A bf16 layer whose rank is no multiple of 8 takes the same
+ * ranks that are multiples of 8 on pairs of SMs with two-CTA MMAs).  A bf16 layer whose rank is no multiple of 8 takes the same
  * paths with A and B zero-padded to the next multiple of 8 inside the workspace (rewritten by every call).  Every other shape
  * runs on a plain CUDA-core path with the same results up to rounding order.  The workspace header
  * must have been zeroed once (meteora_workspace_init) before its first use; the kernels leave it
@@ -155,8 +155,8 @@ int meteora_linear_forward(const void* x, const void* W0, const void* A, const v
  *   y[m][T, d_out[m]] = W0[m] x + sum over module m's own top-k picks.
  * W0, A, B, Wg, y are HOST arrays of n_modules DEVICE pointers (1 <= n_modules <= METEORA_MAX_GROUP), d_out a host
  * array; T, d_in, N, r, k, dtype, temperature come from `shape` (its d_out is ignored).  Results per module are
- * those of meteora_linear_forward up to the rounding order of fp32 sums.  Decode batches (T <= 256, rank 8,
- * bf16, all modules together at most about 120 row tiles of 128) run as ONE kernel launch for the whole group;
+ * those of meteora_linear_forward up to the rounding order of fp32 sums.  Decode batches (T <= 256, rank a
+ * multiple of 8, bf16, all modules together at most about 120 row tiles of 128) run as ONE kernel launch for the whole group;
  * anything else runs module by module.  workspace: meteora_group_workspace_bytes(shape, d_out, n_modules) bytes of
  * device memory, its first 4 KB zeroed once (meteora_workspace_init); meteora_workspace_status reads the group's
  * status word.  meteora_group_workspace_routing returns where module `module` left its routing;

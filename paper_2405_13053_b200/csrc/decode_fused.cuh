@@ -1,11 +1,12 @@
-// Whole MeteoRA linear forward for a decode batch (one token tile, T <= 256, rank 8) as ONE kernel launch.
+// Whole MeteoRA linear forward for a decode batch (one token tile, T <= 256, rank a multiple of 8) as ONE kernel
+// launch, for one module or for up to four modules that share x.
 // Included by wgemm_tcgen05.cu after the device helpers it uses.
 //
 // The grid holds two kinds of CTAs, all resident at the same time (cooperative launch, no clusters):
 //   - main CTAs.  The base product W0 x is cut into units of one 128-row tile of W0 times kc k-steps, numbered
 //     tile by tile, and main CTA i takes the units [U*i/M, U*(i+1)/M): every SM streams the same number of
-//     bytes whatever the shape, and a CTA's range covers the tail of one tile and the head of the next (at most
-//     two segments; the host launches this kernel only when M >= row tiles).  Each segment runs through
+//     bytes whatever the shape, and a CTA's range covers the tail of one tile and the head of the next, or up
+//     to kMaxSeg tiles when a layer has more row tiles than CTAs (the host checks).  Each segment runs through
 //     TMA + tcgen05 into its own TMEM accumulator and goes to an fp32 scratch (it stays in L2).  When all the
 //     CTAs that share a tile have delivered, each of them sums its slice of the tile's rows in CTA order, adds
 //     the LoRA expand of those rows (Eq. 2: the B rows of every adapter wait in shared memory, the routing

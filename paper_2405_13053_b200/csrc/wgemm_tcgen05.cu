@@ -1145,7 +1145,7 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     return launch_wgemm(mA, mG, mX, mX, p, row_tiles, pl, false, st);
 }
 
-// Prefill batches on pairs of SMs (wgemm_pair.cuh): 256 x 256 tiles, rank 8, y stored by TMA.
+// Prefill batches on pairs of SMs (wgemm_pair.cuh): 256 x 256 tiles, ranks that are multiples of 8, y stored by TMA.
 struct PairPlan {
     bool ok;
     int stages, nblk, rb, epi_off;   // blocks of 8 expand columns (adapter, 8 rank entries): all, per round
