@@ -13,7 +13,7 @@
 //     arrives from the aux CTAs) and stores y;
 //   - a few aux CTAs on the SMs the main CTAs leave free: each computes a slice of the stacked shrink
 //     [A_0..A_{N-1}; Wg] x (every adapter's A_i x and the gate logits, Sec. 3.1) on the same main loop and
-//     writes it as an fp32 partial; once all partials are in, the aux CTAs share the tokens and run the
+//     sends its fp32 accumulator tile to scratch as one bulk copy; once all partials are in, the aux CTAs share the tokens and run the
 //     top-k selection and the softmax over the selected logits (Eq. 3), publishing topk_idx, topk_w, uw.
 // While the base product is short (W0 below about 50 MB) the main CTAs give the aux CTAs a head start of two
 // microseconds, so the 2 MB of the shrink are ahead of W0 in the memory queues (measured: a fixed delay does
@@ -37,7 +37,7 @@ struct DecodeModule {
     int32_t* topk_idx;     // selection results, written by aux CTAs, read by main CTAs
     float* topk_w;
     float* uw;
-    float* u_part;         // [aux_slices][T][ld_u] partial stacked shrink
+    float* u_part;         // [aux_slices][aux_tiles][T][128] partial stacked shrink, tile by tile as accumulated
 };
 struct DecodeMaps {
     CUtensorMap W0[kMaxGroup], A[kMaxGroup], At[kMaxGroup], G[kMaxGroup];
@@ -74,6 +74,17 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// One contiguous block from shared memory to global memory as a single bulk copy of the TMA engine (both
+// addresses 16-byte aligned, `bytes` a multiple of 16); returns when the writes are complete.  The data were
+// written to shared memory by ordinary stores: every writer ran fence.proxy.async before the barrier that
+// precedes this call.
+__device__ __forceinline__ void bulk_store_block(void* gdst, uint32_t smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 // Bounded wait until *ctr >= target; false if it did not happen within kWaitLimitCycles.
 __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
     const long long t0 = clock64();
@@ -89,22 +100,27 @@ __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
 // per lane, all loads in flight together) into `wbuf` (shared memory, ld_u floats), then top-k, softmax over
 // the picks (Eq. 3) and uw[t,j,:] = w_j * (A_{i_j} x) come from there.  The rank r is a multiple of 4; 256 floats
 // per 32 lanes and pass, further passes for more columns.
-__device__ __forceinline__ void select_token_wide(const float* u_part, int ld_u, int col_logits, int zsplits,
-                                                  size_t zstride, int t, int N, int r, int k, float inv_tau, int lane,
-                                                  float* wbuf, int32_t* topk_idx, float* topk_w, float* uw) {
+// The partials are laid out as the aux CTAs' accumulator tiles, u_part[slice][tile][T][128]: stacked row R of
+// [A; Wg] sits in tile R / 128 at R % 128, logit n in the gate tile at gate_row0 + n.
+__device__ __forceinline__ void select_token_wide(const float* u_part, int T, int tiles, int gate_tile, int gate_row0,
+                                                  int col_logits, int zsplits, int t, int N, int r, int k,
+                                                  float inv_tau, int lane, float* wbuf, int32_t* topk_idx,
+                                                  float* topk_w, float* uw) {
     constexpr int ZMAX = 16;
     const int n_a4 = N * r / 4, n_c4 = n_a4 + (N + 3) / 4;         // 16-byte chunks: shrink values, then logits
-    const float* row = u_part + (size_t)t * ld_u;
+    const size_t zstride = (size_t)tiles * T * kBM;
     for (int c0 = 0; c0 < n_c4; c0 += 64) {
         float4 acc[2];
         float4 v[2][ZMAX];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int c4 = c0 + h * 32 + lane;
-            const int col = c4 < n_a4 ? 4 * c4 : col_logits + 4 * (c4 - n_a4);
+            const int tile = c4 < n_a4 ? (4 * c4) / kBM : gate_tile;
+            const int within = c4 < n_a4 ? (4 * c4) % kBM : gate_row0 + 4 * (c4 - n_a4);
+            const float* src = u_part + ((size_t)tile * T + t) * kBM + within;
 #pragma unroll
             for (int z = 0; z < ZMAX; ++z)
-                v[h][z] = (c4 < n_c4 && z < zsplits) ? __ldcg(reinterpret_cast<const float4*>(row + z * zstride + col))
+                v[h][z] = (c4 < n_c4 && z < zsplits) ? __ldcg(reinterpret_cast<const float4*>(src + z * zstride))
                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
@@ -420,14 +436,12 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             if (!acc_ok && lane == 0) flag_error(p, 3, 600);
             acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
             tc_fence_after();
-            // accumulators straight to the partial buffer: lane = row, a warp writes 128 contiguous bytes
+            if (etid == 0 && tr_aux) FUSED_STAMP(p, 48, 9);
+            // The accumulator tile goes out as it is, [token][128 rows] fp32: staged in the idle ring (lane = row:
+            // a warp writes 128 contiguous bytes of shared memory), then ONE bulk copy by thread 0 below.  (Plain
+            // 4-byte stores straight to global memory took 2.7 us for the 64 KB of a 128-token tile.)
             const int trow = quad * 32 + lane;                                   // row of the tile
-            int col = -1;                                                        // column of u_part, -1: padding row
-            if (tile < d.a_tiles && tile * kBM + trow < d.a_rows && !(tile == d.gate_tile && trow >= d.gate_row0))
-                col = tile * kBM + trow;
-            if (tile == d.gate_tile && trow >= d.gate_row0 && trow < d.gate_row0 + p.N)
-                col = d.col_logits + trow - d.gate_row0;
-            float* dst = d.mod[am].u_part + (size_t)slice * p.T * d.ld_u + max(col, 0);
+            float* stage = reinterpret_cast<float*>(ring_ptr);
             for (int c = c_begin; c < c_end; c += 16) {
                 float v[16];
                 if (acc_ok) {
@@ -436,17 +450,18 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
 #pragma unroll
                     for (int i = 0; i < 16; ++i) v[i] = 0.f;
                 }
-                if (col >= 0) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (c + i < p.T) dst[(size_t)(c + i) * d.ld_u] = v[i];
-                }
+                for (int i = 0; i < 16; ++i) stage[(c + i) * kBM + trow] = v[i];
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");         // generic writes -> bulk copy reads
+            if (etid == 0 && tr_aux) FUSED_STAMP(p, 48, 10);
         }
         __syncwarp();
         __syncthreads();
         if (active) {
             if (threadIdx.x == 0) {
+                float* dst = d.mod[am].u_part + (((size_t)slice * d.aux_tiles + tile) * p.T) * kBM;
+                bulk_store_block(dst, ring, (uint32_t)p.T * kBM * 4u);
                 if (tr_aux) FUSED_STAMP(p, 48, 2);
                 __threadfence();
                 atomicAdd(d.ctr + 0, 1);
@@ -459,8 +474,8 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             for (int it = aux_id * nwarps + warp; it < d.n_mod * p.T; it += n_active * nwarps) {
                 const int sm = it / p.T, t = it - sm * p.T;
                 const DecodeModule& mo = d.mod[sm];
-                select_token_wide(mo.u_part, d.ld_u, d.col_logits, d.aux_slices, (size_t)p.T * d.ld_u, t, p.N, p.r,
-                                  p.k, d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
+                select_token_wide(mo.u_part, p.T, d.aux_tiles, d.gate_tile, d.gate_row0, d.col_logits, d.aux_slices, t,
+                                  p.N, p.r, p.k, d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
             }
             __syncthreads();
             if (threadIdx.x == 0) {
@@ -635,6 +650,9 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 tc_fence_after();
                 if (etid == 0 && tr_main && sg == nseg - 1) FUSED_STAMP(p, 32, 5);
                 float* part = d.part_g + (size_t)(d_tile[sg] + main_id) * part_stride;
+                // (plain stores: routed through the idle ring and one bulk copy, as the aux CTAs' tiles are, the
+                // delivery was 0 - 1.4 us slower at every shape and batch size measured: the copy's completion has
+                // to be awaited before the counter moves, while these stores drain behind the fence)
                 for (int c = c_begin; c < c_end; c += 16) {
                     float v[16];
                     if (acc_ok) {

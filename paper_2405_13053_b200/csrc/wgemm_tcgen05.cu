@@ -1409,6 +1409,8 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     if (stages < 2 || (size_t)stages * stage_bytes > avail) return fp;
     pl.stages = stages;
     const size_t ring_bytes = (size_t)stages * stage_bytes;
+    // the accumulator tiles leave through the idle ring (128 rows x BN tokens of fp32)
+    if (ring_bytes < (size_t)pl.BN * kBM * 4) return fp;
     // the aux CTAs' selection keeps one summed row of the stacked shrink per warp in the idle ring
     int col_logits = 0;
     if (ring_bytes < (size_t)(kThreads / 32) * tc_stacked_pitch(s, &col_logits) * sizeof(float)) return fp;
