@@ -265,8 +265,8 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "unit_split"     decode kernel's main CTAs: 0 = planner's choice, 1 = even unit ranges over all free SMs,
  *                    2 = whole row tiles per group of CTAs (falls back to the choice that fits)
  *   "aux_ctas"       > 0 = how many CTAs of the decode kernel the stacked shrink and the selection may take
- *   "no_hold"        head start of the decode kernel's aux CTAs: 0 = planner's choice (2100 ns for layers below
- *                    52 MB, none above), 1 = none, 64 = main CTAs wait for a counter, other = nanoseconds
+ *   "no_hold"        head start of the decode kernel's aux CTAs: 0 = planner's choice (1800 ns for layers below
+ *                    40 MB, none above), 1 = none, 64 = main CTAs wait for a counter, other = nanoseconds
  *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)
  *                    where the pairs cover a quarter of the SMs; 0 = never; 2 = wherever the shape allows
  * Unknown names return METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.

@@ -1517,14 +1517,16 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
     d.ld_u = mods[0].ws.ld_u;
     d.col_logits = mods[0].ws.col_logits;
     d.inv_tau = 1.0f / s.temperature;
-    // A head start for the aux CTAs' loads pays only while the base product is short: measured, 4096 -> 4096
-    // (34 MB) loses 0.5 - 1.4 us without it, 5120 -> 5120 (52 MB) gains 0.6 - 1.5 us without it (the routing is
-    // ready long before it is needed either way).  Knob no_hold: 1 = none, 64 = wait for the aux CTAs' counter,
-    // any other value = that many nanoseconds.
+    // A head start for the aux CTAs' loads pays only while the base product is short.  Measured, us per call at
+    // T = 1 / 32 / 128 with none, 1.3, 1.7, 2.1 us: 4096 -> 4096 (34 MB) 15.8 / 15.2 / 15.2 / 15.5, 17.8 / 17.3 /
+    // 16.5 / 16.9, 20.1 / 19.7 / 19.5 / 19.8; 4096 -> 5120 (42 MB) is best without one at T = 1 and 128 (15.9 against
+    // 16.7 - 17.0, 22.3 against 22.9 - 23.2), and so is 5120 -> 5120 (52 MB): there the routing is ready long before
+    // it is needed either way.  Knob no_hold: 1 = none, 64 = wait for the aux CTAs' counter, any other value =
+    // that many nanoseconds.
     {
         const int nh = tuning().no_hold;
-        const bool is_short = fp.w0_bytes < ((size_t)52 << 20);
-        d.hold = nh == 1 ? 0 : nh == 64 ? 1 : nh > 1 ? nh : is_short ? 2100 : 0;
+        const bool is_short = fp.w0_bytes < ((size_t)40 << 20);
+        d.hold = nh == 1 ? 0 : nh == 64 ? 1 : nh > 1 ? nh : is_short ? 1800 : 0;
     }
     d.ctr = status + 16;
     d.part_g = part_g;
