@@ -14,13 +14,13 @@
 //   - a few aux CTAs on the SMs the main CTAs leave free: each computes a slice of the stacked shrink
 //     [A_0..A_{N-1}; Wg] x (every adapter's A_i x and the gate logits, Sec. 3.1) on the same main loop and
 //     sends its fp32 accumulator tile to scratch as one bulk copy; once all partials are in, the aux CTAs share
-//     the tokens and run the top-k selection and the softmax over the selected logits (Eq. 3), publishing topk_idx, topk_w, uw.
+//     the tokens and run the top-k selection and the softmax over the selected logits (Eq. 3), publishing
+//     topk_idx, topk_w, uw.
 // While the base product is short (W0 below 40 MB) the main CTAs give the aux CTAs a head start of 1.8
 // microseconds, so the 2 MB of the shrink are ahead of W0 in the memory queues (measured: a fixed delay does
 // as well as waiting for a counter the aux CTAs bump, without the round trip); they need the routing only after
-// their main loop and the exchange
-// of the partial tiles.  Every wait is bounded; on expiry the status word is set and the kernel drains.  The
-// counters live in the workspace header and are re-armed by the last CTA to exit.
+// their main loop and the exchange of the partial tiles.  Every wait is bounded; on expiry the status word is
+// set and the kernel drains.  The counters live in the workspace header and are re-armed by the last CTA to exit.
 #pragma once
 
 namespace meteora {
