@@ -406,8 +406,9 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
         const int group_tiles = d.n_mod * d.aux_tiles;                       // (module, tile) pairs of the stacked shrinks
         const int am = active ? (aux_id % group_tiles) / d.aux_tiles : 0;    // module
         const int tile = (aux_id % group_tiles) % d.aux_tiles, slice = aux_id / group_tiles;
-        const int ks0 = active ? (int)(((long long)p.ksteps * slice) / d.aux_slices) : 0;
-        const int ks1 = active ? (int)(((long long)p.ksteps * (slice + 1)) / d.aux_slices) : 0;
+        // (k-steps x slices stays far below 2^31: 32-bit divisions, this is on the way to the first load)
+        const int ks0 = active ? (p.ksteps * slice) / d.aux_slices : 0;
+        const int ks1 = active ? (p.ksteps * (slice + 1)) / d.aux_slices : 0;
         const int niter = ks1 - ks0;
         const RingGeom geom = {ring, bar_base, x_tile_bytes, kWTileBytes + x_tile_bytes, d.aux_stages, 1, p.maps3d};
         const uint32_t bar_acc = bar_base + 2 * d.aux_stages * 8;
