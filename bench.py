@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "b6e28e3c64e6ed64", "bytes_per_launch": {"128": 38646699 + 172544}}
+NCU_TRAFFIC = {"kernel_sha": "52ec675d18e213f2", "bytes_per_launch": {"128": 38603776 + 133547}}
 
 
 def parse_args():
