@@ -506,10 +506,11 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                 } else if (d.hold > 1) {                         // a fixed head start for the aux CTAs, in nanoseconds
                     unsigned long long t0, t1;
                     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+                    int spins = 0;                                 // bounded like every other wait: 4096 x 64 ns at most
                     do {
                         __nanosleep(64);
                         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-                    } while (t1 - t0 < (unsigned long long)d.hold);
+                    } while (t1 - t0 < (unsigned long long)d.hold && ++spins < 4096);
                 }
                 if (tr_main) FUSED_STAMP(p, 32, 1);
                 int cur_tile = -1, row0 = 0;
