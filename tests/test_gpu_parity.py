@@ -298,6 +298,29 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
     check_forward(w, y_tol=1e-2)
 
 
+# Planner choices of the decode kernel forced the other way: the aux CTAs' head start (none, the counter wait,
+# a long timed one), how the units are dealt (even ranges over all free SMs: 5 row tiles on 128 CTAs share tiles
+# unevenly; whole tiles per CTA group), and fewer or more aux CTAs (slices of the stacked shrink).  The result
+# must not depend on any of them beyond the rounding order of the fp32 sums.
+@pytest.mark.parametrize("knob,value", [("no_hold", 1), ("no_hold", 64), ("no_hold", 5000), ("unit_split", 1),
+                                        ("unit_split", 2), ("aux_ctas", 4), ("aux_ctas", 40), ("kc", 1), ("stages", 2)])
+def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
+    w = workloads.make_workload("fused_knobs", T=70, d_in=1024, d_out=640, dtype="bf16", x_kind="normal", seed=1234,
+                                b_std=0.3)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    y0, i0, _ = run_forward(w)
+    mb.meteora_set_tuning(knob, value)
+    try:
+        assert "fused_decode" in mb.meteora_describe_plan(shape)
+        check_forward(w, y_tol=1e-2)
+        y1, i1, _ = run_forward(w)
+    finally:
+        mb.meteora_set_tuning(knob, 0)
+    same = np.all(i0 == i1, axis=1)          # another slicing of the shrink may flip a near-tie of two logits
+    assert same.mean() > 0.97
+    assert rel_l2(y1[same], y0[same]) < 4e-3
+
+
 # Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
 # one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
 # (257), a contraction length that is no multiple of 64, and adapters up to an odd count.  The stacked shrink of
