@@ -114,24 +114,25 @@ __device__ __forceinline__ void select_token_wide(const float* u_part, int T, in
         float4 v[2][ZMAX];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int c4 = c0 + h * 32 + lane;
+            // No branch around the loads (the compiler would wait for each one before taking the next): a chunk
+            // or a slice past the end is clamped to the last one, read again and left out of the sum below.
+            const int c4 = min(c0 + h * 32 + lane, n_c4 - 1);
             const int tile = c4 < n_a4 ? (4 * c4) / kBM : gate_tile;
             const int within = c4 < n_a4 ? (4 * c4) % kBM : gate_row0 + 4 * (c4 - n_a4);
             const float* src = u_part + ((size_t)tile * T + t) * kBM + within;
 #pragma unroll
             for (int z = 0; z < ZMAX; ++z)
-                v[h][z] = (c4 < n_c4 && z < zsplits) ? __ldcg(reinterpret_cast<const float4*>(src + z * zstride))
-                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[h][z] = __ldcg(reinterpret_cast<const float4*>(src + (size_t)min(z, zsplits - 1) * zstride));
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int z = 0; z < ZMAX; ++z) {
-                acc[h].x += v[h][z].x;
-                acc[h].y += v[h][z].y;
-                acc[h].z += v[h][z].z;
-                acc[h].w += v[h][z].w;
+                acc[h].x += z < zsplits ? v[h][z].x : 0.f;
+                acc[h].y += z < zsplits ? v[h][z].y : 0.f;
+                acc[h].z += z < zsplits ? v[h][z].z : 0.f;
+                acc[h].w += z < zsplits ? v[h][z].w : 0.f;
             }
             const int c4 = c0 + h * 32 + lane;
             const int col = c4 < n_a4 ? 4 * c4 : col_logits + 4 * (c4 - n_a4);
@@ -195,8 +196,8 @@ __device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, 
             const int t = it / nq, ql = it - t * nq;
             const size_t off = (size_t)t * kBM + (q0 + ql) * 4;
 #pragma unroll
-            for (int q = 0; q < C; ++q)
-                v[u][q] = q < c ? __ldcg(reinterpret_cast<const float4*>(parts[q] + off)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q = 0; q < C; ++q)                // no branch: parts[q] repeats the last real tile for q >= c
+                v[u][q] = __ldcg(reinterpret_cast<const float4*>(parts[q] + off));
         }
         if (routing_pending) {
             asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
@@ -210,10 +211,10 @@ __device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, 
             float4 acc = v[u][0];
 #pragma unroll
             for (int q = 1; q < C; ++q) {
-                acc.x += v[u][q].x;
-                acc.y += v[u][q].y;
-                acc.z += v[u][q].z;
-                acc.w += v[u][q].w;
+                acc.x += q < c ? v[u][q].x : 0.f;
+                acc.y += q < c ? v[u][q].y : 0.f;
+                acc.z += q < c ? v[u][q].z : 0.f;
+                acc.w += q < c ? v[u][q].w : 0.f;
             }
             for (int j = 0; j < k; ++j) {
                 const int slot = t * k + j;
