@@ -245,6 +245,34 @@ __device__ __forceinline__ void finish_rows(__nv_bfloat16* y, int d_out, int k, 
     }
 }
 
+// Rows of row tile `tile` that main CTA `main_id` finishes.  The tile is shared by the main CTAs owner(first
+// unit) .. owner(last unit), `c` of them from `first` on; contributor j takes the groups of 4 rows
+// [32 j / c, 32 (j + 1) / c).  Unit u belongs to main CTA ceil((u + 1) M / U) - 1.
+__device__ __forceinline__ void tile_share(int tile, int upt, int M, unsigned U, int main_id, int& first, int& c,
+                                           int& q0, int& nq) {
+    const unsigned x0 = (unsigned)(tile * upt), x1 = x0 + (unsigned)upt - 1u;
+    first = (int)(((x0 + 1u) * (unsigned)M + U - 1u) / U) - 1;
+    const int last = (int)(((x1 + 1u) * (unsigned)M + U - 1u) / U) - 1;
+    c = last - first + 1;
+    const int j = main_id - first;
+    q0 = 32 * j / c;
+    nq = 32 * (j + 1) / c - q0;
+}
+
+// A main CTA finishes its (one or two) tiles side by side, all B rows staged at once, if they fit the staging
+// buffer together; else tile after tile.  Both the epilogue warps and warp 0 ask.
+__device__ __forceinline__ bool finishes_side_by_side(int tile_a, int nseg, int upt, int M, unsigned U, int main_id,
+                                                      int N, int cpa, int slab_rows) {
+    if (nseg > 2) return false;
+    int words = 0;
+    for (int sg = 0; sg < nseg; ++sg) {
+        int first, c, q0, nq;
+        tile_share(tile_a + sg, upt, M, U, main_id, first, c, q0, nq);
+        words += N * cpa * 4 * nq;
+    }
+    return words <= N * cpa * slab_rows;
+}
+
 // Module that owns a row tile of the group-wide numbering.
 __device__ __forceinline__ int module_of_tile(const DecodeModule* mod, int n_mod, int tile) {
     int m = 0;
@@ -347,6 +375,19 @@ __device__ __forceinline__ bool fused_mma(const RingGeom& g, uint32_t tmem_base,
     return ok;
 }
 
+// One thread per CTA, once the CTA has read the workspace counters for the last time: counts the CTA out; the
+// last one re-arms the counters for the next call on this workspace.  (No fence between the stores: nobody
+// reads them before the next kernel, and the kernel boundary orders them.)
+__device__ __forceinline__ void count_cta_out(const DecodeParams& d) {
+    if (atomicAdd(d.ctr + 2, 1) == (int)gridDim.x - 1) {
+        d.ctr[0] = 0;
+        d.ctr[1] = 0;
+        d.ctr[3] = 0;
+        for (int i = 0; i < d.row_tiles; ++i) d.tile_ctr[i] = 0;
+        d.ctr[2] = 0;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads)
 k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmX1, const DecodeParams d) {
@@ -367,6 +408,7 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
     const bool is_aux = (int)blockIdx.x < d.n_aux;
     const int main_id = (int)blockIdx.x - d.n_aux;
     const int n_active = d.n_mod * d.aux_tiles * d.aux_slices;
+    bool counted_out = false;                      // thread 0: this CTA has been counted out before the end
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < nbar; ++s) mbar_init(bar_base + s * 8, 1);
@@ -582,8 +624,23 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                     }
                 }
                 __syncwarp();
-                asm volatile("bar.arrive 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
-                if (lane == 0 && tr_main) FUSED_STAMP(p, 32, 9);
+                // Side by side, every epilogue thread reaches barrier 2 after its last look at a tile counter,
+                // and this warp has seen the routing counter: from there on the CTA reads no counter, so it is
+                // counted out here, under the last step, instead of after it (the atomic's round trip and the
+                // re-arming by the last CTA then end before y is stored; at the end of the kernel they cost
+                // 1.5 - 2 us per call).  Tile after tile the later waits come after barrier 2: counted out at the end.
+                if (finishes_side_by_side(tile_a, nseg, upt, M, U, main_id, p.N, p.r >> 3, d.slab_rows)) {
+                    asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
+                    if (lane == 0) {
+                        if (tr_main) FUSED_STAMP(p, 32, 9);
+                        __threadfence();
+                        count_cta_out(d);
+                        counted_out = true;
+                    }
+                } else {
+                    asm volatile("bar.arrive 2, %0;" ::"n"(kEpiThreads + 32) : "memory");
+                    if (lane == 0 && tr_main) FUSED_STAMP(p, 32, 9);
+                }
             }
         } else if (warp == 1) {
             if (lane == 0) {
@@ -628,30 +685,23 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             // owner(last unit), in that order; contributor j of c takes the groups of 4 rows [32j/c, 32(j+1)/c).
             int d_tile[kMaxSeg], d_first[kMaxSeg], d_c[kMaxSeg], d_q0[kMaxSeg], d_nq[kMaxSeg], d_mod[kMaxSeg],
                 d_row0[kMaxSeg];
-            bool side_by_side = nseg <= 2;         // else the tiles are finished one after the other, B rows staged each time
             const int cpa = p.r >> 3;                                        // 16-byte words per B row
             uint4* slab = reinterpret_cast<uint4*>(epi + p.slab_off);
             uint4* d_slab[kMaxSeg];
             int slab_words = 0;
             for (int sg = 0; sg < nseg; ++sg) {
                 const int tile = tile_a + sg;
-                const unsigned x0 = (unsigned)(tile * upt), x1 = x0 + (unsigned)upt - 1u;
-                const int first = (int)(((x0 + 1u) * (unsigned)M + U - 1u) / U) - 1;
-                const int last = (int)(((x1 + 1u) * (unsigned)M + U - 1u) / U) - 1;
-                const int c = last - first + 1, j = main_id - first;
                 d_tile[sg] = tile;
-                d_first[sg] = first;
-                d_c[sg] = c;
-                d_q0[sg] = 32 * j / c;
-                d_nq[sg] = 32 * (j + 1) / c - d_q0[sg];
+                tile_share(tile, upt, M, U, main_id, d_first[sg], d_c[sg], d_q0[sg], d_nq[sg]);
                 d_slab[sg] = slab + slab_words;
                 d_mod[sg] = module_of_tile(d.mod, d.n_mod, tile);
                 d_row0[sg] = (tile - d.mod[d_mod[sg]].tile0) * kBM;          // the tile's first row inside its module
                 slab_words += p.N * cpa * 4 * d_nq[sg];
             }
             // side by side only if both tiles' rows fit the staging buffer together (a range longer than a
-            // tile's units can own one tile entirely and share another)
-            if (slab_words > p.N * cpa * d.slab_rows) side_by_side = false;
+            // tile's units can own one tile entirely and share another); else the tiles are finished one after
+            // the other, B rows staged each time
+            const bool side_by_side = finishes_side_by_side(tile_a, nseg, upt, M, U, main_id, p.N, cpa, d.slab_rows);
             if (side_by_side) {
                 // B rows of the CTA's slices for every adapter: no routing needed yet
                 for (int sg = 0; sg < nseg; ++sg)
@@ -754,17 +804,7 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
                      "r"((uint32_t)p.tmem_cols)
                      : "memory");
     }
-    if (threadIdx.x == 0) {
-        // the last CTA out re-arms the counters for the next call on this workspace
-        if (atomicAdd(d.ctr + 2, 1) == (int)gridDim.x - 1) {
-            d.ctr[0] = 0;
-            d.ctr[1] = 0;
-            d.ctr[3] = 0;
-            for (int i = 0; i < d.row_tiles; ++i) d.tile_ctr[i] = 0;
-            __threadfence();
-            d.ctr[2] = 0;
-        }
-    }
+    if (threadIdx.x == 0 && !counted_out) count_cta_out(d);
 }
 
 }  // namespace meteora
