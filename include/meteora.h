@@ -267,6 +267,11 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "aux_ctas"       > 0 = how many CTAs of the decode kernel the stacked shrink and the selection may take
  *   "no_hold"        head start of the decode kernel's aux CTAs: 0 = planner's choice (1800 ns for layers below
  *                    40 MB, none above), 1 = none, 64 = main CTAs wait for a counter, other = nanoseconds
+ *   "pdl_decode"     default 1 = the decode kernel is launched with programmatic stream serialization on top of
+ *                    the co-residency guarantee: the next launch's CTAs take an SM as soon as this kernel's CTA
+ *                    has left it and set up under its tail (the kernel reads nothing before the launch ahead of
+ *                    it has completed); 0 = plain stream order.  If the driver refuses the pair of attributes
+ *                    the kernel is launched without it (pdl_decode_refused in the plan string counts these).
  *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)
  *                    where the pairs cover a quarter of the SMs; 0 = never; 2 = wherever the shape allows
  * Unknown names return METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.

@@ -431,8 +431,9 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
     char tmp[512];
     const bool pad = rank_pad_applies(*shape) && !tuning().force_simt;
     describe_plan(pad ? rank_padded(*shape) : *shape, tmp, sizeof(tmp));
-    snprintf(buf, buf_bytes, "%s%s fused_refused=%d", tmp, pad ? " rank_padded_to_multiple_of_8" : "",
-             tuning().fused_refused);
+    snprintf(buf, buf_bytes, "%s%s fused_refused=%d pdl_decode=%d pdl_decode_refused=%d", tmp,
+             pad ? " rank_padded_to_multiple_of_8" : "", tuning().fused_refused, tuning().pdl_decode,
+             tuning().pdl_decode_refused);
     return METEORA_OK;
 }
 
@@ -455,6 +456,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "unit_split")) t.unit_split = value;
     else if (!strcmp(name, "aux_ctas")) t.aux_ctas = value;
     else if (!strcmp(name, "pair")) t.pair = value;
+    else if (!strcmp(name, "pdl_decode")) t.pdl_decode = value;
     else return METEORA_ERR_INVALID_ARG;
     return METEORA_OK;
 }

@@ -67,6 +67,7 @@ struct DecodeParams {
     int row_tiles;         // of all modules together
     int slab_rows;         // rows of B (of every adapter) the staging buffer of a main CTA holds
     int trace_call;        // trace builds: which record of the trace buffer this launch fills
+    int pdl;               // launched with programmatic stream serialization: trigger the next launch, wait for the previous
 };
 
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
@@ -425,6 +426,13 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+    if (d.pdl) {
+        // Programmatic dependent launch: the next kernel on the stream may take an SM as soon as its CTA of this
+        // kernel has left, and run its own set-up (barriers, TMEM) under our tail; up to here this kernel has
+        // touched no global memory, and it touches none before the kernel ahead of it has completed.
+        if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
     const uint32_t idesc = instr_desc_bf16(p.BN);
     const int quad = warp & 3;
     const int etid = threadIdx.x - 64;

@@ -1539,16 +1539,39 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
-    attr[0].val.cooperative = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (tuning().coop) {
+        attr[na].id = cudaLaunchAttributeCooperative;     // the CTAs wait on one another: all must be resident
+        attr[na].val.cooperative = 1;
+        ++na;
+    }
+    // Programmatic dependent launch on top (knob pdl_decode): the next launch's CTAs move in as this kernel's leave.
+    // If the driver does not take the two attributes together, the kernel is launched without it from then on.
+    static bool pdl_accepted = true;
+    const bool want_pdl = tuning().pdl_decode != 0 && pdl_accepted;
+    if (want_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = tuning().coop ? 1 : 0;
+    cfg.numAttrs = na;
+    d.pdl = want_pdl ? 1 : 0;
 #ifdef METEORA_TRACE
     static int trace_calls = 0;
     d.trace_call = trace_calls++;
 #endif
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_fused, maps, mX, mX1, d));
+    cudaError_t err = cudaLaunchKernelEx(&cfg, k_decode_fused, maps, mX, mX1, d);
+    if (err != cudaSuccess && want_pdl) {
+        cudaGetLastError();
+        pdl_accepted = false;
+        tuning().pdl_decode_refused += 1;
+        cfg.numAttrs = na - 1;
+        d.pdl = 0;
+        err = cudaLaunchKernelEx(&cfg, k_decode_fused, maps, mX, mX1, d);
+    }
+    return cuda_status(err);
 }
 
 int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,

@@ -321,6 +321,47 @@ def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
     assert rel_l2(y1[same], y0[same]) < 4e-3
 
 
+# Back-to-back decode calls in which every call reads what the call before it wrote (y of layer i is x of layer
+# i + 1, as in a decoder stack), launched without any synchronisation in between.  The decode kernel is launched
+# with programmatic stream serialization (its CTAs may move onto an SM as soon as the previous kernel's CTA has
+# left it): it must not touch the previous result before that kernel has completed.  The chain with the
+# attribute and without it (knob pdl_decode) must agree bit for bit, and so must a repeat.
+@pytest.mark.parametrize("T,d", [(40, 512), (130, 1024)])
+def test_dependent_decode_calls_back_to_back(T, d):
+    layers = [workloads.make_workload(f"stack{i}", T=T, d_in=d, d_out=d, dtype="bf16", x_kind="normal",
+                                      seed=4100 + 7 * i, b_std=0.3) for i in range(4)]
+    dev = [to_dev(w, "W0", "A", "B", "Wg") for w in layers]
+    x0 = to_dev(layers[0], "x")[0]
+    shape = mb.make_shape(T, d, d, layers[0].N, layers[0].r, layers[0].k, torch.bfloat16)
+    assert "fused_decode" in mb.meteora_describe_plan(shape)
+    wss = [mb.alloc_workspace(shape) for _ in layers]
+
+    def run_stack():
+        h = x0
+        for (W0, A, B, Wg), ws in zip(dev, wss):
+            h = mb.meteora_linear_forward(h, W0, A, B, Wg, layers[0].k, workspace=ws)
+        torch.cuda.synchronize()
+        for ws in wss:
+            assert mb.meteora_workspace_status(ws) == 0
+        return h.float().cpu().numpy()
+
+    results = {}
+    try:
+        for pdl in (1, 0, 1):
+            mb.meteora_set_tuning("pdl_decode", pdl)
+            results.setdefault(pdl, []).append(run_stack())
+    finally:
+        mb.meteora_set_tuning("pdl_decode", 1)
+    assert np.all(np.isfinite(results[1][0]))
+    np.testing.assert_array_equal(results[1][0], results[0][0])
+    np.testing.assert_array_equal(results[1][0], results[1][1])
+    # and layer 0 alone against the oracle, as everywhere else
+    y0 = mb.meteora_linear_forward(x0, *dev[0], layers[0].k, workspace=wss[0], return_routing=True)
+    ref = oracle.linear_forward_routed(layers[0]["x"], layers[0]["W0"], layers[0]["A"], layers[0]["B"], layers[0]["Wg"],
+                                       y0[1].cpu().numpy())
+    assert rel_l2(y0[0].float().cpu().numpy(), ref) <= 1e-2
+
+
 # Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
 # one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
 # (257), a contraction length that is no multiple of 64, and adapters up to an odd count.  The stacked shrink of
