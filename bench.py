@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "733af14142808e84", "bytes_per_launch": {"128": 38604885 + 106667}}
+NCU_TRAFFIC = {"kernel_sha": "803c244ee550aea7", "bytes_per_launch": {"128": 38604885 + 114347}}
 
 
 def parse_args():

@@ -267,6 +267,8 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "aux_ctas"       > 0 = how many CTAs of the decode kernel the stacked shrink and the selection may take
  *   "no_hold"        head start of the decode kernel's aux CTAs: 0 = planner's choice (1800 ns for layers below
  *                    40 MB, none above), 1 = none, 64 = main CTAs wait for a counter, other = nanoseconds
+ *   "hold_after"     ring stages of W0 the decode kernel's main CTAs request before that head start: 0 = planner's
+ *                    choice (one stage for layers of 20 to 40 MB, none otherwise), -1 = none, n > 0 = n stages
  *   "pdl_decode"     default 1 = the decode kernel is launched with programmatic stream serialization on top of
  *                    the co-residency guarantee: the next launch's CTAs take an SM as soon as this kernel's CTA
  *                    has left it and set up under its tail (the kernel reads nothing before the launch ahead of

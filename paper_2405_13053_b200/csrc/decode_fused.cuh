@@ -60,6 +60,7 @@ struct DecodeParams {
     int bar_stages;        // barriers are laid out for max(main stages, aux stages) ring slots
     int ld_u, col_logits;
     float inv_tau;
+    int hold_after;        // ring stages the main CTAs request before that head start (0: none)
     int hold;              // 1: main CTAs start loading only after the aux CTAs have issued their first loads; > 1: after that many nanoseconds
     int32_t* ctr;          // [0] aux partials written, [1] selections published, [2] CTAs exited, [3] aux loads issued
     float* part_g;         // [row tile + main CTA][BN][128] fp32 partial accumulator tiles of the base product
@@ -552,22 +553,26 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             if (lane == 0) {
                 // let the stacked shrink get its loads into the memory queues first
                 bool ok = true;
-                if (d.hold == 1) {
-                    ok = wait_counter(d.ctr + 3, n_active);
-                } else if (d.hold > 1) {                         // a fixed head start for the aux CTAs, in nanoseconds
-                    unsigned long long t0, t1;
-                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-                    int spins = 0;                                 // bounded like every other wait: 4096 x 64 ns at most
-                    do {
-                        __nanosleep(64);
-                        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-                    } while (t1 - t0 < (unsigned long long)d.hold && ++spins < 4096);
-                }
+                unsigned long long t0 = 0;
+                if (d.hold > 1) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
                 if (tr_main) FUSED_STAMP(p, 32, 1);
                 int cur_tile = -1, row0 = 0;
                 const CUtensorMap* tmW0 = &maps.W0[0];
                 int tile = tile_a, kpos = u0 - tile_a * upt, st = 0, round = 0;
                 for (int it = 0; it < n_it && ok; ++it) {
+                    if (it == d.hold_after) {                    // the first hold_after stages go out at once
+                        if (d.hold == 1) {
+                            ok = wait_counter(d.ctr + 3, n_active);
+                            if (!ok) break;
+                        } else if (d.hold > 1) {                 // a fixed head start for the aux CTAs, in nanoseconds
+                            unsigned long long t1;
+                            int spins = 0;                         // bounded like every other wait: 4096 x 64 ns at most
+                            do {
+                                __nanosleep(64);
+                                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+                            } while (t1 - t0 < (unsigned long long)d.hold && ++spins < 4096);
+                        }
+                    }
                     if (round > 0) ok = mbar_wait(bar_base + (geom.stages + st) * 8, (round & 1) ^ 1);
                     if (!ok) break;
                     const uint32_t full = bar_base + st * 8, dst = ring + st * stage_bytes;

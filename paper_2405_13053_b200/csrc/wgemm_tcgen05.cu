@@ -1527,6 +1527,12 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
         const int nh = tuning().no_hold;
         const bool is_short = fp.w0_bytes < ((size_t)40 << 20);
         d.hold = nh == 1 ? 0 : nh == 64 ? 1 : nh > 1 ? nh : is_short ? 1800 : 0;
+        // The first ring stage of W0 may go out before that head start: measured with 1 stage ahead, 4096 -> 4096
+        // (34 MB) 14.0 -> 13.6 / 14.8 -> 14.6 / 17.9 -> 17.5 us at T = 1 / 32 / 128, 4096 -> 1024 (8 MB) 11.8 -> 12.0 /
+        // 13.1 -> 13.4 / 15.4 -> 15.9 us; two stages ahead lose the gain again.  Taken from 20 MB of W0 up.
+        // Knob hold_after: 0 = this choice, -1 = none, n > 0 = n stages.
+        const int ha = tuning().hold_after;
+        d.hold_after = ha > 0 ? ha : ha < 0 ? 0 : (d.hold > 0 && fp.w0_bytes >= ((size_t)20 << 20)) ? 1 : 0;
     }
     d.ctr = status + 16;
     d.part_g = part_g;
