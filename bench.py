@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "803c244ee550aea7", "bytes_per_launch": {"128": 38604885 + 114347}}
+NCU_TRAFFIC = {"kernel_sha": "f561b4eaea50329b", "bytes_per_launch": {"128": 38605056 + 145067}}
 
 
 def parse_args():
@@ -51,7 +51,7 @@ def parse_args():
     ap.add_argument("--launch", choices=["graph", "stream"], default="graph")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target length of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-streams", type=int, default=3,
+    ap.add_argument("--e2e-streams", type=int, default=4,
                     help="streams the end-to-end step spreads its independent modules over")
     ap.add_argument("--sweep", action="store_true",
                     help="time every (shape, T) of configs 1-3 instead of the headline step; one JSON line each")
@@ -265,7 +265,7 @@ def run_ours(args):
         for m in mods:
             call_device(m)
 
-    # End-to-end step: the modules are independent, so their calls go round-robin onto three streams and the
+    # End-to-end step: the modules are independent, so their calls go round-robin onto a few streams and the
     # host-to-device copy of one module, the kernel of another and the device-to-host copy of a third overlap
     # (the two copy engines and the SMs); every stream is joined before the step ends.
     e2e_streams = [torch.cuda.Stream() for _ in range(max(1, args.e2e_streams))]

@@ -1373,6 +1373,20 @@ static FusedPlan make_fused_plan(const meteora_shape_t& s, const int* d_outs, in
     if (tn.splits > 0 && tn.splits * fp.row_tiles <= m_max) n_main = std::min(tn.splits, 8) * fp.row_tiles;
     n_main = (int)std::min<long long>(n_main, units);
     if (n_main < 1 || (units + 1) * (n_main + 1) >= (1LL << 31)) return fp;   // 32-bit unit arithmetic on the device
+    // SMs the main CTAs leave idle anyway (narrow layers: 8 row tiles use 64 main CTAs) go to the stacked shrink
+    // as further slices: its loads are the head of the chain that ends in the routing.  Measured at 4096 -> 1024
+    // and 5120 -> 1024, 20 -> 32 aux CTAs: 11.9 -> 11.3 / 13.4 -> 12.8 / 16.0 -> 15.5 us at T = 1 / 32 / 128.  (Where
+    // the aux CTAs would take SMs from the main CTAs, 4096 -> 2048 and wider, more of them lose at 128 tokens.)
+    // A few spare SMs do not pay: 120 main CTAs + 8 more aux CTAs (14 slices instead of 10) cost 0.2 - 0.5 us at
+    // 5120 -> 5120 and 13824 -> 5120 (more partial copies for the selection to add), so only the full 16 slices are taken.
+    if (tn.aux_ctas == 0) {
+        const int spare = sms - n_main - fp.n_aux;
+        const int full = std::min(ksteps, 16);
+        if (fp.aux_slices < full && fp.aux_slices + spare / group_tiles >= full) {
+            fp.aux_slices = full;
+            fp.n_aux = group_tiles * fp.aux_slices;
+        }
+    }
     // Row tiles a CTA's unit range can touch: 1 for whole tiles per CTA group, 2 while a range is no longer than a
     // tile's units, more beyond that (one TMEM accumulator of BN columns each: at most 4, and 512 columns in all).
     const long long range = (units + n_main - 1) / n_main;
