@@ -270,9 +270,9 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "hold_after"     ring stages of W0 the decode kernel's main CTAs request before that head start: 0 = planner's
  *                    choice (one stage for layers of 20 to 40 MB, none otherwise), -1 = none, n > 0 = n stages
  *   "pdl_decode"     default 1 = the decode kernel is launched with programmatic stream serialization on top of
- *                    the co-residency guarantee: the next launch's CTAs take an SM as soon as this kernel's CTA
- *                    has left it and set up under its tail (the kernel reads nothing before the launch ahead of
- *                    it has completed); 0 = plain stream order.  If the driver refuses the pair of attributes
+ *                    the co-residency guarantee: the next launch is processed and its CTAs set up under this
+ *                    kernel's tail (the kernel touches no global memory before the launch ahead of it has
+ *                    completed); 0 = plain stream order.  If the driver refuses the pair of attributes
  *                    the kernel is launched without it (pdl_decode_refused in the plan string counts these).
  *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)
  *                    where the pairs cover a quarter of the SMs; 0 = never; 2 = wherever the shape allows

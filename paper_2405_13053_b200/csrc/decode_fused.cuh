@@ -428,9 +428,9 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
     if (d.pdl) {
-        // Programmatic dependent launch: the next kernel on the stream may take an SM as soon as its CTA of this
-        // kernel has left, and run its own set-up (barriers, TMEM) under our tail; up to here this kernel has
-        // touched no global memory, and it touches none before the kernel ahead of it has completed.
+        // Programmatic dependent launch: the next kernel on the stream is launched and runs its own set-up
+        // (barriers, TMEM) under this kernel's tail; up to here this kernel has touched no global memory, and it
+        // touches none before the kernel ahead of it has completed.
         if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }

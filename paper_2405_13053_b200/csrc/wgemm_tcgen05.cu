@@ -1566,7 +1566,7 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
         attr[na].val.cooperative = 1;
         ++na;
     }
-    // Programmatic dependent launch on top (knob pdl_decode): the next launch's CTAs move in as this kernel's leave.
+    // Programmatic dependent launch on top (knob pdl_decode): the next launch is processed under this kernel's tail.
     // If the driver does not take the two attributes together, the kernel is launched without it from then on.
     static bool pdl_accepted = true;
     const bool want_pdl = tuning().pdl_decode != 0 && pdl_accepted;
