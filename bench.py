@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "f561b4eaea50329b", "bytes_per_launch": {"128": 38605056 + 145067}}
+NCU_TRAFFIC = {"kernel_sha": "36438807b8c24de5", "bytes_per_launch": {"128": 38620416 + 64597}}
 
 
 def parse_args():

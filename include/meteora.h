@@ -269,6 +269,9 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *                    40 MB, none above), 1 = none, 64 = main CTAs wait for a counter, other = nanoseconds
  *   "hold_after"     ring stages of W0 the decode kernel's main CTAs request before that head start: 0 = planner's
  *                    choice (one stage for layers of 20 to 40 MB, none otherwise), -1 = none, n > 0 = n stages
+ *   "narrow_select"  selection inside the decode kernel: 0 = by batch size (from 16 tokens up the logits are read
+ *                    first and then only the picks' shrink values, below that the whole stacked row at once),
+ *                    1 = always the former, -1 = always the latter; same results bit for bit
  *   "pdl_decode"     default 1 = the decode kernel is launched with programmatic stream serialization on top of
  *                    the co-residency guarantee: the next launch is processed and its CTAs set up under this
  *                    kernel's tail (the kernel touches no global memory before the launch ahead of it has

@@ -458,6 +458,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "pair")) t.pair = value;
     else if (!strcmp(name, "pdl_decode")) t.pdl_decode = value;
     else if (!strcmp(name, "hold_after")) t.hold_after = value;
+    else if (!strcmp(name, "narrow_select")) t.narrow_select = value;
     else return METEORA_ERR_INVALID_ARG;
     return METEORA_OK;
 }

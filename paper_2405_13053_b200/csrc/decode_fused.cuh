@@ -68,6 +68,7 @@ struct DecodeParams {
     int row_tiles;         // of all modules together
     int slab_rows;         // rows of B (of every adapter) the staging buffer of a main CTA holds
     int trace_call;        // trace builds: which record of the trace buffer this launch fills
+    int narrow_select;     // selection in two round trips (logits, then the picks' shrink values) instead of one wide one
     int pdl;               // launched with programmatic stream serialization: trigger the next launch, wait for the previous
 };
 
@@ -160,6 +161,54 @@ __device__ __forceinline__ void select_token_wide(const float* u_part, int T, in
         if (c < k * r) uw[(size_t)t * k * r + c] = wj * wbuf[ij * r + q];
     }
     __syncwarp();
+}
+
+// The same selection in two round trips that move far less: first the N logits of the token from every slice
+// (lane n owns logit n, n + 32, ...), top-k and softmax, then only the k * r shrink values of the picks.  A token
+// costs (N + k r) * slices floats instead of the whole stacked row (N r + N) * slices: 1.8 KB instead of 10 KB
+// at N = 28, r = 8, k = 2 and 10 slices, which is what counts once every aux warp has a token (the aux SMs
+// take in the partial copies at 50 - 60 GB/s each).  Same sums in the same slice order as select_token_wide.
+__device__ __forceinline__ void select_token_narrow(const float* u_part, int T, int tiles, int gate_tile, int gate_row0,
+                                                    int zsplits, int t, int N, int r, int k, float inv_tau, int lane,
+                                                    int32_t* topk_idx, float* topk_w, float* uw) {
+    constexpr int ZMAX = 16;
+    const size_t zstride = (size_t)tiles * T * kBM;
+    float v[kSelVals];
+    const float* grow = u_part + ((size_t)gate_tile * T + t) * kBM + gate_row0;
+#pragma unroll
+    for (int i = 0; i < kSelVals; ++i) {
+        v[i] = 0.f;
+        if (32 * i < N) {                                   // uniform across the warp
+            const float* src = grow + min(lane + 32 * i, N - 1);
+            float part[ZMAX];
+#pragma unroll
+            for (int z = 0; z < ZMAX; ++z) part[z] = __ldcg(src + (size_t)min(z, zsplits - 1) * zstride);
+#pragma unroll
+            for (int z = 0; z < ZMAX; ++z) v[i] += z < zsplits ? part[z] : 0.f;
+        }
+    }
+    int idx;
+    float w;
+    warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
+    if (lane < k) {
+        topk_idx[(size_t)t * k + lane] = idx;
+        topk_w[(size_t)t * k + lane] = w;
+    }
+    for (int c0 = 0; c0 < k * r; c0 += 32) {
+        const int c = min(c0 + lane, k * r - 1);
+        const int j = c / r, q = c - j * r;
+        const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
+        const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
+        const int R = ij * r + q;                           // row of the stacked matrix [A_0 .. A_{N-1}]
+        const float* src = u_part + ((size_t)(R / kBM) * T + t) * kBM + (R % kBM);
+        float part[ZMAX];
+#pragma unroll
+        for (int z = 0; z < ZMAX; ++z) part[z] = __ldcg(src + (size_t)min(z, zsplits - 1) * zstride);
+        float u = 0.f;
+#pragma unroll
+        for (int z = 0; z < ZMAX; ++z) u += z < zsplits ? part[z] : 0.f;
+        if (c0 + lane < k * r) uw[(size_t)t * k * r + c0 + lane] = wj * u;
+    }
 }
 
 // B rows [row0, row0 + nrows) of every adapter (8 bf16 = 16 bytes each) as slab[e][row % 4][row / 4], so that
@@ -527,8 +576,12 @@ k_decode_fused(const __grid_constant__ DecodeMaps maps, const __grid_constant__ 
             for (int it = aux_id * nwarps + warp; it < d.n_mod * p.T; it += n_active * nwarps) {
                 const int sm = it / p.T, t = it - sm * p.T;
                 const DecodeModule& mo = d.mod[sm];
-                select_token_wide(mo.u_part, p.T, d.aux_tiles, d.gate_tile, d.gate_row0, d.col_logits, d.aux_slices, t,
-                                  p.N, p.r, p.k, d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
+                if (d.narrow_select)
+                    select_token_narrow(mo.u_part, p.T, d.aux_tiles, d.gate_tile, d.gate_row0, d.aux_slices, t, p.N, p.r,
+                                        p.k, d.inv_tau, lane, mo.topk_idx, mo.topk_w, mo.uw);
+                else
+                    select_token_wide(mo.u_part, p.T, d.aux_tiles, d.gate_tile, d.gate_row0, d.col_logits, d.aux_slices, t,
+                                      p.N, p.r, p.k, d.inv_tau, lane, wbuf, mo.topk_idx, mo.topk_w, mo.uw);
             }
             __syncthreads();
             if (threadIdx.x == 0) {

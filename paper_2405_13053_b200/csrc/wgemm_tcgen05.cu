@@ -1474,6 +1474,11 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
                     pl.lora_mma ? "mma" : "simt");
 }
 
+// (module, token) items from which the selection reads in two narrow round trips.  Measured, narrow against wide, us
+// per call at T = 1 / 16 / 32 / 64 / 128 / 256: 4096 -> 4096 +0.25 / -0.25 / -0.1 / -0.4 / -0.35 / -1.05; 4096 -> 1024
+// 0 / -0.2 / -0.1 / -0.4 / -0.4 / -0.4; 5120 -> 5120 0 / -0.4 / -0.2 / 0 / +0.1 / +0.2; 13824 -> 5120 within +-0.2.
+constexpr int kNarrowSelectTokens = 16;
+
 int launch_decode_group(const void* x, const GroupModule* mods, int G, const meteora_shape_t& s, int32_t* status,
                         float* part_g, int32_t* tile_ctr, cudaStream_t st) {
     int d_outs[kMaxGroup] = {};
@@ -1547,6 +1552,11 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
         // Knob hold_after: 0 = this choice, -1 = none, n > 0 = n stages.
         const int ha = tuning().hold_after;
         d.hold_after = ha > 0 ? ha : ha < 0 ? 0 : (d.hold > 0 && fp.w0_bytes >= ((size_t)20 << 20)) ? 1 : 0;
+    }
+    {
+        // knob narrow_select: 0 = by batch size, 1 = always, -1 = never
+        const int ns = tuning().narrow_select;
+        d.narrow_select = ns > 0 ? 1 : ns < 0 ? 0 : (G * s.T >= kNarrowSelectTokens ? 1 : 0);
     }
     d.ctr = status + 16;
     d.part_g = part_g;

@@ -304,7 +304,8 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
 # must not depend on any of them beyond the rounding order of the fp32 sums.
 @pytest.mark.parametrize("knob,value", [("no_hold", 1), ("no_hold", 64), ("no_hold", 5000), ("unit_split", 1),
                                         ("unit_split", 2), ("aux_ctas", 4), ("aux_ctas", 40), ("kc", 1), ("stages", 2),
-                                        ("hold_after", 1), ("hold_after", 3)])
+                                        ("hold_after", 1), ("hold_after", 3), ("narrow_select", -1),
+                                        ("narrow_select", 1)])
 def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
     w = workloads.make_workload("fused_knobs", T=70, d_in=1024, d_out=640, dtype="bf16", x_kind="normal", seed=1234,
                                 b_std=0.3)
