@@ -323,6 +323,27 @@ def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
     assert rel_l2(y1[same], y0[same]) < 4e-3
 
 
+# The decode kernel's selection has two forms (the whole stacked row of a token in one round trip, or the logits
+# first and then only the picks' shrink values); both add the partial copies in slice order, so routing, weights and
+# y must agree bit for bit, for one pick and several, rank 8 and above, few and many adapters.
+@pytest.mark.parametrize("T,N,r,k", [(70, 28, 8, 2), (9, 28, 8, 1), (40, 40, 16, 3), (33, 128, 8, 4), (20, 28, 32, 8)])
+def test_both_forms_of_the_selection_agree_bit_for_bit(T, N, r, k):
+    w = workloads.make_workload("select_forms", T=T, d_in=1024, d_out=384, N=N, r=r, k=k, dtype="bf16",
+                                x_kind="normal", seed=5200 + T, b_std=0.3)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    out = {}
+    try:
+        for form in (-1, 1):
+            mb.meteora_set_tuning("narrow_select", form)
+            assert "fused_decode" in mb.meteora_describe_plan(shape)
+            out[form] = run_forward(w)
+    finally:
+        mb.meteora_set_tuning("narrow_select", 0)
+    for a, b in zip(out[-1], out[1]):
+        np.testing.assert_array_equal(a, b)
+    check_forward(w, y_tol=1e-2)
+
+
 # Back-to-back decode calls in which every call reads what the call before it wrote (y of layer i is x of layer
 # i + 1, as in a decoder stack), launched without any synchronisation in between.  The decode kernel is launched
 # with programmatic stream serialization (its CTAs may move onto an SM as soon as the previous kernel's CTA has
