@@ -107,9 +107,8 @@ int meteora_lora_delta(const void* x, const void* A, const void* B, const int32_
  * way the library is embedded, not for the method.)
  *
  * Who it is for: callers that cannot allocate device memory at the point where they need the LoRA term,
- * and so have no workspace to pass: code running inside another framework's allocator lock or stream
- * callback, serving loops whose memory pool is frozen after start-up, bindings that can launch but not
- * allocate.  The scratch that meteora_lora_delta takes from its workspace (the shrunk activations, T*k*r
+ * and so have no workspace to pass: code running while another framework holds its allocator lock,
+ * serving loops whose memory pool is frozen after start-up, bindings that can launch but not allocate.  The scratch that meteora_lora_delta takes from its workspace (the shrunk activations, T*k*r
  * floats) lives here in a fixed device array inside the library, METEORA_STATIC_SCRATCH_FLOATS floats
  * (256 KB) on every GPU that loads the library, for the life of the process.  The call allocates nothing
  * and frees nothing.
@@ -119,7 +118,11 @@ int meteora_lora_delta(const void* x, const void* A, const void* B, const int32_
  *   - T * k * r > METEORA_STATIC_SCRATCH_FLOATS returns METEORA_ERR_UNSUPPORTED_SHAPE and launches nothing;
  *     larger problems need meteora_lora_delta and a workspace.
  *   - The first call on each device looks up the device address of the built-in array (a runtime query,
- *     with that device current).  Make that first call outside any stream capture.
+ *     with that device current; it may make the runtime load the module, which can allocate driver memory
+ *     and synchronise).  Make that first call at start-up, in a warm-up step: outside any stream capture
+ *     and outside the region in which allocation is forbidden.  Later calls on that device only launch.
+ *   - `stream` must belong to the device that is current when the call is made: the array's address is
+ *     looked up for the current device.
  *   - All calls on a device share the one array and it keeps whatever the previous call left in it.  No
  *     part of it needs clearing (every value is written before it is read within a call), but two calls
  *     whose kernels can overlap on the GPU (different streams, no ordering between them) race on it: keep

@@ -1,11 +1,13 @@
 // meteora_lora_delta_static: the LoRA term of the layer for callers that cannot hand the library any scratch.
 //
 // meteora_lora_delta keeps the shrunk activations u[T*k, r] (fp32) in a caller-provided workspace.  Some
-// callers cannot provide one: a plug-in that runs inside another framework's stream callback or memory-pool
-// critical section, a real-time serving loop whose allocator is frozen after start-up, a driver written in a
-// language binding that exposes launches but no allocator.  For them this file keeps that scratch in a
+// callers cannot provide one: a plug-in that runs inside another framework's memory-pool critical section, a
+// real-time serving loop whose allocator is frozen after start-up, a driver written in a language binding
+// that exposes launches but no allocator.  For them this file keeps that scratch in a
 // file-scope device array of fixed size.  Every GPU that loads the library holds the array (256 KB) until the
 // process exits.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace meteora {
@@ -14,18 +16,23 @@ namespace meteora {
 static __device__ __align__(256) float g_static_u[METEORA_STATIC_SCRATCH_FLOATS];
 
 // In host code `g_static_u` is only a handle for the runtime, not a device address; the address a kernel can
-// use comes from cudaGetSymbolAddress, once per device, with that device current.
+// use comes from cudaGetSymbolAddress, once per device, with that device current (the caller's stream must
+// belong to that device).  The lookup can load the module (driver memory, a synchronisation), which is why
+// the first call per device belongs at start-up.  Threads may race to the first lookup: they store the same
+// address, through an atomic.
 static int static_scratch(float** out) {
-    static float* ptr[64] = {};
+    static std::atomic<float*> ptr[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
     if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
-    if (!ptr[dev]) {
+    float* cached = ptr[dev].load(std::memory_order_acquire);
+    if (!cached) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_u) != cudaSuccess || !p) return METEORA_ERR_CUDA;
-        ptr[dev] = static_cast<float*>(p);
+        cached = static_cast<float*>(p);
+        ptr[dev].store(cached, std::memory_order_release);
     }
-    *out = ptr[dev];
+    *out = cached;
     return METEORA_OK;
 }
 

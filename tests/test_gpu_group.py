@@ -7,7 +7,7 @@ import torch
 import oracle
 from paper_2405_13053_b200 import binding as mb
 from paper_2405_13053_b200 import workloads
-from .gpu_util import check_selection, rel_l2, to_dev
+from .gpu_util import bf16_bound_ok, check_selection, clear_tokens, rel_l2, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -39,10 +39,12 @@ def check_group(ws, y_tol):
     for w, y, (idx, wts) in zip(ws, ys, routing):
         o_idx, o_w, o_logits = oracle.gate_topk(w["x"], w["Wg"], w.k, w.temperature)
         clear = check_selection(idx, o_idx, o_logits, w.k)
-        np.testing.assert_allclose(wts[clear], o_w[clear], rtol=2e-3, atol=1e-5)
+        np.testing.assert_allclose(wts[clear], o_w[clear], rtol=1e-4, atol=1e-5)   # fp32 on shared bf16 inputs
         ref = oracle.linear_forward_routed(w["x"], w["W0"], w["A"], w["B"], w["Wg"], idx, w.temperature)
         err = rel_l2(y, ref)
         assert err <= y_tol, (w.name, err)
+        if w.dtype == "bf16":                                        # element by element: 5e-2 + one bf16 ulp of ref
+            assert bf16_bound_ok(y, ref) <= 0.0, w.name
     return ys, routing
 
 
@@ -70,6 +72,8 @@ def test_group_agrees_with_separate_calls():
         y1, i1, _ = mb.meteora_linear_forward(x, W0, A, B, Wg, w.k, return_routing=True)
         torch.cuda.synchronize()
         same = np.all(i1.cpu().numpy() == idx, axis=1)
+        _, _, o_logits = oracle.gate_topk(w["x"], w["Wg"], w.k, w.temperature)
+        assert np.all(same[clear_tokens(o_logits, w.k)])             # the two may differ only at near-ties
         assert same.mean() > 0.98
         assert rel_l2(y[same], y1.float().cpu().numpy()[same]) < 5e-3
 

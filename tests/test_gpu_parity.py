@@ -2,8 +2,10 @@
 seeded inputs.  Tolerances (stated where used):
   - indices, counts, offsets, perm: bit-exact (selections only where the logit gap exceeds 1e-3);
   - fp32 layers: relative L2 <= 1e-4 (measured ~1e-6);
-  - bf16 layers: y relative L2 <= 1e-2 and max-abs <= 5e-2; fp32 intermediates (weights, delta) <= 1e-4,
-    since both sides read the same bf16 values and the GPU accumulates in fp32.
+  - bf16 layers: y relative L2 <= 1e-2 and, element by element, |y - ref| <= 5e-2 + 2^-8 |ref| (the absolute
+    bound plus one bf16 ulp of the reference, so that large outputs are not excused wholesale: a wrong row
+    tile, a dropped pick or a stale partial tile breaks it); fp32 intermediates (routing weights, delta)
+    <= 1e-4, since both sides read the same bf16 values and the GPU accumulates in fp32.
 """
 import numpy as np
 import pytest
@@ -13,7 +15,7 @@ import oracle
 from paper_2405_13053_b200 import binding as mb
 from paper_2405_13053_b200 import workloads
 
-from .gpu_util import check_selection, max_abs, rel_l2, to_dev
+from .gpu_util import bf16_bound_ok, check_selection, clear_tokens, max_abs, rel_l2, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -139,6 +141,12 @@ def test_lora_delta_with_empty_adapters_and_single_hot_adapter():
 
 
 # ----------------------------------------------------------------------------------------- whole layer
+# Routing weights of the fused paths against the oracle: fp32 logits from the stacked tensor-core product (bf16
+# inputs, fp32 accumulation, slices of the contraction axis added in fp32) differ from the fp64 logits by a few
+# 1e-6, and a softmax weight moves by at most a quarter of the logit error.
+W_RTOL, W_ATOL = 1e-4, 1e-5
+
+
 def run_forward(w, **kw):
     x, W0, A, B, Wg = to_dev(w, "x", "W0", "A", "B", "Wg")
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, x.dtype, w.temperature)
@@ -149,18 +157,32 @@ def run_forward(w, **kw):
 
 
 def check_forward(w, y_tol, abs_tol=None, tokens=None):
-    """Compare the fused forward with the oracle; `tokens` restricts the y comparison to sampled rows."""
+    """Compare the fused forward with the oracle; `tokens` restricts the y comparison to sampled rows.
+    The routing (selection and weights) is always checked on every token."""
     y, idx, wts = run_forward(w)
     o_idx, o_w, o_logits = oracle.gate_topk(w["x"], w["Wg"], w.k, w.temperature)
     clear = check_selection(idx, o_idx, o_logits, w.k)
-    np.testing.assert_allclose(wts[clear], o_w[clear], rtol=2e-3, atol=1e-5)
+    np.testing.assert_allclose(wts[clear], o_w[clear], rtol=W_RTOL, atol=W_ATOL)
+    np.testing.assert_allclose(wts.sum(axis=1), 1.0, atol=1e-6)
     sel = np.arange(w.T) if tokens is None else np.asarray(tokens)
     ref = oracle.linear_forward_routed(w["x"][sel], w["W0"], w["A"], w["B"], w["Wg"], idx[sel], w.temperature)
     err = rel_l2(y[sel], ref)
     assert err <= y_tol, err
+    if w.dtype == "bf16":
+        excess = bf16_bound_ok(y[sel], ref)
+        assert excess <= 0.0, excess
     if abs_tol is not None:
         assert max_abs(y[sel], ref) <= abs_tol
     return y, idx, err
+
+
+def assert_same_outside_the_band(w, i0, i1):
+    """Two paths may pick differently only where the oracle's logits are within GAP of a tie."""
+    _, _, o_logits = oracle.gate_topk(w["x"], w["Wg"], w.k, w.temperature)
+    clear = clear_tokens(o_logits, w.k)
+    same = np.all(i0 == i1, axis=1)
+    assert np.all(same[clear]), np.nonzero(clear & ~same)[0]
+    return same
 
 
 def test_config0_fp32():
@@ -196,13 +218,13 @@ def test_forward_small_shapes(case):
     if w.dtype == "f32":
         check_forward(w, y_tol=1e-4)
     else:
-        check_forward(w, y_tol=1e-2, abs_tol=5e-2 * max(1.0, float(np.abs(w["x"]).max())))
+        check_forward(w, y_tol=1e-2)
 
 
 @pytest.mark.parametrize("T", workloads.CONFIG1_T)
 def test_config1_decode_shapes(T):
     w = workloads.config1(T)
-    y, idx, err = check_forward(w, y_tol=1e-2, abs_tol=5e-2)
+    y, idx, err = check_forward(w, y_tol=1e-2, abs_tol=5e-2)                # at |y| ~ 1.3 the plain bound holds too
     assert err < 5e-3                                                # one bf16 rounding of y: ~2^-9 per element
 
 
@@ -237,7 +259,7 @@ def test_tensor_core_and_plain_paths_agree():
         y_simt, i_simt, _ = run_forward(w)
     finally:
         mb.meteora_set_tuning("force_simt", 0)
-    same = np.all(i_tc == i_simt, axis=1)
+    same = assert_same_outside_the_band(w, i_tc, i_simt)
     assert same.mean() > 0.95
     assert rel_l2(y_tc[same], y_simt[same]) < 5e-3
 
@@ -318,7 +340,7 @@ def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
         y1, i1, _ = run_forward(w)
     finally:
         mb.meteora_set_tuning(knob, 0)
-    same = np.all(i0 == i1, axis=1)          # another slicing of the shrink may flip a near-tie of two logits
+    same = assert_same_outside_the_band(w, i0, i1)   # another slicing of the shrink may flip a near-tie of two logits
     assert same.mean() > 0.97
     assert rel_l2(y1[same], y0[same]) < 4e-3
 
@@ -445,7 +467,7 @@ def test_chain_and_single_launch_paths_agree():
         y_c, i_c, _ = run_forward(w)
     finally:
         mb.meteora_set_tuning("fused", 1)
-    same = np.all(i_f == i_c, axis=1)
+    same = assert_same_outside_the_band(w, i_f, i_c)
     assert same.mean() > 0.98
     assert rel_l2(y_f[same], y_c[same]) < 5e-3
 
@@ -464,19 +486,32 @@ def test_host_buffer_entry_point():
 
 
 # ----------------------------------------------------------------------------------------- full-size shapes
-@pytest.mark.parametrize("shape,T", [("gate_up", 512), ("down", 2048), ("kv", 8192)])
+# Every (shape, T) cell of configs 2, 3 and 4 at full size: the routing of all T tokens against the oracle, y on
+# sampled tokens (first, last, the edges of the 128- and 256-token tiles, and random ones), all d_out outputs of each.
+def sampled_tokens(T, seed, n=18):
+    edges = [t for t in (0, 127, 128, 255, 256, T // 2, T - 257, T - 129, T - 1) if 0 <= t < T]
+    return np.unique(np.concatenate([edges, np.random.default_rng(seed).integers(0, T, min(n, T))]).astype(np.int64))
+
+
+@pytest.mark.parametrize("T", workloads.CONFIG2_T)
+@pytest.mark.parametrize("shape", list(workloads.CONFIG2_SHAPES))
 def test_config2_prefill_sampled_rows(shape, T):
     w = workloads.config2(shape, T)
-    rng = np.random.default_rng(5)
-    rows = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, 22)]))
-    check_forward(w, y_tol=1e-2, abs_tol=5e-2 * 8, tokens=rows)       # |x| reaches ~4 here, y ~ 4x larger than config 1
+    check_forward(w, y_tol=1e-2, tokens=sampled_tokens(T, 5))
 
 
-@pytest.mark.parametrize("shape,T", [("qkvo", 64), ("gate_up", 1), ("down", 64)])
+@pytest.mark.parametrize("T", workloads.CONFIG3_T)
+@pytest.mark.parametrize("shape", list(workloads.CONFIG3_SHAPES))
 def test_config3_sampled_rows(shape, T):
     w = workloads.config3(shape, T)
-    rows = np.unique(np.concatenate([[0, T - 1], np.random.default_rng(6).integers(0, T, 14)]))
-    check_forward(w, y_tol=1e-2, abs_tol=5e-2 * 8, tokens=rows)
+    check_forward(w, y_tol=1e-2, tokens=sampled_tokens(T, 6))
+
+
+@pytest.mark.parametrize("T", workloads.CONFIG4_T)
+@pytest.mark.parametrize("linear", list(workloads.CONFIG4_LINEARS))
+def test_config4_linears(linear, T):
+    w = workloads.config4(linear, T)
+    check_forward(w, y_tol=1e-2, tokens=sampled_tokens(T, 7))
 
 
 # ----------------------------------------------------------------------------------------- error behaviour
