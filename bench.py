@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--variants", action="store_true",
                     help="time the variants of the method at 4096 -> 4096 (top-k, rank, adapter count, temperature), "
                          "the axes of the paper's synthetic sweep (App. A.7); one JSON line each")
+    ap.add_argument("--knob", action="append", default=[], metavar="NAME=VALUE",
+                    help="set a measurement knob of the library (meteora_set_tuning) before timing; repeatable")
     ap.add_argument("--decode-loop", action="store_true",
                     help="time one autoregressive decode step over the 224 MeteoRA linears of a LLaMA3-8B-shaped "
                          "stack (ms per generated token, the unit of App. A.7); also part of --sweep")
@@ -88,7 +90,7 @@ def kernel_sha():
     white space removed, so that an edit of a comment does not void the figure and an edit of the code does."""
     import re
     h = hashlib.sha256()
-    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "wgemm_pair.cuh", "select.cuh"):
+    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "decode_stream.cuh", "wgemm_pair.cuh", "select.cuh"):
         with open(os.path.join(ROOT, "paper_2405_13053_b200", "csrc", name), "r") as fh:
             text = fh.read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
@@ -240,10 +242,18 @@ def run_ours(args):
             host_w0 = w
         m = {n: torch.from_numpy(w[n]).to(dt).cuda() for n in ("x", "W0", "A", "B", "Wg")}
         m["y"] = torch.empty((T, D_OUT), dtype=dt, device="cuda")
-        m["ws"] = mb.alloc_workspace(shape)
         m["x_host"] = torch.from_numpy(w["x"]).to(dt).pin_memory()
         m["y_host"] = torch.empty((T, D_OUT), dtype=dt).pin_memory()
         mods.append(m)
+    # Scratch: the calls of the device-resident step are ordered on one stream and share ONE workspace, the way a
+    # decoder passes the same scratch buffer to every layer; the end-to-end step spreads its modules over several
+    # streams, so there every stream has its own (calls that may overlap in time must not share one).
+    n_e2e = max(1, args.e2e_streams)
+    ws_dev = mb.alloc_workspace(shape)
+    ws_e2e = [mb.alloc_workspace(shape) for _ in range(n_e2e)]
+    for i, m in enumerate(mods):
+        m["ws"] = ws_dev
+        m["ws_host"] = ws_e2e[i % n_e2e]
     torch.cuda.synchronize()
 
     def call_device(m):
@@ -256,7 +266,7 @@ def run_ours(args):
     def call_host(m):
         rc = lib.meteora_linear_forward_host(m["x_host"].data_ptr(), m["W0"].data_ptr(), m["A"].data_ptr(),
                                              m["B"].data_ptr(), m["Wg"].data_ptr(), ctypes.byref(shape),
-                                             m["y_host"].data_ptr(), m["ws"].data_ptr(), m["ws"].numel(),
+                                             m["y_host"].data_ptr(), m["ws_host"].data_ptr(), m["ws_host"].numel(),
                                              torch.cuda.current_stream().cuda_stream)
         if rc != 0:
             raise mb.MeteoraError(rc, "meteora_linear_forward_host")
@@ -268,7 +278,7 @@ def run_ours(args):
     # End-to-end step: the modules are independent, so their calls go round-robin onto a few streams and the
     # host-to-device copy of one module, the kernel of another and the device-to-host copy of a third overlap
     # (the two copy engines and the SMs); every stream is joined before the step ends.
-    e2e_streams = [torch.cuda.Stream() for _ in range(max(1, args.e2e_streams))]
+    e2e_streams = [torch.cuda.Stream() for _ in range(n_e2e)]
 
     def step_host():
         cur = torch.cuda.current_stream()
@@ -317,8 +327,8 @@ def run_ours(args):
         return max_over_ranks(e0.elapsed_time(e1), world, "cuda")
 
     def check_status():
-        for m in mods:
-            st = mb.meteora_workspace_status(m["ws"])
+        for ws in [ws_dev] + ws_e2e:
+            st = mb.meteora_workspace_status(ws)
             if st != 0:
                 raise mb.MeteoraError(st, "device status after the timed region")
 
@@ -354,10 +364,11 @@ def run_ours(args):
     #   three-launch chain: event pairs around the base-product launch of every call, in a second region of the
     #     same launches issued behind a long blocker kernel so that the host is never the bottleneck.
     plan = mb.meteora_describe_plan(shape)
-    single_launch = "path=fused_decode" in plan
+    single_launch = "path=fused_decode" in plan or "path=stream_decode" in plan
     launches_per_call = 1 if single_launch else 3
     if single_launch:
-        kernel_name = "k_decode_fused (base product + stacked shrink + selection + LoRA expand, one launch per call)"
+        kernel_name = ("k_decode_stream" if "path=stream_decode" in plan else "k_decode_fused") + \
+            " (base product + stacked shrink + selection + LoRA expand, one launch per call)"
         kernel_ms, kernel_launches = ms_total, K * R
     else:
         kernel_name = ("k_wgemm_pair (base product + LoRA expand on pairs of SMs)" if "pairs_of_ctas" in plan
@@ -376,7 +387,9 @@ def run_ours(args):
     check_status()
 
     # ---- algorithmic bytes (adapters actually selected, from the realised routing of module 0)
-    idx0, _ = mb.meteora_workspace_routing(shape, mods[0]["ws"])
+    step_device()                                              # the shared workspace holds the last module's routing
+    torch.cuda.synchronize()
+    idx0, _ = mb.meteora_workspace_routing(shape, ws_dev)
     touched = int(torch.unique(idx0).numel())
     bytes_base = (D_IN * D_OUT + touched * D_OUT * RANK + T * (D_IN + D_OUT)) * es
     bytes_path = bytes_base + (N_ADAPTERS * D_IN + touched * RANK * D_IN) * es
@@ -404,6 +417,7 @@ def run_ours(args):
                    "tokens_per_module": T, "modules_per_step": R, "launch": mode, "e2e_launch": mode_e2e, "e2e_streams": len(e2e_streams),
                    "l2": f"weights of the {R} modules total {R * bytes_path / 1e6:.0f} MB > 126 MB L2, "
                          "so no weight is L2-resident between visits",
+                   "workspace": "one scratch buffer shared by the step's stream-ordered calls (one per stream end to end)",
                    "parallelism": f"token-sharded replicas x{world}, no collective", "plan": plan},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": R * T * D_IN * es,
                 "d2h_bytes_per_step": R * T * D_OUT * es, "ms_per_step": ms_e2e / K},
@@ -476,13 +490,14 @@ def run_sweep(args):
         g = torch.Generator(device="cuda").manual_seed(7)
         x_np = workloads.make_x(T, d_in, x_kind, 5, "bf16")          # token statistics of the config; weights on device
         mods = []
+        ws_shared = mb.alloc_workspace(shape)                        # stream-ordered calls share one scratch buffer
         for i in range(R):
             m = {"x": torch.from_numpy(x_np).to(dt).cuda(),
                  "W0": (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt),
                  "A": ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt),
                  "B": (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt),
                  "Wg": (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt),
-                 "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": mb.alloc_workspace(shape)}
+                 "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": ws_shared}
             mods.append(m)
 
         def step():
@@ -802,6 +817,7 @@ def run_variants():
             shape = mb.make_shape(T, d_in, d_out, N, r, k, dt, tau)
             g = torch.Generator(device="cuda").manual_seed(3)
             mods = []
+            ws_shared = mb.alloc_workspace(shape)
             for i in range(R):
                 x = torch.randn(T, d_in, device="cuda", generator=g)
                 x = (x / x.pow(2).mean(dim=1, keepdim=True).sqrt()).to(dt)
@@ -809,7 +825,7 @@ def run_variants():
                              "A": ((torch.rand(N, r, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt),
                              "B": (0.01 * torch.randn(N, d_out, r, device="cuda", generator=g)).to(dt),
                              "Wg": (torch.randn(N, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt),
-                             "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": mb.alloc_workspace(shape)})
+                             "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": ws_shared})
 
             def step():
                 for m in mods:
@@ -858,8 +874,22 @@ def run_variants():
             del mods, graph
 
 
+def apply_knobs(args):
+    if not args.knob:
+        return
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import build as lib_build
+
+    lib_build.build_library()
+    for kv in args.knob:
+        name, value = kv.split("=")
+        mb.meteora_set_tuning(name, int(value))
+
+
 def main():
     args = parse_args()
+    if args.impl != "reference":
+        apply_knobs(args)
     if args.variants:
         run_variants()
     elif args.decode_loop:

@@ -109,6 +109,12 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
     }
     Profile& pf = profile();
     const bool timed = pf.open && 2 * (pf.used + 1) <= (int)pf.ev.size();
+    if (decode_stream_supported(s)) {
+        if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
+        rc = launch_decode_stream(x, W0, A, B, Wg, s, ws, y, st);
+        if (timed) cudaEventRecord(pf.ev[2 * pf.used++ + 1], st);
+        return rc;
+    }
     if (decode_fused_supported(s)) {
         if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
         rc = launch_decode_fused(x, W0, A, B, Wg, s, ws, y, st);
@@ -451,6 +457,9 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "force_simt")) t.force_simt = value;
     else if (!strcmp(name, "pdl")) t.pdl = value;
     else if (!strcmp(name, "fused")) t.fused = value;
+    else if (!strcmp(name, "stream")) t.stream = value;
+    else if (!strcmp(name, "pf")) t.pf = value;
+    else if (!strcmp(name, "own_local")) t.own_local = value;
     else if (!strcmp(name, "coop")) t.coop = value;
     else if (!strcmp(name, "no_hold")) t.no_hold = value;
     else if (!strcmp(name, "unit_split")) t.unit_split = value;

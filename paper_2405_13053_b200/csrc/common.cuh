@@ -105,6 +105,10 @@ int launch_decode_group(const void* x, const GroupModule* mods, int n_modules, c
 int describe_plan(const meteora_shape_t& s, char* buf, size_t n);
 int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
+// streamed decode kernel (wgemm_tcgen05.cu + decode_stream.cuh): up to 128 tokens, two launches resident at a time
+bool decode_stream_supported(const meteora_shape_t& s);
+int launch_decode_stream(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
 
 struct Tuning {
     int splits = 0;
@@ -117,6 +121,10 @@ struct Tuning {
     int simt_expand = 0;   // 1: keep the LoRA expand on CUDA cores even for rank 8
     int force_simt = 0;
     int pdl = 1;
+    int stream = 1;          // streamed decode kernel (two launches resident at a time): 0 never, 1 where the planner takes it,
+                             // 2 the same kernel with one CTA per SM and a deep ring, 3 wherever the shape allows
+    int own_local = 1;       // streamed decode kernel: a CTA keeps its own row slice of its accumulator in shared memory
+    int pf = 0;              // its L2 prefetch of the weights beyond the ring: 0 planner's cap, -1 none, n > 0 cap in MB
     int fused = 1;           // 0: never use the single-launch decode kernel
     int coop = 1;            // 0 (measurement only): launch it without the co-residency guarantee
     int pair = 1;            // prefill base product on pairs of SMs (256 x 256 tiles, two-CTA MMA): 0 never, 1 where

@@ -697,6 +697,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
 }  // namespace meteora
 
 #include "decode_fused.cuh"
+#include "decode_stream.cuh"
 #include "wgemm_pair.cuh"
 
 namespace meteora {
@@ -1449,31 +1450,6 @@ bool decode_group_supported(const meteora_shape_t& s, const int* d_outs, int G) 
     return make_fused_plan(s, d_outs, G).ok;
 }
 
-// Human-readable launch plan of meteora_linear_forward for this shape (for logs and benchmark records).
-int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
-    if (!tc_path_supported(s)) return snprintf(buf, n, "path=simt");
-    const FusedPlan fp = make_fused_plan(s);
-    if (fp.ok)
-        return snprintf(buf, n,
-                        "path=fused_decode launches=1 main_ctas=%d row_tiles=%d units_per_cta=%.1f aux_ctas=%d "
-                        "aux_slices=%d tile_tokens=%d stages=%d kc=%d smem=%zu resident_ctas=%d",
-                        fp.n_main, fp.row_tiles, (double)fp.row_tiles * fp.upt / fp.n_main, fp.n_aux, fp.aux_slices,
-                        fp.main.BN, fp.main.stages, fp.main.kc, fp.main.smem, max_resident_ctas(fp.main.smem));
-    const int row_tiles = (s.d_out + kBM - 1) / kBM;
-    const PairPlan pp = make_pair_plan(s);
-    if (pp.ok)
-        return snprintf(buf, n,
-                        "path=chain(not fused: reason %d) launches=3 base=pairs_of_ctas pairs=%d tile=256x256 stages=%d "
-                        "smem=%zu expand=mma",
-                        fp.why, (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens), pp.stages, pp.smem);
-    const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
-    return snprintf(buf, n,
-                    "path=chain(not fused: reason %d) launches=3 base_ctas=%d cluster=%d tile_tokens=%d stages=%d kc=%d "
-                    "smem=%zu expand=%s",
-                    fp.why, row_tiles * pl.splits * pl.n_tiles, pl.splits, pl.BN, pl.stages, pl.kc, pl.smem,
-                    pl.lora_mma ? "mma" : "simt");
-}
-
 // (module, token) items from which the selection reads in two narrow round trips.  Measured, narrow against wide, us
 // per call at T = 1 / 16 / 32 / 64 / 128 / 256: 4096 -> 4096 +0.25 / -0.25 / -0.1 / -0.4 / -0.35 / -1.05; 4096 -> 1024
 // 0 / -0.2 / -0.1 / -0.4 / -0.4 / -0.4; 5120 -> 5120 0 / -0.4 / -0.2 / 0 / +0.1 / +0.2; 13824 -> 5120 within +-0.2.
@@ -1608,6 +1584,244 @@ int launch_decode_fused(const void* x, const void* W0, const void* A, const void
                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st) {
     GroupModule gm = {W0, A, B, Wg, y, s.d_out, ws};
     return launch_decode_group(x, &gm, 1, s, ws.status, ws.part_g, ws.tile_ctr, st);
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// Streamed decode launch (decode_stream.cuh): one launch per call, two launches resident at a time.
+// ------------------------------------------------------------------------------------------------
+struct StreamPlan {
+    bool ok;
+    int why;       // why not: 1 knob/shape, 2 more row tiles than SMs, 5 shared memory
+    int BN, kc, stages, aux_stages, tmem_cols, S, n_main, row_tiles;
+    int n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices;
+    int pf_main, pf_aux, slab_off, ring_bytes, ctas_per_sm;
+    size_t smem;
+};
+constexpr int kStreamBarSlots = 16;
+constexpr size_t kTwoPerSmBytes = 113 * 1024;    // dynamic shared memory with which two CTAs share an SM
+
+static StreamPlan make_stream_plan(const meteora_shape_t& s) {
+    const Tuning& tn = tuning();
+    StreamPlan sp = {};
+    sp.why = 1;
+    if (!tn.fused || !tn.stream || tn.simt_expand) return sp;
+    if (!tc_path_supported(s) || s.T > 128 || s.r % 8 != 0 || s.d_in % kBK != 0 || s.d_out <= 0) return sp;
+    // Two CTAs per SM means half the ring each.  Measured per call, this kernel against the cooperative one (one CTA
+    // per SM, twice the ring): 4096 -> 4096 (34 MB of W0) 11.8 / 12.7 / 16.7 us against 13.5 / 14.2 / 17.1 at 1 / 32 / 128
+    // tokens; 5120 -> 5120 (52 MB) 15.1 against 15.7 at one token but 19.3 against 18.0 at 64; 13824 -> 5120 (142 MB)
+    // 39.3 against 35.3 at 64: the longer the stream, the more the deeper ring counts and the less the set-up and the
+    // first tiles loaded under the call ahead.  Taken up to 40 MB of W0 (knob stream = 3: always).
+    if ((size_t)s.d_out * s.d_in * 2 > ((size_t)40 << 20) && tn.stream != 3) return sp;
+    const int sms = std::min(sm_count(), 148);                   // the workspace holds partial tiles for 148 CTAs
+    const int ksteps = s.d_in / kBK;
+    sp.row_tiles = (s.d_out + kBM - 1) / kBM;
+    if (sp.row_tiles > kMaxFusedRowTiles) return sp;
+    // stacked shrink: tiles of [A; Wg] (Wg behind A's last rows when the tile has room), slices of the contraction axis
+    sp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
+    const int tail_rows = s.N * s.r - (sp.a_tiles - 1) * kBM;
+    const bool merged = tail_rows % 8 == 0 && tail_rows + s.N <= kBM;
+    sp.aux_tiles = merged ? sp.a_tiles : sp.a_tiles + 1;
+    sp.gate_tile = sp.aux_tiles - 1;
+    sp.gate_row0 = merged ? tail_rows : 0;
+    sp.why = 2;
+    int aux_budget = std::max(20, 4 * sp.aux_tiles);
+    if (tn.aux_ctas > 0) aux_budget = std::max(tn.aux_ctas, sp.aux_tiles);
+    aux_budget = std::min(aux_budget, sms - 8);
+    sp.aux_slices = std::min(std::min(aux_budget / sp.aux_tiles, ksteps), 16);
+    if (sp.aux_slices < 1) return sp;
+    sp.n_aux = sp.aux_tiles * sp.aux_slices;
+    sp.kc = 1;
+    if (tn.kc > 0 && tn.kc <= 4 && ksteps % tn.kc == 0) sp.kc = tn.kc;
+    const int nst = ksteps / sp.kc;
+    int S = std::min(8, (sms - sp.n_aux) / sp.row_tiles);
+    if (tn.splits > 0) S = std::min(tn.splits, 8);
+    S = std::min(S, nst);
+    // at most two CTAs per SM in all, and the workspace holds row tiles + 148 partial tiles
+    if (S < 1 || sp.row_tiles * S + sp.n_aux > 2 * sms || sp.row_tiles * S > sp.row_tiles + 148) return sp;
+    sp.S = S;
+    sp.n_main = sp.row_tiles * S;
+    // narrow layers leave SMs idle: give them to the stacked shrink as further slices (all 16 or none)
+    if (tn.aux_ctas == 0) {
+        const int spare = sms - sp.n_main - sp.n_aux;
+        const int full = std::min(ksteps, 16);
+        if (sp.aux_slices < full && sp.aux_slices + spare / sp.aux_tiles >= full) {
+            sp.aux_slices = full;
+            sp.n_aux = sp.aux_tiles * sp.aux_slices;
+        }
+    }
+    sp.why = 5;
+    sp.BN = (s.T + 15) / 16 * 16;
+    int cols = 32;
+    while (cols < sp.BN) cols *= 2;
+    sp.tmem_cols = cols;
+    const int cpa = s.r / 8;
+    const int nq_max = (32 + S - 1) / S;
+    const size_t slab_bytes = (size_t)s.N * cpa * 4 * nq_max * 16;
+    sp.slab_off = (int)align_up((size_t)(2 * kStreamBarSlots + 4) * 8 + 16, 128);
+    const size_t stage_bytes = (size_t)sp.kc * (kWTileBytes + (size_t)sp.BN * 128);
+    const size_t aux_stage_bytes = kWTileBytes + (size_t)sp.BN * 128;
+    const int ntok = s.T;
+    // what the last step fetches into the idle ring: S row slices of partial tiles (or the CTA's own tile), the
+    // adapter indices and uw of every token; the aux CTAs stage their accumulator tile there
+    // (S blocks of partials and one of the expand, each a row slice of at most 4 nq_max rows for all tokens)
+    const size_t parts = (size_t)(S + 1) * align_up((size_t)ntok * 4 * nq_max * 4, 128);
+    const size_t landing = parts + align_up(align_up((size_t)ntok * s.k * 4, 16), 128) + (size_t)ntok * s.k * s.r * 4;
+    // an aux CTA stages its accumulator tile there, later its tokens' rows of every partial tile of the stacked shrink
+    const size_t aux_rows = (size_t)sp.n_aux * ((s.T + sp.n_aux - 1) / sp.n_aux) * kBM * 4;
+    const size_t ring_need = std::max(std::max(landing, (size_t)sp.BN * kBM * 4), aux_rows);
+    const int n_it_max = (nst + S - 1) / S;
+    const int nks_aux = (ksteps + sp.aux_slices - 1) / sp.aux_slices;
+    for (int per_sm = 2; per_sm >= 1; --per_sm) {
+        if (per_sm == 2 && tn.stream == 2) continue;               // knob: one CTA per SM, deep ring
+        const size_t budget = per_sm == 2 ? kTwoPerSmBytes : 226 * 1024;
+        const size_t fixed = 1024 + sp.slab_off + slab_bytes;
+        if (fixed + ring_need > budget || fixed + 2 * stage_bytes > budget) continue;
+        const size_t avail = budget - fixed;
+        int stages = (int)std::min<size_t>(avail / stage_bytes, (size_t)std::min(kStreamBarSlots, std::max(n_it_max, 2)));
+        if (tn.stages > 0) stages = std::min(tn.stages, (int)std::min<size_t>(avail / stage_bytes, kStreamBarSlots));
+        if (stages < 2) continue;
+        const size_t ring_bytes = align_up(std::max((size_t)stages * stage_bytes, ring_need), 128);
+        if (fixed + ring_bytes > budget) continue;
+        sp.stages = stages;
+        sp.aux_stages = (int)std::min<size_t>(std::min<size_t>(ring_bytes / aux_stage_bytes, kStreamBarSlots),
+                                              (size_t)std::max(nks_aux, 1));
+        sp.ring_bytes = (int)ring_bytes;
+        sp.smem = fixed + ring_bytes;
+        sp.ctas_per_sm = per_sm;
+        break;
+    }
+    if (sp.ctas_per_sm == 0) return sp;
+    // L2 prefetch of the weights beyond the ring, issued before the wait for the kernel ahead: everything up to a
+    // cap (the L2 holds this call's weights and the next call's at the same time).  Knob pf: -1 none, n > 0 cap in MB.
+    // (measured at 4096 -> 4096: with the prefetch a call takes 20.2 us at 128 tokens and 13.9 at one, without it 18.1
+    // and 13.0; a prefetch 4 - 8 ring stages ahead of the loads inside the main loop costs 0.6 - 1.4 us as well: the
+    // prefetches take the TMA engine's and the memory system's time without shortening the loads' latency.  Off by default.)
+    const size_t cap = tn.pf > 0 ? (size_t)tn.pf << 20 : 0;
+    const size_t per_stage_all = (size_t)sp.n_main * sp.kc * kWTileBytes;
+    sp.pf_main = (int)std::min<size_t>((size_t)std::max(0, n_it_max - sp.stages), cap / per_stage_all);
+    sp.pf_aux = cap > 0 ? std::max(0, nks_aux - sp.aux_stages) : 0;
+    sp.why = 0;
+    sp.ok = true;
+    return sp;
+}
+
+bool decode_stream_supported(const meteora_shape_t& s) { return make_stream_plan(s).ok; }
+
+int launch_decode_stream(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st) {
+    const StreamPlan sp = make_stream_plan(s);
+    if (!sp.ok) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    CUtensorMap mW, mA, mAt, mG, mX, mX1;
+    int rc;
+    const int tail_box = sp.gate_row0 > 0 ? sp.gate_row0 : kBM, gate_box = kBM - sp.gate_row0;
+    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, sp.kc, &mW)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, 1, &mA)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, tail_box, 1, &mAt)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Wg, s.d_in, s.N, gate_box, 1, &mG)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, sp.BN, sp.kc, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, sp.BN, 1, &mX1)) != METEORA_OK) return rc;
+    StreamParams d = {};
+    d.T = s.T;
+    d.BN = sp.BN;
+    d.ksteps = s.d_in / kBK;
+    d.stages = sp.stages;
+    d.kc = sp.kc;
+    d.aux_stages = sp.aux_stages;
+    d.tmem_cols = sp.tmem_cols;
+    d.N = s.N;
+    d.r = s.r;
+    d.k = s.k;
+    d.d_out = s.d_out;
+    d.row_tiles = sp.row_tiles;
+    d.S = sp.S;
+    d.n_main = sp.n_main;
+    d.n_aux = sp.n_aux;
+    d.aux_tiles = sp.aux_tiles;
+    d.aux_slices = sp.aux_slices;
+    d.a_tiles = sp.a_tiles;
+    d.gate_tile = sp.gate_tile;
+    d.gate_row0 = sp.gate_row0;
+    d.pf_main = sp.pf_main;
+    d.pf_aux = sp.pf_aux;
+    d.slab_off = sp.slab_off;
+    d.ring_bytes = sp.ring_bytes;
+    d.bar_slots = kStreamBarSlots;
+    d.inv_tau = 1.0f / s.temperature;
+    d.B = (const __nv_bfloat16*)B;
+    d.y = (__nv_bfloat16*)y;
+    d.topk_idx = ws.topk_idx;
+    d.topk_w = ws.topk_w;
+    d.uw = ws.uw;
+    d.u_part = ws.u_all;
+    d.part_g = ws.part_g;
+    d.ctr = ws.status + 16;
+    d.tile_ctr = ws.tile_ctr;
+    d.status = ws.status;
+    d.own_local = tuning().own_local && sp.S > 1 ? 1 : 0;
+    if (sp.S == 1) d.own_local = 1;                             // the tile is the CTA's alone: nothing goes through scratch
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            return METEORA_ERR_CUDA;
+        // the whole shared-memory / L1 array as shared memory, so that two CTAs of 113 KB fit
+        if (cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+            return METEORA_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sp.n_main + sp.n_aux);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = sp.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    const bool want_pdl = tuning().pdl_decode != 0;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = want_pdl ? 1 : 0;
+    d.pdl = want_pdl ? 1 : 0;
+#ifdef METEORA_TRACE
+    static int trace_calls = 0;
+    d.trace_call = trace_calls++;
+#endif
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_stream, mW, mA, mAt, mG, mX, mX1, d));
+}
+
+// Human-readable launch plan of meteora_linear_forward for this shape (for logs and benchmark records).
+int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
+    if (!tc_path_supported(s)) return snprintf(buf, n, "path=simt");
+    const StreamPlan sp = make_stream_plan(s);
+    if (sp.ok)
+        return snprintf(buf, n,
+                        "path=stream_decode launches=1 main_ctas=%d row_tiles=%d ctas_per_tile=%d aux_ctas=%d aux_slices=%d "
+                        "tile_tokens=%d stages=%d kc=%d smem=%zu ctas_per_sm=%d l2_prefetch_stages=%d",
+                        sp.n_main, sp.row_tiles, sp.S, sp.n_aux, sp.aux_slices, sp.BN, sp.stages, sp.kc, sp.smem,
+                        sp.ctas_per_sm, sp.pf_main);
+    const FusedPlan fp = make_fused_plan(s);
+    if (fp.ok)
+        return snprintf(buf, n,
+                        "path=fused_decode launches=1 main_ctas=%d row_tiles=%d units_per_cta=%.1f aux_ctas=%d "
+                        "aux_slices=%d tile_tokens=%d stages=%d kc=%d smem=%zu resident_ctas=%d",
+                        fp.n_main, fp.row_tiles, (double)fp.row_tiles * fp.upt / fp.n_main, fp.n_aux, fp.aux_slices,
+                        fp.main.BN, fp.main.stages, fp.main.kc, fp.main.smem, max_resident_ctas(fp.main.smem));
+    const int row_tiles = (s.d_out + kBM - 1) / kBM;
+    const PairPlan pp = make_pair_plan(s);
+    if (pp.ok)
+        return snprintf(buf, n,
+                        "path=chain(not fused: reason %d) launches=3 base=pairs_of_ctas pairs=%d tile=256x256 stages=%d "
+                        "smem=%zu expand=mma",
+                        fp.why, (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens), pp.stages, pp.smem);
+    const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
+    return snprintf(buf, n,
+                    "path=chain(not fused: reason %d) launches=3 base_ctas=%d cluster=%d tile_tokens=%d stages=%d kc=%d "
+                    "smem=%zu expand=%s",
+                    fp.why, row_tiles * pl.splits * pl.n_tiles, pl.splits, pl.BN, pl.stages, pl.kc, pl.smem,
+                    pl.lora_mma ? "mma" : "simt");
 }
 
 }  // namespace meteora

@@ -140,6 +140,14 @@ def test_lora_delta_with_empty_adapters_and_single_hot_adapter():
     assert rel_l2(delta.cpu().numpy(), ref) <= 1e-4
 
 
+@pytest.fixture
+def cooperative_decode_kernel():
+    """The earlier one-launch decode kernel (cooperative launch, one CTA per SM) instead of the streamed one."""
+    mb.meteora_set_tuning("stream", 0)
+    yield
+    mb.meteora_set_tuning("stream", 1)
+
+
 # ----------------------------------------------------------------------------------------- whole layer
 # Routing weights of the fused paths against the oracle: fp32 logits from the stacked tensor-core product (bf16
 # inputs, fp32 accumulation, slices of the contraction axis added in fp32) differ from the fp64 logits by a few
@@ -287,7 +295,7 @@ def test_split_k_cluster_sizes_agree_with_oracle(splits, stages):
     (512, 9000, 24, 0), (1024, 1280, 64, 1), (1024, 1280, 200, 3),
     (128, 40000, 4, 0), (128, 60000, 70, 0),     # more row tiles than CTAs: unit ranges over three and four tiles
 ])
-def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
+def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile, cooperative_decode_kernel):
     # one kernel per call: base product + stacked shrink + selection + LoRA expand
     w = workloads.make_workload("fused", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="rms",
                                 seed=50 + T + d_out, b_std=0.3)
@@ -312,7 +320,7 @@ def test_single_launch_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
 @pytest.mark.parametrize("N,k,T,r", [(4, 2, 9, 8), (16, 4, 40, 8), (33, 3, 130, 8), (2, 1, 3, 8),
                                      (28, 2, 20, 16), (28, 2, 128, 32), (10, 3, 64, 24),
                                      (128, 2, 64, 8), (100, 8, 7, 8), (72, 4, 128, 16)])   # more than 64 adapters
-def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
+def test_single_launch_decode_kernel_adapter_counts(N, k, T, r, cooperative_decode_kernel):
     w = workloads.make_workload("fused_n", T=T, d_in=768, d_out=896, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
                                 seed=900 + N + r, b_std=0.3)
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
@@ -328,7 +336,7 @@ def test_single_launch_decode_kernel_adapter_counts(N, k, T, r):
                                         ("unit_split", 2), ("aux_ctas", 4), ("aux_ctas", 40), ("kc", 1), ("stages", 2),
                                         ("hold_after", 1), ("hold_after", 3), ("narrow_select", -1),
                                         ("narrow_select", 1)])
-def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
+def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value, cooperative_decode_kernel):
     w = workloads.make_workload("fused_knobs", T=70, d_in=1024, d_out=640, dtype="bf16", x_kind="normal", seed=1234,
                                 b_std=0.3)
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
@@ -349,7 +357,7 @@ def test_decode_kernel_planner_choices_do_not_change_the_result(knob, value):
 # first and then only the picks' shrink values); both add the partial copies in slice order, so routing, weights and
 # y must agree bit for bit, for one pick and several, rank 8 and above, few and many adapters.
 @pytest.mark.parametrize("T,N,r,k", [(70, 28, 8, 2), (9, 28, 8, 1), (40, 40, 16, 3), (33, 128, 8, 4), (20, 28, 32, 8)])
-def test_both_forms_of_the_selection_agree_bit_for_bit(T, N, r, k):
+def test_both_forms_of_the_selection_agree_bit_for_bit(T, N, r, k, cooperative_decode_kernel):
     w = workloads.make_workload("select_forms", T=T, d_in=1024, d_out=384, N=N, r=r, k=k, dtype="bf16",
                                 x_kind="normal", seed=5200 + T, b_std=0.3)
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
@@ -371,14 +379,21 @@ def test_both_forms_of_the_selection_agree_bit_for_bit(T, N, r, k):
 # with programmatic stream serialization (its CTAs may move onto an SM as soon as the previous kernel's CTA has
 # left it): it must not touch the previous result before that kernel has completed.  The chain with the
 # attribute and without it (knob pdl_decode) must agree bit for bit, and so must a repeat.
-@pytest.mark.parametrize("T,d", [(40, 512), (130, 1024)])
-def test_dependent_decode_calls_back_to_back(T, d):
+@pytest.mark.parametrize("stream_kernel", [1, 0])
+@pytest.mark.parametrize("T,d", [(40, 512), (130, 1024), (128, 2048)])
+def test_dependent_decode_calls_back_to_back(T, d, stream_kernel):
     layers = [workloads.make_workload(f"stack{i}", T=T, d_in=d, d_out=d, dtype="bf16", x_kind="normal",
                                       seed=4100 + 7 * i, b_std=0.3) for i in range(4)]
     dev = [to_dev(w, "W0", "A", "B", "Wg") for w in layers]
     x0 = to_dev(layers[0], "x")[0]
     shape = mb.make_shape(T, d, d, layers[0].N, layers[0].r, layers[0].k, torch.bfloat16)
-    assert "fused_decode" in mb.meteora_describe_plan(shape)
+    mb.meteora_set_tuning("stream", stream_kernel)
+    try:
+        plan = mb.meteora_describe_plan(shape)
+    finally:
+        mb.meteora_set_tuning("stream", 1)
+    # the streamed kernel takes up to 128 tokens: its CTAs are resident, and load weights, while the call ahead runs
+    assert ("stream_decode" if stream_kernel and T <= 128 else "fused_decode") in plan
     wss = [mb.alloc_workspace(shape) for _ in layers]
 
     def run_stack():
@@ -392,11 +407,13 @@ def test_dependent_decode_calls_back_to_back(T, d):
 
     results = {}
     try:
+        mb.meteora_set_tuning("stream", stream_kernel)
         for pdl in (1, 0, 1):
             mb.meteora_set_tuning("pdl_decode", pdl)
             results.setdefault(pdl, []).append(run_stack())
     finally:
         mb.meteora_set_tuning("pdl_decode", 1)
+        mb.meteora_set_tuning("stream", 1)
     assert np.all(np.isfinite(results[1][0]))
     np.testing.assert_array_equal(results[1][0], results[0][0])
     np.testing.assert_array_equal(results[1][0], results[1][1])
@@ -405,6 +422,95 @@ def test_dependent_decode_calls_back_to_back(T, d):
     ref = oracle.linear_forward_routed(layers[0]["x"], layers[0]["W0"], layers[0]["A"], layers[0]["B"], layers[0]["Wg"],
                                        y0[1].cpu().numpy())
     assert rel_l2(y0[0].float().cpu().numpy(), ref) <= 1e-2
+
+
+# ----------------------------------------------------------------------------------------- streamed decode kernel
+# The decode kernel whose CTAs share an SM two at a time (up to 128 tokens).  Shapes chosen for every way its work
+# splits: one CTA per row tile (1280 rows with splits = 1; 9000 rows = 71 tiles), several CTAs per tile with even
+# row slices (2, 4, 8) and uneven ones (3, 5, 6, 7: slices of 10 / 11 groups of 4 rows), a ragged last tile (1000
+# rows, 1001 rows: scalar stores), k-steps that do not divide by the CTAs per tile (1088 = 17 k-steps), one token,
+# a token count that is no multiple of 16, and the full 128.
+@pytest.mark.parametrize("d_in,d_out,T,per_tile", [
+    (1024, 640, 1, 0), (1024, 640, 8, 0), (1024, 640, 100, 0), (1024, 640, 128, 0),
+    (1536, 1000, 37, 0), (1088, 768, 16, 0), (2048, 4224, 5, 0), (2048, 4224, 128, 0),
+    (512, 9000, 24, 0), (1024, 1280, 64, 1), (1024, 1280, 128, 2), (1024, 1280, 77, 3), (1024, 1001, 50, 5),
+    (1024, 384, 128, 6), (1024, 384, 19, 7), (4096, 1024, 128, 0),
+])
+def test_streamed_decode_kernel_matches_oracle(d_in, d_out, T, per_tile):
+    w = workloads.make_workload("stream", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="rms",
+                                seed=150 + T + d_out, b_std=0.3)
+    mb.meteora_set_tuning("splits", per_tile)
+    try:
+        shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+        plan = mb.meteora_describe_plan(shape)
+        assert "stream_decode" in plan
+        if per_tile:
+            assert f"ctas_per_tile={per_tile} " in plan
+        check_forward(w, y_tol=1e-2)
+        y1, i1, w1 = run_forward(w)
+        y2, i2, w2 = run_forward(w)
+        np.testing.assert_array_equal(y1, y2)                        # fixed summation order: reproducible bit for bit
+        np.testing.assert_array_equal(i1, i2)
+        np.testing.assert_array_equal(w1, w2)
+    finally:
+        mb.meteora_set_tuning("splits", 0)
+
+
+# Adapter counts and ranks that change the stacked shrink's tiles (Wg behind A's rows, in a tile of its own, three
+# tiles of A, nine with 128 adapters) and the width of the staged B rows.
+@pytest.mark.parametrize("N,k,T,r", [(4, 2, 9, 8), (16, 4, 40, 8), (33, 3, 128, 8), (2, 1, 3, 8), (28, 2, 20, 16),
+                                     (28, 2, 128, 32), (10, 3, 64, 24), (128, 2, 64, 8), (100, 8, 7, 8),
+                                     (72, 4, 128, 16), (28, 1, 128, 8), (28, 2, 33, 8)])
+def test_streamed_decode_kernel_adapter_counts(N, k, T, r):
+    w = workloads.make_workload("stream_n", T=T, d_in=768, d_out=896, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
+                                seed=1900 + N + r, b_std=0.3, temperature=1.0 if N != 16 else 15.0)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16, w.temperature)
+    assert "stream_decode" in mb.meteora_describe_plan(shape)
+    check_forward(w, y_tol=1e-2)
+
+
+# Its planner's choices forced the other way: a shallow ring, two k-steps per stage, no L2 prefetch, a small prefetch
+# cap, one CTA per SM with a deep ring, few and many aux CTAs, no programmatic dependent launch.  None of them may
+# change the result beyond the order of the fp32 sums of the stacked shrink's slices.
+@pytest.mark.parametrize("knob,value", [("stages", 2), ("kc", 2), ("pf", -1), ("pf", 1), ("stream", 2), ("aux_ctas", 4),
+                                        ("aux_ctas", 40), ("pdl_decode", 0)])
+def test_streamed_decode_kernel_planner_choices(knob, value):
+    w = workloads.make_workload("stream_knobs", T=70, d_in=2048, d_out=640, dtype="bf16", x_kind="normal", seed=2234,
+                                b_std=0.3)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    y0, i0, _ = run_forward(w)
+    default = {"stream": 1, "pdl_decode": 1}.get(knob, 0)
+    mb.meteora_set_tuning(knob, value)
+    try:
+        assert "stream_decode" in mb.meteora_describe_plan(shape)
+        check_forward(w, y_tol=1e-2)
+        y1, i1, _ = run_forward(w)
+    finally:
+        mb.meteora_set_tuning(knob, default)
+    same = assert_same_outside_the_band(w, i0, i1)
+    assert same.mean() > 0.97
+    assert rel_l2(y1[same], y0[same]) < 4e-3
+
+
+def test_streamed_decode_calls_share_one_workspace_back_to_back():
+    # Eight calls in a row on ONE workspace without any synchronisation: a call's CTAs are resident while the call
+    # ahead still runs, but touch the workspace (counters, scratch) only after that call has completed.
+    T, d_in, d_out = 96, 1024, 768
+    ws_list = [workloads.make_workload(f"shared_ws{i}", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="normal",
+                                       seed=7100 + i, b_std=0.3) for i in range(8)]
+    shape = mb.make_shape(T, d_in, d_out, 28, 8, 2, torch.bfloat16)
+    assert "stream_decode" in mb.meteora_describe_plan(shape)
+    dev = [to_dev(w, "x", "W0", "A", "B", "Wg") for w in ws_list]
+    workspace = mb.alloc_workspace(shape)
+    ys = [mb.meteora_linear_forward(*t, 2, workspace=workspace) for t in dev]
+    torch.cuda.synchronize()
+    assert mb.meteora_workspace_status(workspace) == 0
+    for w, t, y in zip(ws_list, dev, ys):
+        y_alone, idx, _ = mb.meteora_linear_forward(*t, 2, return_routing=True)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(y.float().cpu().numpy(), y_alone.float().cpu().numpy())
+        ref = oracle.linear_forward_routed(w["x"], w["W0"], w["A"], w["B"], w["Wg"], idx.cpu().numpy())
+        assert rel_l2(y.float().cpu().numpy(), ref) <= 1e-2
 
 
 # Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
@@ -461,7 +567,7 @@ def test_prefill_on_single_sms_matches_oracle(d_in, d_out, T):
 
 def test_chain_and_single_launch_paths_agree():
     w = workloads.config1(128)
-    y_f, i_f, _ = run_forward(w)                                     # T = 128 takes the single launch by default
+    y_f, i_f, _ = run_forward(w)                                     # T = 128 takes a single launch by default
     mb.meteora_set_tuning("fused", 0)
     try:
         y_c, i_c, _ = run_forward(w)
