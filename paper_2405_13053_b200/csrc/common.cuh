@@ -103,6 +103,7 @@ bool decode_group_supported(const meteora_shape_t& s, const int* d_outs, int n_m
 int launch_decode_group(const void* x, const GroupModule* mods, int n_modules, const meteora_shape_t& s,
                         int32_t* status, float* part_g, int32_t* tile_ctr, cudaStream_t st);
 int describe_plan(const meteora_shape_t& s, char* buf, size_t n);
+int set_wait_limit_us(int us);   // limit of the bounded device-side waits on the current device (0: default)
 int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
 // streamed decode kernel (wgemm_tcgen05.cu + decode_stream.cuh): up to 128 tokens, two launches resident at a time

@@ -88,11 +88,11 @@ __device__ __forceinline__ void bulk_store_block(void* gdst, uint32_t smem_src, 
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-// Bounded wait until *ctr >= target; false if it did not happen within kWaitLimitCycles.
+// Bounded wait until *ctr >= target; false if it did not happen within the wait limit.
 __device__ __forceinline__ bool wait_counter(const int32_t* ctr, int target) {
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = g_wait_limit_cycles;
     while (ld_acquire(ctr) < target) {
-        if (clock64() - t0 > kWaitLimitCycles) return false;
+        if (clock64() - t0 > limit) return false;
         __nanosleep(32);
     }
     return true;

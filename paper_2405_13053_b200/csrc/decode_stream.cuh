@@ -73,9 +73,9 @@ __device__ __forceinline__ void bulk_load_block(uint32_t smem_dst, const void* g
 // Bounded wait until *ctr >= target with a longer pause between looks than wait_counter: over a hundred CTAs watch
 // the same cache line that others add to, and every look is a request to that line.
 __device__ __forceinline__ bool wait_counter_slow(const int32_t* ctr, int target, unsigned pause_ns) {
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = g_wait_limit_cycles;
     while (ld_acquire(ctr) < target) {
-        if (clock64() - t0 > kWaitLimitCycles) return false;
+        if (clock64() - t0 > limit) return false;
         __nanosleep(pause_ns);
     }
     return true;
@@ -395,6 +395,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                 bulk_load_block(ring + idx_off, d.topk_idx, idx_bytes, bar_route);
                 bulk_load_block(ring + uw_off, d.uw, uw_bytes, bar_route);
                 if (atomicAdd_block(s_done, 1) == 1) stream_count_out(d);   // the CTA reads no workspace counter any more
+                mbar_wait(bar_route, 0);    // own copies have landed before the CTA may leave (the epilogue may have given up)
             }
         } else if (warp == 1) {
             if (lane == 0) {
@@ -436,6 +437,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                                         d.part_g + (size_t)(tile * S + c) * ((size_t)d.BN * kBM) + (size_t)ntok * 4 * q0, one,
                                         bar_land);
                 if (atomicAdd_block(s_done, 1) == 1) stream_count_out(d);
+                mbar_wait(bar_land, 0);     // own copies have landed before the CTA may leave
             }
         } else {
             // B rows of this CTA's row slice for every adapter: weights, staged before the wait

@@ -73,10 +73,10 @@ __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) 
 // Bounded wait on a barrier that threads of the peer CTA arrive on.
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
     if (mbar_try_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = g_wait_limit_cycles;
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_cluster(bar, parity)) return true;
-        if ((spin & 0x3FF) == 0 && clock64() - t0 > kWaitLimitCycles) return false;
+        if ((spin & 0x3FF) == 0 && clock64() - t0 > limit) return false;
     }
 }
 // fp32 accumulate, bf16 x bf16, both operands K-major, M = 256 over the pair, N = 256.

@@ -34,7 +34,9 @@ constexpr int kUmmaK = 16;     // contraction elements per tcgen05.mma (32 bytes
 constexpr int kThreads = 320;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2-9: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kWTileBytes = kBM * kBK * 2;
-constexpr long long kWaitLimitCycles = 2000000000LL;  // about a second
+constexpr long long kDefaultWaitLimitCycles = 2000000000LL;  // about a second
+// Limit of every bounded device-side wait in SM clock cycles (knob wait_limit_us; one value per device).
+__device__ long long g_wait_limit_cycles = kDefaultWaitLimitCycles;
 constexpr int kMaxZSplits = 32;
 
 enum { MODE_STACKED = 0, MODE_LORA = 1 };
@@ -114,13 +116,13 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitLimitCycles.
+// Bounded wait: false if the phase did not complete within the wait limit.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = g_wait_limit_cycles;
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try(bar, parity)) return true;
-        if ((spin & 0x3FF) == 0 && clock64() - t0 > kWaitLimitCycles) return false;
+        if ((spin & 0x3FF) == 0 && clock64() - t0 > limit) return false;
     }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
@@ -1822,6 +1824,12 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
                     "smem=%zu expand=%s",
                     fp.why, row_tiles * pl.splits * pl.n_tiles, pl.splits, pl.BN, pl.stages, pl.kc, pl.smem,
                     pl.lora_mma ? "mma" : "simt");
+}
+
+// Knob wait_limit_us: the limit of the bounded device-side waits on the current device (0: the default, about a second).
+int set_wait_limit_us(int us) {
+    const long long cycles = us > 0 ? (long long)us * 2000LL : kDefaultWaitLimitCycles;   // ~2 GHz SM clock
+    return cuda_status(cudaMemcpyToSymbol(g_wait_limit_cycles, &cycles, sizeof(cycles)));
 }
 
 }  // namespace meteora
