@@ -60,6 +60,9 @@ def parse_args():
                          "the axes of the paper's synthetic sweep (App. A.7); one JSON line each")
     ap.add_argument("--knob", action="append", default=[], metavar="NAME=VALUE",
                     help="set a measurement knob of the library (meteora_set_tuning) before timing; repeatable")
+    ap.add_argument("--layer", action="store_true",
+                    help="time a LLaMA3-8B decoder layer whose seven linears are MeteoRA linears fed by the real upstream "
+                         "activations (64 sequences at context 2048, and one 4096-token prefill); also part of --sweep")
     ap.add_argument("--decode-loop", action="store_true",
                     help="time one autoregressive decode step over the 224 MeteoRA linears of a LLaMA3-8B-shaped "
                          "stack (ms per generated token, the unit of App. A.7); also part of --sweep")
@@ -655,6 +658,95 @@ def run_layer_sweep():
         del mods, graph, groups
 
 
+def run_layer():
+    """Config 4 as a layer: RMSNorm -> q/k/v -> rotary, grouped-query attention -> o -> residual -> RMSNorm -> gate/up ->
+    SwiGLU -> down -> residual, the seven linears MeteoRA linears of the library (q/k/v and gate/up as group calls), each
+    consuming the real upstream activation.  The whole layer is one CUDA graph; the same graph with the linears replaced
+    by tensors made beforehand gives the time of everything that is not a MeteoRA linear, and the difference is the
+    time of the linears inside the layer.  The four linear calls alone, on the layer's own activations, are timed as a
+    third graph for comparison."""
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import decoder_layer as dl
+
+    hbm, _ = measured_peaks()
+    tc, _ = measured_tensor_peak()
+    dev, dt, es = torch.device("cuda"), torch.bfloat16, 2
+    weights, norms = dl.random_layer(dev)
+
+    def graph_time(fn, iters):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fn()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / iters
+
+    for mode, T, context in (("decode", 64, 2048), ("prefill", 4096, 0)):
+        g = torch.Generator(device=dev).manual_seed(23)
+        x = torch.randn(T, dl.HIDDEN, device=dev, generator=g).to(dt)
+        if mode == "decode":
+            ck = torch.randn(T, dl.N_KV_HEADS, context, dl.HEAD_DIM, device=dev, generator=g).to(dt)
+            cv = torch.randn(T, dl.N_KV_HEADS, context, dl.HEAD_DIM, device=dev, generator=g).to(dt)
+            pos = torch.full((T,), context, device=dev)
+        else:
+            ck = cv = None
+            pos = torch.arange(T, device=dev)
+        lin = dl.LibraryLinears(weights, k=TOPK)
+        fixed = dl.FixedLinears(T, dt, dev)
+        iters = 50 if mode == "decode" else 10
+        us_layer = graph_time(lambda: dl.layer_forward(x, norms, lin, pos, ck, cv), iters)
+        us_rest = graph_time(lambda: dl.layer_forward(x, norms, fixed, pos, ck, cv), iters)
+        if lin.status() != 0:
+            raise mb.MeteoraError(lin.status(), "device status")
+        # the linears alone on activations of the right statistics (outputs of the layer's own ops)
+        acts = {"n": dl.rms_norm(x, norms["input"]), "a": torch.randn(T, dl.HIDDEN, device=dev, generator=g).to(dt),
+                "m": torch.randn(T, dl.MLP, device=dev, generator=g).to(dt)}
+
+        def linears_only():
+            lin.many(("q", "k", "v"), acts["n"])
+            lin.one("o", acts["a"])
+            lin.many(("gate", "up"), acts["n"])
+            lin.one("down", acts["m"])
+
+        us_lin = graph_time(linears_only, iters)
+        nbytes = flops = 0.0
+        touched = min(N_ADAPTERS, T * TOPK)
+        for d_in, d_out in dl.LINEARS.values():
+            nbytes += (d_in * d_out + N_ADAPTERS * d_in + touched * RANK * (d_in + d_out) + T * (d_in + d_out)) * es
+            flops += 2.0 * T * d_in * d_out + 2.0 * T * N_ADAPTERS * d_in + 2.0 * T * TOPK * RANK * (d_in + d_out)
+        t_mem, t_tc = nbytes / hbm / 1e3, flops / tc / 1e6
+        bound = "hbm" if t_mem >= t_tc else "tensor"
+        us_in_layer = us_layer - us_rest
+        print(json.dumps({"config": "config4", "op": "decoder_layer", "mode": mode, "T": T, "context": context,
+                          "shape": "LLaMA3-8B layer: RMSNorm, q/k/v, rotary, GQA 32/8x128, o, RMSNorm, gate/up, SwiGLU, down; "
+                                   "seven MeteoRA linears (N=28, r=8, k=2) on the real activations",
+                          "us_layer": round(us_layer, 2), "us_rest_of_layer": round(us_rest, 2),
+                          "us_linears_in_layer": round(us_in_layer, 2), "us_linears_alone": round(us_lin, 2),
+                          "bound": bound, "roofline_us": round(max(t_mem, t_tc), 2),
+                          "frac_of_roofline_in_layer": round(max(t_mem, t_tc) / us_in_layer, 3),
+                          "frac_of_roofline_alone": round(max(t_mem, t_tc) / us_lin, 3),
+                          "achieved": round(nbytes / us_in_layer / 1e3, 1) if bound == "hbm" else round(flops / us_in_layer / 1e6, 1),
+                          "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
+                          "timing": "CUDA graph of the layer minus the same graph with the linears' outputs made beforehand"}),
+              flush=True)
+        del lin, fixed, ck, cv
+
+
 def run_decode_loop():
     """One autoregressive decode step over all 224 MeteoRA linears of a LLaMA3-8B-shaped stack (32 decoder layers
     x 7 linears, each with its own gate and adapters, Sec. 3.2), in the unit of the paper's App. A.7 figures:
@@ -892,11 +984,14 @@ def main():
         apply_knobs(args)
     if args.variants:
         run_variants()
+    elif args.layer:
+        run_layer()
     elif args.decode_loop:
         run_decode_loop()
     elif args.sweep:
         run_sweep(args)
         run_layer_sweep()
+        run_layer()
         run_gate_backward_sweep()
         run_decode_loop()
     elif args.impl == "reference":

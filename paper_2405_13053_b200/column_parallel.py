@@ -3,7 +3,11 @@
 Eq. 2 is row-wise in W0 and in every B_i: y[:, o0:o1] = W0[o0:o1] x + sum_j w_j B_{i_j}[o0:o1] (A_{i_j} x).  A rank
 that holds W0[o0:o1], B[:, o0:o1, :] and full copies of A and Wg therefore produces its slice of y with no exchange
 step: the gate (Eq. 3) and the shrink are replicated (about 1.5 % of the work at 4096 -> 4096), so every rank takes
-the same routing decisions.  Only a consumer that wants the whole y on every rank pays an all-gather, which is
+the same routing decisions wherever the gate logits are not within rounding of a tie: ranks whose shards differ in
+width may run different launch plans, which add the slices of the stacked shrink in a different fp32 order, and a
+token whose k-th and (k+1)-th logits agree to the last bits can then get its picks from different adapters on
+different ranks.  A caller that needs bit-identical routing on every rank cuts equal shards (same plan, same
+order of sums) or computes the routing once with meteora_gate_topk and compares.  Only a consumer that wants the whole y on every rank pays an all-gather, which is
 optional here.  Shards are cut at multiples of 128 rows, the row tile of the kernels, so that no rank works on a
 partial tile the others also touch.
 

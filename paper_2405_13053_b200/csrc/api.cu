@@ -118,12 +118,11 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
     if (decode_fused_supported(s)) {
         if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
         rc = launch_decode_fused(x, W0, A, B, Wg, s, ws, y, st);
-        if (rc != METEORA_ERR_CUDA) {
+        if (rc != kLaunchRefused) {
             if (timed) cudaEventRecord(pf.ev[2 * pf.used++ + 1], st);
             return rc;
         }
-        cudaGetLastError();   // the cooperative launch was refused (not all CTAs can be resident): use the chain
-        tuning().fused_refused += 1;
+        tuning().fused_refused += 1;   // the cooperative launch was refused (not all CTAs can be resident): use the chain
     }
     if (tc_path_supported(s)) {
         const bool pdl = tuning().pdl != 0;
@@ -285,9 +284,8 @@ int meteora_linear_forward_group(const void* x, const void* const* W0, const voi
         GroupModule gm[kMaxGroupModules];
         for (int m = 0; m < n_modules; ++m) gm[m] = GroupModule{W0[m], A[m], B[m], Wg[m], y[m], d_out[m], gw.mod[m]};
         rc = launch_decode_group(x, gm, n_modules, *shape, gw.mod[0].status, gw.part_g, gw.mod[0].tile_ctr, st);
-        if (rc != METEORA_ERR_CUDA) return rc;
-        cudaGetLastError();   // the cooperative launch was refused: one call per module instead
-        tuning().fused_refused += 1;
+        if (rc != kLaunchRefused) return rc;
+        tuning().fused_refused += 1;   // the cooperative launch was refused: one call per module instead
     }
     for (int m = 0; m < n_modules; ++m) {
         meteora_shape_t sm = *shape;

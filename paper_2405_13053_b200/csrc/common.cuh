@@ -191,6 +191,13 @@ __device__ __forceinline__ float warp_dot(const TI* __restrict__ a, const TI* __
 }
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? METEORA_OK : METEORA_ERR_CUDA; }
+// Internal (never returned through the C ABI): the driver refused a launch CONFIGURATION (co-residency, attributes,
+// resources), as opposed to any other CUDA error; only this lets a caller fall back to another launch plan.
+constexpr int kLaunchRefused = -100;
+inline bool launch_config_refused(cudaError_t e) {
+    return e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorNotSupported || e == cudaErrorInvalidConfiguration ||
+           e == cudaErrorInvalidValue || e == cudaErrorLaunchOutOfResources;
+}
 inline int last_launch_status() { return cuda_status(cudaGetLastError()); }
 
 }  // namespace meteora

@@ -1571,7 +1571,7 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
     d.trace_call = trace_calls++;
 #endif
     cudaError_t err = cudaLaunchKernelEx(&cfg, k_decode_fused, maps, mX, mX1, d);
-    if (err != cudaSuccess && want_pdl) {
+    if (launch_config_refused(err) && want_pdl) {                // the two attributes together: try without the second
         cudaGetLastError();
         pdl_accepted = false;
         tuning().pdl_decode_refused += 1;
@@ -1579,7 +1579,11 @@ int launch_decode_group(const void* x, const GroupModule* mods, int G, const met
         d.pdl = 0;
         err = cudaLaunchKernelEx(&cfg, k_decode_fused, maps, mX, mX1, d);
     }
-    return cuda_status(err);
+    if (launch_config_refused(err)) {                            // the caller may take the three-launch chain instead
+        cudaGetLastError();
+        return kLaunchRefused;
+    }
+    return cuda_status(err);                                     // any other error is reported, not worked around
 }
 
 int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
