@@ -34,6 +34,8 @@ METRIC = "MeteoRA-linear tokens/s at LLaMA3-8B shapes (N=28, r=8, k=2)"
 D_IN = D_OUT = 4096
 N_ADAPTERS, RANK, TOPK = 28, 8, 2
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0          # the figure quoted for the part (7.7 - 8 TB/s); context beside the measured peak
+NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, nominal
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
@@ -47,6 +49,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--tokens", type=int, default=128, help="decode batch T per module")
+    ap.add_argument("--repeats", type=int, default=5,
+                    help="the timed region of --steps steps is run this many times; the line reports the median region "
+                         "(value, ms_per_step) and the spread")
+    ap.add_argument("--no-prefill-line", action="store_true", help="skip the prefill_roofline measurement")
     ap.add_argument("--modules", type=int, default=16, help="independent MeteoRA modules visited per step")
     ap.add_argument("--launch", choices=["graph", "stream"], default="graph")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target length of the cpu_baseline sample")
@@ -60,6 +66,9 @@ def parse_args():
                          "the axes of the paper's synthetic sweep (App. A.7); one JSON line each")
     ap.add_argument("--knob", action="append", default=[], metavar="NAME=VALUE",
                     help="set a measurement knob of the library (meteora_set_tuning) before timing; repeatable")
+    ap.add_argument("--standalone", action="store_true",
+                    help="time the standalone entry points (gate + top-k, bucketing, LoRA term by segments) beside the fused "
+                         "forward's stacked shrink + selection; also part of --sweep")
     ap.add_argument("--layer", action="store_true",
                     help="time a LLaMA3-8B decoder layer whose seven linears are MeteoRA linears fed by the real upstream "
                          "activations (64 sequences at context 2048, and one 4096-token prefill); also part of --sweep")
@@ -208,6 +217,69 @@ def whole_job_value(modules, tokens, world, steps, ms_total):
     return modules * tokens * world * steps / (ms_total * 1e-3)
 
 
+def prefill_line(mb, lib, tc_peak, tc_kind, hbm_peak):
+    """One prefill figure for the default line (the headline workload is a decode batch and HBM-bound): config 2's
+    gate/up shape, 4096 -> 14336 with 2048 tokens from 4 clusters, the whole MeteoRA linear per call (three launches:
+    stacked shrink, selection, base product with the expand) against the sustained bf16 tensor peak, and the
+    base-product kernel alone from event pairs around its launches."""
+    import ctypes
+
+    import torch
+
+    from paper_2405_13053_b200 import workloads
+
+    d_in, d_out, T = workloads.CONFIG2_SHAPES["gate_up"][0], workloads.CONFIG2_SHAPES["gate_up"][1], 2048
+    dt = torch.bfloat16
+    g = torch.Generator(device="cuda").manual_seed(29)
+    x = torch.from_numpy(workloads.make_x(T, d_in, "clusters", 2001, "bf16")).to(dt).cuda()
+    W0 = (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt)
+    A = ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt)
+    B = (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt)
+    Wg = (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt)
+    y = torch.empty(T, d_out, device="cuda", dtype=dt)
+    shape = mb.make_shape(T, d_in, d_out, N_ADAPTERS, RANK, TOPK, dt)
+    ws = mb.alloc_workspace(shape)
+
+    def call():
+        rc = lib.meteora_linear_forward(x.data_ptr(), W0.data_ptr(), A.data_ptr(), B.data_ptr(), Wg.data_ptr(),
+                                        ctypes.byref(shape), y.data_ptr(), ws.data_ptr(), ws.numel(),
+                                        torch.cuda.current_stream().cuda_stream)
+        if rc != 0:
+            raise mb.MeteoraError(rc, "meteora_linear_forward")
+
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    regions = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        regions.append(e0.elapsed_time(e1) * 1e3 / 20)
+    us_call = float(np.median(regions))
+    mb.meteora_profile_begin(20)
+    for _ in range(20):
+        call()
+    ms, n = mb.meteora_profile_end()
+    if mb.meteora_workspace_status(ws) != 0:
+        raise mb.MeteoraError(-6, "device status after the prefill region")
+    us_base = ms * 1e3 / max(n, 1)
+    flops = 2.0 * T * d_in * d_out + 2.0 * T * N_ADAPTERS * d_in + 2.0 * T * TOPK * RANK * (d_in + d_out)
+    flops_base = 2.0 * T * d_in * d_out + 2.0 * T * TOPK * RANK * d_out
+    plan = mb.meteora_describe_plan(shape).split(" fused_refused")[0]
+    return {"workload": f"config2 gate_up: 4096->14336 MeteoRA linear, N=28 r=8 k=2, bf16, prefill batch T={T} (4 clusters)",
+            "bound": "tensor", "unit": "TFLOP/s", "peak": tc_peak, "peak_kind": f"of {tc_kind} (sustained dense bf16)",
+            "us_per_call": us_call, "us_per_call_min": min(regions), "us_per_call_max": max(regions),
+            "algorithmic_flops_per_call": flops, "achieved": flops / us_call / 1e6, "frac": flops / us_call / 1e6 / tc_peak,
+            "frac_of_nominal": flops / us_call / 1e6 / NOMINAL_BF16_TFLOPS,
+            "base_product_kernel": {"us_per_launch": us_base, "achieved": flops_base / us_base / 1e6,
+                                    "frac": flops_base / us_base / 1e6 / tc_peak, "launches_timed": n},
+            "launches_per_call": 3, "plan": plan}
+
+
 # --------------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -340,8 +412,10 @@ def run_ours(args):
     uuid = str(torch.cuda.get_device_properties(local).uuid)
     uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
     sampler = ClockSampler(uuid)
-    ms_total = timed(run_dev, K, W)
-    # keep the GPU under the same load a little longer if the region was too short for a clock sample
+    reps = max(1, args.repeats)
+    regions = [timed(run_dev, K, W if i == 0 else 0) for i in range(reps)]     # every region: exactly K steps
+    ms_total = float(np.median(regions))
+    # keep the GPU under the same load a little longer if the regions were too short for a clock sample
     t_extra = time.time()
     while time.time() - t_extra < 0.7:
         run_dev()
@@ -357,7 +431,8 @@ def run_ours(args):
         run_e2e()
         torch.cuda.current_stream().synchronize()          # the step's result is read on the host
 
-    ms_e2e = timed(e2e_step, K, W)
+    e2e_regions = [timed(e2e_step, K, W if i == 0 else 0) for i in range(reps)]
+    ms_e2e = float(np.median(e2e_regions))
     check_status()
     e2e_value = whole_job_value(R, T, world, K, ms_e2e)
 
@@ -415,6 +490,11 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
+        "repeats": {"regions": reps, "steps_per_region": K, "statistic": "median",
+                    "ms_per_step_min": min(regions) / K, "ms_per_step_median": ms_total / K,
+                    "ms_per_step_max": max(regions) / K,
+                    "value_best": whole_job_value(R, T, world, K, min(regions)),
+                    "value_worst": whole_job_value(R, T, world, K, max(regions))},
         "config": {"workload": f"config1: LLaMA3-8B q_proj MeteoRA linear 4096->4096, N=28 r=8 k=2, bf16, "
                                f"{'decode' if T <= 256 else 'prefill'} batch T={T}; step = {R} independent modules",
                    "tokens_per_module": T, "modules_per_step": R, "launch": mode, "e2e_launch": mode_e2e, "e2e_streams": len(e2e_streams),
@@ -423,16 +503,20 @@ def run_ours(args):
                    "workspace": "one scratch buffer shared by the step's stream-ordered calls (one per stream end to end)",
                    "parallelism": f"token-sharded replicas x{world}, no collective", "plan": plan},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": R * T * D_IN * es,
-                "d2h_bytes_per_step": R * T * D_OUT * es, "ms_per_step": ms_e2e / K},
+                "d2h_bytes_per_step": R * T * D_OUT * es, "ms_per_step": ms_e2e / K,
+                "ms_per_step_min": min(e2e_regions) / K, "ms_per_step_max": max(e2e_regions) / K},
         "gpu_launches": launches_per_call * R * K,
         "clocks": clocks,
         "roofline": ({"bound": "tensor", "kernel": kernel_name, "achieved": flops_kernel / per_launch_s / 1e12,
                       "peak": tc_peak, "peak_kind": f"of {tc_kind} (sustained dense bf16)", "unit": "TFLOP/s",
                       "frac": flops_kernel / per_launch_s / 1e12 / tc_peak, "traffic": None,
+                      "frac_of_nominal": flops_kernel / per_launch_s / 1e12 / NOMINAL_BF16_TFLOPS,
+                      "nominal_peak": NOMINAL_BF16_TFLOPS,
                       "algorithmic_flops_per_launch": flops_kernel, "us_per_launch": per_launch_s * 1e6,
                       "launches_timed": kernel_launches} if tensor_bound else
                      {"bound": "hbm", "kernel": kernel_name, "achieved": achieved,
                       "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                      "frac_of_nominal": achieved / NOMINAL_HBM_GBS, "nominal_peak": NOMINAL_HBM_GBS,
                       "traffic": traffic, "algorithmic_bytes_per_launch": bytes_kernel,
                       "us_per_launch": per_launch_s * 1e6, "launches_timed": kernel_launches}),
         "path_roofline": ({"bound": "tensor", "algorithmic_flops_per_call": flops_path, "us_per_call": per_call_s * 1e6,
@@ -443,6 +527,9 @@ def run_ours(args):
                            "achieved": bytes_path / per_call_s / 1e9, "peak": peak, "unit": "GB/s",
                            "frac": bytes_path / per_call_s / 1e9 / peak, "adapters_touched": touched}),
     }
+
+    if world == 1 and not args.no_prefill_line:
+        line["prefill_roofline"] = prefill_line(mb, lib, tc_peak, tc_kind, peak)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
@@ -455,8 +542,20 @@ def run_ours(args):
             oracle.linear_forward(w["x"][sl], w["W0"], w["A"], w["B"], w["Wg"], w.k)
             t_cpu += time.perf_counter() - t0
             n_tok += chunk
+        # the same oracle on one core (a short sample: ~3 s)
+        oracle.set_threads(1)
+        n1, t1 = 0, 0.0
+        while t1 < 3.0 and n1 < 4096:
+            t0 = time.perf_counter()
+            oracle.linear_forward(w["x"][:1], w["W0"], w["A"], w["B"], w["Wg"], w.k)
+            t1 += time.perf_counter() - t0
+            n1 += 1
+        oracle.set_threads(cores)
         line["cpu_baseline"] = {"value": n_tok / t_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                                "sample": f"{n_tok} tokens of module 0 in chunks of {chunk} ({t_cpu:.1f} s)"}
+                                "sample": f"{n_tok} tokens of module 0 in chunks of {chunk} ({t_cpu:.1f} s)",
+                                "value_1core": n1 / t1, "sample_1core": f"{n1} tokens one at a time ({t1:.1f} s)",
+                                "note": "the oracle as it stands: plain C, fp64 accumulation, -O2 -ffp-contract=off, "
+                                        "OpenMP over tokens; never tuned"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -747,6 +846,90 @@ def run_layer():
         del lin, fixed, ck, cv
 
 
+def run_standalone_sweep():
+    """The standalone entry points (gate + top-k, bucketing, LoRA term by per-adapter segments) at config 1 (T = 128) and
+    config 2 (4096 -> 14336, T = 2048), each against the HBM time of its algorithmic bytes, beside what the fused
+    forward spends on the same job with the stacked dense shrink [A; Wg] x on the tensor cores plus the selection
+    (time of a three-launch call minus its base-product launch).  This is the measured side of "per-adapter segments
+    or one stacked dense shrink" (Sec. 3.3's gather against Eq. 5's batched view)."""
+    import torch
+
+    from paper_2405_13053_b200 import binding as mb
+    from paper_2405_13053_b200 import workloads
+
+    hbm, _ = measured_peaks()
+    dt, es = torch.bfloat16, 2
+
+    def timed_us(fn, iters=50):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / iters
+
+    for cfg, d_in, d_out, T, x_kind in (("config1", 4096, 4096, 128, "rms"), ("config2", 4096, 14336, 2048, "clusters")):
+        g = torch.Generator(device="cuda").manual_seed(9)
+        x = torch.from_numpy(workloads.make_x(T, d_in, x_kind, 5, "bf16")).to(dt).cuda()
+        W0 = (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt)
+        A = ((torch.rand(N_ADAPTERS, RANK, d_in, device="cuda", generator=g) * 2 - 1) / d_in ** 0.5).to(dt)
+        B = (0.01 * torch.randn(N_ADAPTERS, d_out, RANK, device="cuda", generator=g)).to(dt)
+        Wg = (torch.randn(N_ADAPTERS, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt)
+        shape = mb.make_shape(T, d_in, d_out, N_ADAPTERS, RANK, TOPK, dt)
+        ws = mb.alloc_workspace(shape)
+        idx, w, _ = mb.meteora_gate_topk(x, Wg, TOPK)
+        idx, w = idx.clone(), w.clone()
+        counts, offsets, perm = mb.meteora_route(idx, N_ADAPTERS)
+        touched = int((counts > 0).sum().item())
+        rows = []
+        us = timed_us(lambda: mb.meteora_gate_topk(x, Wg, TOPK))
+        rows.append(("meteora_gate_topk (k_gate_topk)", us, (T * d_in + N_ADAPTERS * d_in) * es + T * TOPK * 8))
+        us = timed_us(lambda: mb.meteora_route(idx, N_ADAPTERS))
+        rows.append(("meteora_route (k_route)", us, T * TOPK * 8 + (2 * N_ADAPTERS + 1) * 4))
+        us = timed_us(lambda: mb.meteora_lora_delta(x, A, B, idx, w, offsets, perm, workspace=ws))
+        rows.append(("meteora_lora_delta (k_shrink_segments + k_expand)", us,
+                     (T * d_in + touched * RANK * (d_in + d_out)) * es + T * d_out * 4 + 2 * T * TOPK * RANK * 4))
+        # the fused forward's side of the same job: three-launch chain, whole call minus its base-product launch
+        y = torch.empty(T, d_out, device="cuda", dtype=dt)
+        mb.meteora_set_tuning("fused", 0)
+        try:
+            call = lambda: mb.meteora_linear_forward(x, W0, A, B, Wg, TOPK, workspace=ws, out=y)
+            us_call = timed_us(call, 20)
+            call()
+            torch.cuda.synchronize()
+            mb.meteora_profile_begin(8)
+            for _ in range(8):
+                call()
+            ms, n = mb.meteora_profile_end()
+        finally:
+            mb.meteora_set_tuning("fused", 1)
+        us_base = ms * 1e3 / max(n, 1)
+        stacked_bytes = (T * d_in + (N_ADAPTERS * RANK + N_ADAPTERS) * d_in) * es + T * TOPK * (RANK + 2) * 4
+        rows.append(("stacked dense shrink [A; Wg] x on tcgen05 + selection (three-launch call minus its base product)",
+                     us_call - us_base, stacked_bytes))
+        seg_total = sum(r[1] for r in rows[:3])
+        for name, us, nbytes in rows:
+            print(json.dumps({"op": "standalone", "config": cfg, "shape": f"{d_in}->{d_out}", "T": T, "kernel": name,
+                              "us": round(us, 2), "algorithmic_bytes": int(nbytes), "bound": "hbm",
+                              "roofline_us": round(nbytes / hbm / 1e3, 3),
+                              "frac_of_roofline": round(nbytes / hbm / 1e3 / us, 4), "adapters_touched": touched}), flush=True)
+        print(json.dumps({"op": "segments_vs_stacked", "config": cfg, "shape": f"{d_in}->{d_out}", "T": T,
+                          "us_segments_path (gate_topk + route + shrink by segments + expand)": round(seg_total, 2),
+                          "us_stacked_path (stacked shrink + selection; the expand rides in the base product)":
+                              round(us_call - us_base, 2),
+                          "us_three_launch_call": round(us_call, 2), "us_base_product_launch": round(us_base, 2)}), flush=True)
+
+
 def run_decode_loop():
     """One autoregressive decode step over all 224 MeteoRA linears of a LLaMA3-8B-shaped stack (32 decoder layers
     x 7 linears, each with its own gate and adapters, Sec. 3.2), in the unit of the paper's App. A.7 figures:
@@ -986,12 +1169,15 @@ def main():
         run_variants()
     elif args.layer:
         run_layer()
+    elif args.standalone:
+        run_standalone_sweep()
     elif args.decode_loop:
         run_decode_loop()
     elif args.sweep:
         run_sweep(args)
         run_layer_sweep()
         run_layer()
+        run_standalone_sweep()
         run_gate_backward_sweep()
         run_decode_loop()
     elif args.impl == "reference":
