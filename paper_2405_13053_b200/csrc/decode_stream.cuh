@@ -70,6 +70,15 @@ __device__ __forceinline__ void bulk_load_block(uint32_t smem_dst, const void* g
                  : "memory");
 }
 
+// 3-D tile load of a CTA pair: the completion bytes go to a barrier that may live in the pair's other CTA.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2,
+                                                 uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"((uint64_t)tm), "r"(c0), "r"(c1), "r"(c2), "r"(cluster_bar)
+        : "memory");
+}
+
 // Bounded wait until *ctr >= target with a longer pause between looks than wait_counter: over a hundred CTAs watch
 // the same cache line that others add to, and every look is a request to that line.
 __device__ __forceinline__ bool wait_counter_slow(const int32_t* ctr, int target, unsigned pause_ns) {
@@ -150,6 +159,13 @@ __device__ __forceinline__ void row_slice(int j, int S, int& q0, int& nq) {
     nq = 32 * (j + 1) / S - q0;
 }
 
+// kPair: the grid runs in clusters of two CTAs and a pair of main CTAs multiplies TWO row tiles of W0 (one each) with
+// the same slice of the contraction axis by tcgen05.mma.cta_group::2: each CTA loads its own 128 rows of W0 but only
+// HALF of the token tile, and the tensor cores of both SMs read both halves.  At 128 tokens the token tile is as large
+// as the W0 tile, so this takes a quarter off what an SM takes in and lets the ring hold four stages instead of three.
+// No load is multicast; every copy of the pair signals the leader's barrier, which expects both CTAs' bytes; the
+// leader alone issues MMAs and releases stages by commits that arrive in both CTAs.  Aux CTAs work alone as before.
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 2)
 k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmA,
                 const __grid_constant__ CUtensorMap tmAt, const __grid_constant__ CUtensorMap tmG,
@@ -159,9 +175,10 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;
     uint8_t* ring_ptr = smem_raw + (ring - raw);
-    const uint32_t x_tile_bytes = d.BN * 128;
+    const uint32_t aux_x_bytes = d.BN * 128;                                  // an aux CTA takes the whole token tile
+    const uint32_t x_tile_bytes = kPair ? d.BN * 64 : d.BN * 128;             // a main CTA of a pair half of it
     const uint32_t stage_bytes = d.kc * (kWTileBytes + x_tile_bytes);
-    const uint32_t aux_stage_bytes = kWTileBytes + x_tile_bytes;
+    const uint32_t aux_stage_bytes = kWTileBytes + aux_x_bytes;
     const uint32_t ring_bytes = (uint32_t)d.ring_bytes;
     const uint32_t bar_base = ring + ring_bytes;              // full[slots], empty[slots], acc, land, route, deliv
     const uint32_t bar_acc = bar_base + 2 * d.bar_slots * 8;
@@ -182,13 +199,25 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"((uint32_t)d.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (kPair && !is_aux) {                                               // the pair-wide form, by both CTAs
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                         "r"((uint32_t)d.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                         "r"((uint32_t)d.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
-    __syncthreads();
+    if (kPair) {
+        __syncwarp();
+        cluster_sync();                                                       // both CTAs' barriers exist before anyone signals
+    } else {
+        __syncthreads();
+    }
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
     // The next launch on the stream may become resident from here on (it only touches weights until this
@@ -233,7 +262,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                 STREAM_STAMP(1);
                 for (int i = 0; i < pre; ++i) {
                     const uint32_t full = bar_base + i * 8, dst = ring + i * aux_stage_bytes;
-                    mbar_expect_tx(full, x_tile_bytes);
+                    mbar_expect_tx(full, aux_x_bytes);
                     tma_load_3d(dst + kWTileBytes, &tmX1, 0, 0, ks0 + i, full);
                 }
                 bool ok = true;
@@ -336,7 +365,13 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
         // ================================================================== main CTA
         const int main_id = (int)blockIdx.x - d.n_aux;
         const int S = d.S;
-        const int tile = main_id / S, j = main_id - tile * S;
+        // alone: CTA = (tile, slice j); in pairs: pair = (two adjacent tiles, slice j), the CTA's rank picks the tile
+        const uint32_t rank = kPair ? cluster_rank() : 0u;
+        const bool leader = rank == 0;
+        const int tile = kPair ? 2 * ((main_id >> 1) / S) + (int)rank : main_id / S;
+        const int j = kPair ? (main_id >> 1) % S : main_id - tile * S;
+        const bool live = tile < d.row_tiles;                       // an odd tile count leaves the last pair's second CTA without rows
+        const int slot_id = tile * S + j;                            // this CTA's partial tile in the scratch
         const int nst = d.ksteps / d.kc;                             // stages of the whole contraction axis
         const int it0 = nst * j / S, it1 = nst * (j + 1) / S;
         const int n_it = it1 - it0;
@@ -356,29 +391,41 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
         if (warp == 0) {
             if (lane == 0) {
                 const uint32_t w_bytes = d.kc * kWTileBytes, xs_bytes = d.kc * x_tile_bytes;
+                const uint32_t both = kPair ? 2u : 1u;               // the leader's barrier expects both CTAs' bytes
+                const int tok0 = kPair ? (int)rank * (d.BN / 2) : 0;  // own half of the token tile
                 const int pre = min(n_it, d.stages);
+                auto full_bar = [&](int s_) {                        // where this CTA's copies report: the leader's barrier
+                    const uint32_t local = bar_base + s_ * 8;
+                    return kPair ? map_to_cta(local, 0) : local;
+                };
+                auto load_w = [&](uint32_t dst, int it, uint32_t bar) {
+                    if (kPair) tma_load_3d_pair(dst, &tmW0, 0, row0, it * d.kc, bar);
+                    else tma_load_3d(dst, &tmW0, 0, row0, it * d.kc, bar);
+                };
+                auto load_x = [&](uint32_t dst, int it, uint32_t bar) {
+                    if (kPair) tma_load_3d_pair(dst, &tmX, 0, tok0, it * d.kc, bar);
+                    else tma_load_3d(dst, &tmX, 0, tok0, it * d.kc, bar);
+                };
                 for (int i = 0; i < pre; ++i) {
-                    const uint32_t full = bar_base + i * 8;
-                    mbar_expect_tx_only(full, w_bytes);
-                    tma_load_3d(ring + i * stage_bytes, &tmW0, 0, row0, (it0 + i) * d.kc, full);
+                    if (leader) mbar_expect_tx_only(bar_base + i * 8, both * w_bytes);
+                    load_w(ring + i * stage_bytes, it0 + i, full_bar(i));
                 }
                 for (int i = pre; i < min(n_it, pre + d.pf_main); ++i) tma_prefetch_l2_3d(&tmW0, 0, row0, (it0 + i) * d.kc);
                 if (d.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
                 STREAM_STAMP(1);
                 for (int i = 0; i < pre; ++i) {
-                    const uint32_t full = bar_base + i * 8;
-                    mbar_expect_tx(full, xs_bytes);
-                    tma_load_3d(ring + i * stage_bytes + w_bytes, &tmX, 0, 0, (it0 + i) * d.kc, full);
+                    if (leader) mbar_expect_tx(bar_base + i * 8, both * xs_bytes);
+                    load_x(ring + i * stage_bytes + w_bytes, it0 + i, full_bar(i));
                 }
                 bool ok = true;
                 int st = pre == d.stages ? 0 : pre, round = pre == d.stages ? 1 : 0;
                 for (int i = pre; i < n_it; ++i) {
                     ok = mbar_wait(bar_base + (d.bar_slots + st) * 8, (round & 1) ^ 1);
                     if (!ok) break;
-                    const uint32_t full = bar_base + st * 8, dst = ring + st * stage_bytes;
-                    mbar_expect_tx(full, stage_bytes);
-                    tma_load_3d(dst, &tmW0, 0, row0, (it0 + i) * d.kc, full);
-                    tma_load_3d(dst + w_bytes, &tmX, 0, 0, (it0 + i) * d.kc, full);
+                    const uint32_t dst = ring + st * stage_bytes;
+                    if (leader) mbar_expect_tx(bar_base + st * 8, both * stage_bytes);
+                    load_w(dst, it0 + i, full_bar(st));
+                    load_x(dst + w_bytes, it0 + i, full_bar(st));
                     if (++st == d.stages) {
                         st = 0;
                         ++round;
@@ -400,38 +447,51 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
         } else if (warp == 1) {
             if (lane == 0) {
                 bool ok = true;
-                int st = 0, round = 0;
-                for (int i = 0; i < n_it; ++i) {
-                    ok = mbar_wait(bar_base + st * 8, round & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t wa = ring + st * stage_bytes, xa = wa + d.kc * kWTileBytes;
-                    for (int c = 0; c < d.kc; ++c) {
-                        const uint64_t da = smem_desc_sw128(wa + c * kWTileBytes);
-                        const uint64_t db = smem_desc_sw128(xa + c * x_tile_bytes);
+                if (leader) {                                        // of a pair, the leader alone issues the MMAs
+                    const uint32_t idesc_main =
+                        kPair ? (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(d.BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24)
+                              : idesc;
+                    int st = 0, round = 0;
+                    for (int i = 0; i < n_it; ++i) {
+                        ok = mbar_wait(bar_base + st * 8, round & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t wa = ring + st * stage_bytes, xa = wa + d.kc * kWTileBytes;
+                        for (int c = 0; c < d.kc; ++c) {
+                            const uint64_t da = smem_desc_sw128(wa + c * kWTileBytes);
+                            const uint64_t db = smem_desc_sw128(xa + c * x_tile_bytes);
 #pragma unroll
-                        for (int kk = 0; kk < kBK / kUmmaK; ++kk)
-                            umma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (i | c | kk) != 0);
+                            for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
+                                if (kPair)
+                                    umma_bf16_pair(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc_main,
+                                                   (i | c | kk) != 0);
+                                else
+                                    umma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc_main,
+                                              (i | c | kk) != 0);
+                            }
+                        }
+                        if (kPair) umma_commit_pair(bar_base + (d.bar_slots + st) * 8);   // both rings may refill the stage
+                        else umma_commit(bar_base + (d.bar_slots + st) * 8);
+                        if (++st == d.stages) {
+                            st = 0;
+                            ++round;
+                        }
                     }
-                    umma_commit(bar_base + (d.bar_slots + st) * 8);
-                    if (++st == d.stages) {
-                        st = 0;
-                        ++round;
-                    }
+                    if (kPair) umma_commit_pair(bar_acc);            // accumulators complete in both CTAs
+                    else umma_commit(bar_acc);
+                    if (!ok) stream_flag_error(d, 2, 200);
                 }
-                umma_commit(bar_acc);
-                if (!ok) stream_flag_error(d, 2, 200);
                 STREAM_STAMP(3);
                 // The other CTAs' partials of this CTA's row slice into the landing area, once the ring is idle and
                 // all S CTAs of the tile have delivered (this CTA's own delivery included).
                 ok = mbar_wait(bar_deliv, 0);                      // not before this CTA's own partial is out
                 if (d.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
-                if (ok && S > 1) ok = wait_counter_slow(d.tile_ctr + tile, S, 100);
+                if (ok && S > 1 && live) ok = wait_counter_slow(d.tile_ctr + tile, S, 100);
                 if (!ok) stream_flag_error(d, 4, 900);
                 STREAM_STAMP(6);
                 const uint32_t one = (uint32_t)(ntok * 4 * nq * 4);
-                mbar_expect_tx(bar_land, (uint32_t)(d.own_local ? S - 1 : S) * one);
-                for (int c = 0; c < S; ++c)
+                mbar_expect_tx(bar_land, live ? (uint32_t)(d.own_local ? S - 1 : S) * one : 0u);
+                for (int c = 0; c < S && live; ++c)
                     if (c != j || !d.own_local)
                         bulk_load_block(ring + c * blk_bytes,
                                         d.part_g + (size_t)(tile * S + c) * ((size_t)d.BN * kBM) + (size_t)ntok * 4 * q0, one,
@@ -441,33 +501,33 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             }
         } else {
             // B rows of this CTA's row slice for every adapter: weights, staged before the wait
-            stage_slab_rows(d.B, d.d_out, d.N, cpa, slab, row0 + 4 * q0, 4 * nq, etid);
+            if (live) stage_slab_rows(d.B, d.d_out, d.N, cpa, slab, row0 + 4 * q0, 4 * nq, etid);
+            // Where this thread's accumulator row goes (worked out before the accumulator is ready): the accumulator
+            // is cut into the S row slices, each stored [token][rows of the slice] so that the CTA that finishes a
+            // slice fetches it as one contiguous block: the own slice straight into the landing area, the others to scratch.
+            const int row_in_tile = quad * 32 + lane;
+            float* land = reinterpret_cast<float*>(ring_ptr);          // the ring is idle once the accumulator is complete
+            int sj = 0, sq0 = 0, snq = 32;                             // the slice this thread's row belongs to
+            for (int c = 0; c < S; ++c) {
+                int a, b;
+                row_slice(c, S, a, b);
+                if (row_in_tile / 4 >= a) {
+                    sj = c;
+                    sq0 = a;
+                    snq = b;
+                }
+            }
+            float* part = sj == j && d.own_local
+                              ? land + (size_t)j * (blk_bytes / 4) + (row_in_tile - 4 * sq0)
+                              : d.part_g + (size_t)slot_id * ((size_t)d.BN * kBM) + (size_t)ntok * 4 * sq0 +
+                                    (row_in_tile - 4 * sq0);
             if (d.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
             bool acc_ok = mbar_wait(bar_acc, 0);
             if (!acc_ok && lane == 0) stream_flag_error(d, 3, 300);
             acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
             tc_fence_after();
             if (etid == 0) STREAM_STAMP(4);
-            const int row_in_tile = quad * 32 + lane;
-            float* land = reinterpret_cast<float*>(ring_ptr);          // the ring is idle from here on
             {
-                // The accumulator, cut into the S row slices, each stored [token][rows of the slice] so that the CTA
-                // that finishes a slice fetches it as one contiguous block: the own slice straight into the landing
-                // area, the others to scratch.
-                int sj = 0, sq0 = 0, snq = 32;                         // the slice this thread's row belongs to
-                for (int c = 0; c < S; ++c) {
-                    int a, b;
-                    row_slice(c, S, a, b);
-                    if (row_in_tile / 4 >= a) {
-                        sj = c;
-                        sq0 = a;
-                        snq = b;
-                    }
-                }
-                float* part = sj == j && d.own_local
-                                  ? land + (size_t)j * (blk_bytes / 4) + (row_in_tile - 4 * sq0)
-                                      : d.part_g + (size_t)main_id * ((size_t)d.BN * kBM) + (size_t)ntok * 4 * sq0 +
-                                            (row_in_tile - 4 * sq0);
                 const int pitch = 4 * snq;
                 for (int c = c_begin; c < c_end; c += 16) {
                     float v[16];
@@ -479,13 +539,13 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                     }
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        if (c + i < ntok) part[(size_t)(c + i) * pitch] = v[i];
+                        if (c + i < ntok && live) part[(size_t)(c + i) * pitch] = v[i];
                 }
                 if (etid == 0) STREAM_STAMP(11);
                 epi_barrier();                                         // also orders the own slice for the threads below
                 if (etid == 0) {
                     STREAM_STAMP(12);
-                    if (S > 1) {
+                    if (S > 1 && live) {
                         __threadfence();
                         STREAM_STAMP(13);
                         atomicAdd(d.tile_ctr + tile, 1);
@@ -500,7 +560,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             const int* s_idx = reinterpret_cast<const int*>(ring_ptr + idx_off);
             const float4* s_uw4 = reinterpret_cast<const float4*>(ring_ptr + uw_off);
             float4* dblk = reinterpret_cast<float4*>(ring_ptr + delta_off);
-            const int items = nq * ntok, slab_rows = 4 * nq;
+            const int items = live ? nq * ntok : 0, slab_rows = 4 * nq;
             for (int it = etid; it < items && ok; it += kEpiThreads) {
                 const int t = it / nq, ql = it - t * nq;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -519,7 +579,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                 dblk[it] = acc;                                      // read back by the same thread below
             }
             if (etid == 0) STREAM_STAMP(8);
-            if (S > 1) ok = mbar_wait(bar_land, 0) && ok;
+            if (S > 1 && live) ok = mbar_wait(bar_land, 0) && ok;
             if (!ok && lane == 0) stream_flag_error(d, 4, 950);
             if (etid == 0) STREAM_STAMP(9);
             const int blk4 = (int)(blk_bytes / 16);
@@ -559,11 +619,19 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
     }
 
     tc_fence_before();
-    __syncthreads();
+    if (kPair) {
+        __syncwarp();
+        cluster_sync();                     // nobody leaves while the pair's other CTA may still signal it
+    } else {
+        __syncthreads();
+    }
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                     "r"((uint32_t)d.tmem_cols)
-                     : "memory");
+        if (kPair && !is_aux)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)d.tmem_cols)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)d.tmem_cols)
+                         : "memory");
     }
 }
 

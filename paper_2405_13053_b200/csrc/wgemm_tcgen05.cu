@@ -699,8 +699,8 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
 }  // namespace meteora
 
 #include "decode_fused.cuh"
-#include "decode_stream.cuh"
 #include "wgemm_pair.cuh"
+#include "decode_stream.cuh"
 
 namespace meteora {
 
@@ -1602,6 +1602,7 @@ struct StreamPlan {
     int BN, kc, stages, aux_stages, tmem_cols, S, n_main, row_tiles;
     int n_aux, a_tiles, aux_tiles, gate_tile, gate_row0, aux_slices;
     int pf_main, pf_aux, slab_off, ring_bytes, ctas_per_sm;
+    int pair;      // main CTAs in pairs (clusters of two, two-CTA MMA): each loads half of the token tile
     size_t smem;
 };
 constexpr int kStreamBarSlots = 16;
@@ -1640,13 +1641,21 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     sp.kc = 1;
     if (tn.kc > 0 && tn.kc <= 4 && ksteps % tn.kc == 0) sp.kc = tn.kc;
     const int nst = ksteps / sp.kc;
-    int S = std::min(8, (sms - sp.n_aux) / sp.row_tiles);
+    // Pairs of main CTAs (knob pair_decode: 0 never, the default; 1 from 64 tokens up; 2 from 17 tokens up): each CTA of
+    // a pair loads half of the token tile, which at 128 tokens is as large as the W0 tile, and the ring gets a fourth
+    // stage.  Measured at 4096 -> 4096: the main loop ends no earlier (8.6 against 8.3 us after the call ahead at 128
+    // tokens, 8.4 against 8.0 at 64) and a call takes 18.1 against 16.9 us and 15.4 against 14.6: the loop waits for W0's
+    // lines, not for the token tile, and the pair adds two cluster barriers.  Kept as a knob, off by default.
+    sp.pair = tn.pair_decode == 0 ? 0 : (s.T >= (tn.pair_decode >= 2 ? 17 : 64) ? 1 : 0);
+    const int tiles_padded = sp.pair ? (sp.row_tiles + 1) / 2 * 2 : sp.row_tiles;
+    if (sp.pair) sp.n_aux = (sp.n_aux + 1) / 2 * 2;              // whole clusters of two
+    int S = std::min(8, (sms - sp.n_aux) / tiles_padded);
     if (tn.splits > 0) S = std::min(tn.splits, 8);
     S = std::min(S, nst);
     // at most two CTAs per SM in all, and the workspace holds row tiles + 148 partial tiles
-    if (S < 1 || sp.row_tiles * S + sp.n_aux > 2 * sms || sp.row_tiles * S > sp.row_tiles + 148) return sp;
+    if (S < 1 || tiles_padded * S + sp.n_aux > 2 * sms || sp.row_tiles * S > sp.row_tiles + 148) return sp;
     sp.S = S;
-    sp.n_main = sp.row_tiles * S;
+    sp.n_main = tiles_padded * S;
     // narrow layers leave SMs idle: give them to the stacked shrink as further slices (all 16 or none)
     if (tn.aux_ctas == 0) {
         const int spare = sms - sp.n_main - sp.n_aux;
@@ -1654,10 +1663,11 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
         if (sp.aux_slices < full && sp.aux_slices + spare / sp.aux_tiles >= full) {
             sp.aux_slices = full;
             sp.n_aux = sp.aux_tiles * sp.aux_slices;
+            if (sp.pair) sp.n_aux = (sp.n_aux + 1) / 2 * 2;
         }
     }
     sp.why = 5;
-    sp.BN = (s.T + 15) / 16 * 16;
+    sp.BN = sp.pair ? (s.T + 31) / 32 * 32 : (s.T + 15) / 16 * 16;
     int cols = 32;
     while (cols < sp.BN) cols *= 2;
     sp.tmem_cols = cols;
@@ -1665,7 +1675,7 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     const int nq_max = (32 + S - 1) / S;
     const size_t slab_bytes = (size_t)s.N * cpa * 4 * nq_max * 16;
     sp.slab_off = (int)align_up((size_t)(2 * kStreamBarSlots + 4) * 8 + 16, 128);
-    const size_t stage_bytes = (size_t)sp.kc * (kWTileBytes + (size_t)sp.BN * 128);
+    const size_t stage_bytes = (size_t)sp.kc * (kWTileBytes + (size_t)sp.BN * (sp.pair ? 64 : 128));
     const size_t aux_stage_bytes = kWTileBytes + (size_t)sp.BN * 128;
     const int ntok = s.T;
     // what the last step fetches into the idle ring: S row slices of partial tiles (or the CTA's own tile), the
@@ -1725,7 +1735,7 @@ int launch_decode_stream(const void* x, const void* W0, const void* A, const voi
     if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, 1, &mA)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, tail_box, 1, &mAt)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(Wg, s.d_in, s.N, gate_box, 1, &mG)) != METEORA_OK) return rc;
-    if ((rc = get_tensor_map(x, s.d_in, s.T, sp.BN, sp.kc, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, sp.pair ? sp.BN / 2 : sp.BN, sp.kc, &mX)) != METEORA_OK) return rc;
     if ((rc = get_tensor_map(x, s.d_in, s.T, sp.BN, 1, &mX1)) != METEORA_OK) return rc;
     StreamParams d = {};
     d.T = s.T;
@@ -1771,10 +1781,12 @@ int launch_decode_stream(const void* x, const void* W0, const void* A, const voi
     if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
     if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-            return METEORA_ERR_CUDA;
         // the whole shared-memory / L1 array as shared memory, so that two CTAs of 113 KB fit
-        if (cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributePreferredSharedMemoryCarveout,
+        if (cudaFuncSetAttribute(k_decode_stream<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_decode_stream<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_decode_stream<false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess ||
+            cudaFuncSetAttribute(k_decode_stream<true>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared) != cudaSuccess)
             return METEORA_ERR_CUDA;
         attr_set[dev] = true;
@@ -1784,18 +1796,30 @@ int launch_decode_stream(const void* x, const void* W0, const void* A, const voi
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = sp.smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     const bool want_pdl = tuning().pdl_decode != 0;
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    int na = 0;
+    if (sp.pair) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 2;
+        attr[na].val.clusterDim.y = 1;
+        attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (want_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = want_pdl ? 1 : 0;
+    cfg.numAttrs = na;
     d.pdl = want_pdl ? 1 : 0;
 #ifdef METEORA_TRACE
     static int trace_calls = 0;
     d.trace_call = trace_calls++;
 #endif
-    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_stream, mW, mA, mAt, mG, mX, mX1, d));
+    if (sp.pair) return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_stream<true>, mW, mA, mAt, mG, mX, mX1, d));
+    return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_stream<false>, mW, mA, mAt, mG, mX, mX1, d));
 }
 
 // Human-readable launch plan of meteora_linear_forward for this shape (for logs and benchmark records).
@@ -1805,9 +1829,9 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     if (sp.ok)
         return snprintf(buf, n,
                         "path=stream_decode launches=1 main_ctas=%d row_tiles=%d ctas_per_tile=%d aux_ctas=%d aux_slices=%d "
-                        "tile_tokens=%d stages=%d kc=%d smem=%zu ctas_per_sm=%d l2_prefetch_stages=%d",
+                        "tile_tokens=%d stages=%d kc=%d smem=%zu ctas_per_sm=%d pairs=%d l2_prefetch_stages=%d",
                         sp.n_main, sp.row_tiles, sp.S, sp.n_aux, sp.aux_slices, sp.BN, sp.stages, sp.kc, sp.smem,
-                        sp.ctas_per_sm, sp.pf_main);
+                        sp.ctas_per_sm, sp.pair, sp.pf_main);
     const FusedPlan fp = make_fused_plan(s);
     if (fp.ok)
         return snprintf(buf, n,

@@ -471,15 +471,16 @@ def test_streamed_decode_kernel_adapter_counts(N, k, T, r):
 
 # Its planner's choices forced the other way: a shallow ring, two k-steps per stage, no L2 prefetch, a small prefetch
 # cap, one CTA per SM with a deep ring, few and many aux CTAs, no programmatic dependent launch.  None of them may
-# change the result beyond the order of the fp32 sums of the stacked shrink's slices.
+# change the result beyond the order of the fp32 sums of the stacked shrink's slices.  (pair_decode = 1 runs the 70
+# tokens on pairs of CTAs with a two-CTA MMA, own_local = 0 sends a CTA's own row slice through scratch too.)
 @pytest.mark.parametrize("knob,value", [("stages", 2), ("kc", 2), ("pf", -1), ("pf", 1), ("stream", 2), ("aux_ctas", 4),
-                                        ("aux_ctas", 40), ("pdl_decode", 0)])
+                                        ("aux_ctas", 40), ("pdl_decode", 0), ("pair_decode", 1), ("own_local", 0)])
 def test_streamed_decode_kernel_planner_choices(knob, value):
     w = workloads.make_workload("stream_knobs", T=70, d_in=2048, d_out=640, dtype="bf16", x_kind="normal", seed=2234,
                                 b_std=0.3)
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
     y0, i0, _ = run_forward(w)
-    default = {"stream": 1, "pdl_decode": 1}.get(knob, 0)
+    default = {"stream": 1, "pdl_decode": 1, "own_local": 1}.get(knob, 0)
     mb.meteora_set_tuning(knob, value)
     try:
         assert "stream_decode" in mb.meteora_describe_plan(shape)
@@ -490,6 +491,26 @@ def test_streamed_decode_kernel_planner_choices(knob, value):
     same = assert_same_outside_the_band(w, i0, i1)
     assert same.mean() > 0.97
     assert rel_l2(y1[same], y0[same]) < 4e-3
+
+
+@pytest.mark.parametrize("d_in,d_out,T,per_tile", [(1024, 640, 20, 0), (1024, 896, 33, 2), (2048, 4224, 48, 0)])
+def test_streamed_decode_kernel_on_pairs_at_small_batches(d_in, d_out, T, per_tile):
+    # pairs of CTAs (two-CTA MMA, each CTA half of the token tile; a knob, off by default), forced here for token
+    # tiles of 32 and 64, an odd number of row tiles (7: the last pair's second CTA has no rows) and 33 tiles
+    w = workloads.make_workload("stream_pairs", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="rms",
+                                seed=250 + T + d_out, b_std=0.3)
+    mb.meteora_set_tuning("pair_decode", 2)
+    mb.meteora_set_tuning("splits", per_tile)
+    try:
+        shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+        assert "pairs=1" in mb.meteora_describe_plan(shape)
+        check_forward(w, y_tol=1e-2)
+        y1, i1, _ = run_forward(w)
+        y2, i2, _ = run_forward(w)
+        np.testing.assert_array_equal(y1, y2)
+    finally:
+        mb.meteora_set_tuning("pair_decode", 0)
+        mb.meteora_set_tuning("splits", 0)
 
 
 def test_streamed_decode_calls_share_one_workspace_back_to_back():
