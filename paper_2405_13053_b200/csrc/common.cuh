@@ -125,6 +125,7 @@ struct Tuning {
     int stream = 1;          // streamed decode kernel (two launches resident at a time): 0 never, 1 where the planner takes it,
                              // 2 the same kernel with one CTA per SM and a deep ring, 3 wherever the shape allows
     int pair_decode = 0;     // streamed decode kernel, main CTAs in pairs (two-CTA MMA): 0 never (measured slower), 1 from 64 tokens up, 2 from 17
+    int bulk_deliver = 0;    // streamed decode kernel: partial tiles leave through shared memory and bulk copies (1: where the row slices are equal; default plain stores)
     int own_local = 1;       // streamed decode kernel: a CTA keeps its own row slice of its accumulator in shared memory
     int pf = 0;              // its L2 prefetch of the weights beyond the ring: 0 planner's cap, -1 none, n > 0 cap in MB
     int fused = 1;           // 0: never use the single-launch decode kernel

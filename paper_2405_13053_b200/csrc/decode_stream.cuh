@@ -50,6 +50,7 @@ struct StreamParams {
     int32_t* ctr;              // [0] aux partials in, [1] routing published, [2] CTAs counted out
     int32_t* tile_ctr;         // [row tiles] partials delivered
     int32_t* status;
+    int bulk_deliver;          // the other CTAs' row slices leave through shared memory and bulk copies instead of plain stores
     int own_local;             // the CTA's own row slice of its accumulator stays in shared memory (else through scratch like the others)
     int pdl;
     int trace_call;
@@ -68,6 +69,65 @@ __device__ __forceinline__ void bulk_load_block(uint32_t smem_dst, const void* g
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
                  "l"(gsrc), "r"(bytes), "r"(bar)
                  : "memory");
+}
+
+// TMEM -> registers, 16 columns of this warp's 32 lanes, WITHOUT waiting: several of these go out back to back and
+// one tmem_ld_wait() covers them all (a load and its wait take about half a microsecond; four in a row, each
+// waited for, cost the epilogue 2 us at 128 tokens).
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// The accumulator columns [c_begin, c_end) of this warp's 32 rows (whole chunks of 16 columns, at most 64 per round) to
+// column * pitch floats behind a shared-memory address or a global pointer; `valid` false stores zeros (a wait gave
+// up).  No store is predicated: columns beyond the last token hold zeros (the token tile's rows past T are zero-filled)
+// and every destination is sized for the padded token count.  (Bounds checked per store, or stores through a
+// pointer that may be shared or global, made this loop five times slower: 2.4 us for 64 columns.)
+__device__ __forceinline__ void tmem_rows_out(uint32_t taddr, int c_begin, int c_end, bool valid, float* dst,
+                                              uint32_t dst_shared, bool to_shared, int pitch,
+                                              unsigned long long* t_ld = nullptr) {
+    for (int c0 = c_begin; c0 < c_end; c0 += 64) {
+        uint32_t r[4][16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (valid && c0 + 16 * q < c_end) {                          // warp-uniform
+                tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * q), r[q]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) r[q][i] = 0u;
+            }
+        }
+        tmem_ld_wait();
+        if (t_ld) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(*t_ld));
+        const int nchunks = min(4, (c_end - c0) / 16);
+        if (to_shared) {
+            const uint32_t a0 = dst_shared + (uint32_t)(c0 * pitch * 4);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q < nchunks) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(a0 + (uint32_t)((16 * q + i) * pitch * 4)), "r"(r[q][i])
+                                     : "memory");
+                }
+            }
+        } else {
+            float* g0 = dst + (size_t)c0 * pitch;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q < nchunks) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) g0[(size_t)(16 * q + i) * pitch] = __uint_as_float(r[q][i]);
+                }
+            }
+        }
+    }
 }
 
 // 3-D tile load of a CTA pair: the completion bytes go to a barrier that may live in the pair's other CTA.
@@ -305,17 +365,10 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             // the accumulator tile as it is, [token][128 rows] fp32, through the idle ring and one bulk copy
             const int trow = quad * 32 + lane;
             float* stage = reinterpret_cast<float*>(ring_ptr);
-            for (int c = c_begin; c < c_end; c += 16) {
-                float v[16];
-                if (acc_ok && niter > 0) {
-                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c, v);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                }
-#pragma unroll
-                for (int i = 0; i < 16; ++i) stage[(c + i) * kBM + trow] = v[i];
-            }
+            // (all BN columns are written: the bulk copy below moves T of them, the rest are zero rows of the x tile)
+            tmem_rows_out(tmem_base + ((uint32_t)(quad * 32) << 16), c_begin, c_end, acc_ok && niter > 0, nullptr,
+                          ring + (uint32_t)trow * 4u, true, kBM);
+            (void)stage;
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         __syncwarp();
@@ -382,7 +435,8 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
         uint4* slab = reinterpret_cast<uint4*>(slab_ptr);
         // Landing area in the idle ring: block c = row slice j of partial c ([token][4 nq rows] fp32; block j is
         // written by this CTA's own threads), then one block for the LoRA expand of the slice, then the routing.
-        const uint32_t blk_bytes = ((uint32_t)(ntok * 4 * nq * 4) + 127u) & ~127u;
+        // (blocks hold the padded token count BN: the accumulator leaves in whole chunks of 16 token columns)
+        const uint32_t blk_bytes = (uint32_t)(d.BN * 4 * nq * 4);
         const uint32_t delta_off = S * blk_bytes;
         const uint32_t idx_bytes = ((uint32_t)(ntok * d.k * 4) + 15u) & ~15u;
         const uint32_t uw_bytes = (uint32_t)(ntok * d.k * d.r * 4);
@@ -489,12 +543,12 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                 if (ok && S > 1 && live) ok = wait_counter_slow(d.tile_ctr + tile, S, 100);
                 if (!ok) stream_flag_error(d, 4, 900);
                 STREAM_STAMP(6);
-                const uint32_t one = (uint32_t)(ntok * 4 * nq * 4);
+                const uint32_t one = blk_bytes;
                 mbar_expect_tx(bar_land, live ? (uint32_t)(d.own_local ? S - 1 : S) * one : 0u);
                 for (int c = 0; c < S && live; ++c)
                     if (c != j || !d.own_local)
                         bulk_load_block(ring + c * blk_bytes,
-                                        d.part_g + (size_t)(tile * S + c) * ((size_t)d.BN * kBM) + (size_t)ntok * 4 * q0, one,
+                                        d.part_g + (size_t)(tile * S + c) * ((size_t)d.BN * kBM) + (size_t)d.BN * 4 * q0, one,
                                         bar_land);
                 if (atomicAdd_block(s_done, 1) == 1) stream_count_out(d);
                 mbar_wait(bar_land, 0);     // own copies have landed before the CTA may leave
@@ -517,10 +571,12 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                     snq = b;
                 }
             }
-            float* part = sj == j && d.own_local
-                              ? land + (size_t)j * (blk_bytes / 4) + (row_in_tile - 4 * sq0)
-                              : d.part_g + (size_t)slot_id * ((size_t)d.BN * kBM) + (size_t)ntok * 4 * sq0 +
-                                    (row_in_tile - 4 * sq0);
+            // (bulk_deliver: the slices for the other CTAs are staged where their counterparts will land later, block c of
+            // the landing area, and leave as one bulk copy each; the host takes this only where all slices have equal size)
+            const bool part_shared = (sj == j && d.own_local) || d.bulk_deliver;
+            const uint32_t part_s = ring + (uint32_t)sj * blk_bytes + (uint32_t)(row_in_tile - 4 * sq0) * 4u;
+            float* part = d.part_g + (size_t)slot_id * ((size_t)d.BN * kBM) + (size_t)d.BN * 4 * sq0 + (row_in_tile - 4 * sq0);
+            (void)land;
             if (d.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
             bool acc_ok = mbar_wait(bar_acc, 0);
             if (!acc_ok && lane == 0) stream_flag_error(d, 3, 300);
@@ -529,22 +585,37 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             if (etid == 0) STREAM_STAMP(4);
             {
                 const int pitch = 4 * snq;
-                for (int c = c_begin; c < c_end; c += 16) {
-                    float v[16];
-                    if (acc_ok && n_it > 0) {
-                        tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c, v);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = 0.f;
-                    }
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (c + i < ntok && live) part[(size_t)(c + i) * pitch] = v[i];
-                }
+#ifdef METEORA_TRACE
+                unsigned long long t_ld = 0;
+                if (live)
+                    tmem_rows_out(tmem_base + ((uint32_t)(quad * 32) << 16), c_begin, c_end, acc_ok && n_it > 0, part, part_s,
+                                  part_shared, pitch, &t_ld);
+                if (etid == 0 && blockIdx.x < kTraceCtas)
+                    g_fused_trace[((d.trace_call % kTraceCalls) * kTraceCtas + blockIdx.x) * kTraceSlots + 14] = t_ld;
+#else
+                if (live)
+                    tmem_rows_out(tmem_base + ((uint32_t)(quad * 32) << 16), c_begin, c_end, acc_ok && n_it > 0, part, part_s,
+                                  part_shared, pitch);
+#endif
                 if (etid == 0) STREAM_STAMP(11);
+                if (d.bulk_deliver) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> bulk copy reads
                 epi_barrier();                                         // also orders the own slice for the threads below
                 if (etid == 0) {
                     STREAM_STAMP(12);
+                    if (d.bulk_deliver && S > 1 && live) {
+                        const uint32_t one = blk_bytes;
+                        for (int c = 0; c < S; ++c)
+                            if (c != j) {
+                                int a, b;
+                                row_slice(c, S, a, b);
+                                float* dst = d.part_g + (size_t)slot_id * ((size_t)d.BN * kBM) + (size_t)d.BN * 4 * a;
+                                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+                                             "r"(ring + c * blk_bytes), "r"(one)
+                                             : "memory");
+                            }
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                    }
                     if (S > 1 && live) {
                         __threadfence();
                         STREAM_STAMP(13);
