@@ -53,6 +53,8 @@ def parse_args():
                     help="the timed region of --steps steps is run this many times; the line reports the median region "
                          "(value, ms_per_step) and the spread")
     ap.add_argument("--no-prefill-line", action="store_true", help="skip the prefill_roofline measurement")
+    ap.add_argument("--prefill-only", action="store_true",
+                    help="run only the prefill_roofline measurement (config 2 gate/up, T = 2048) and print it")
     ap.add_argument("--modules", type=int, default=16, help="independent MeteoRA modules visited per step")
     ap.add_argument("--launch", choices=["graph", "stream"], default="graph")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target length of the cpu_baseline sample")
@@ -1165,7 +1167,18 @@ def main():
     args = parse_args()
     if args.impl != "reference":
         apply_knobs(args)
-    if args.variants:
+    if args.prefill_only:
+        import torch
+
+        from paper_2405_13053_b200 import binding as mb
+        from paper_2405_13053_b200 import build as lib_build
+
+        lib_build.build_library()
+        torch.cuda.set_device(0)
+        tc_peak, tc_kind = measured_tensor_peak()
+        print(json.dumps({"prefill_roofline": prefill_line(mb, mb.load_library(), tc_peak, tc_kind, measured_peaks()[0])}),
+              flush=True)
+    elif args.variants:
         run_variants()
     elif args.layer:
         run_layer()

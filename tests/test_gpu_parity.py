@@ -37,6 +37,9 @@ GATE_CASES = [
     dict(T=17, d_in=256, d_out=8, N=100, k=4, dtype="bf16"),     # the last lanes' fourth logit is out of range
     dict(T=1, d_in=4096, d_out=8, N=28, k=2, dtype="bf16"),
     dict(T=300, d_in=512, d_out=8, N=28, k=2, dtype="bf16", temperature=15.0),
+    dict(T=128, d_in=4096, d_out=8, N=28, k=2, dtype="bf16"),     # long rows: 8 warps share a token's contraction axis
+    dict(T=1101, d_in=1024, d_out=8, N=28, k=2, dtype="bf16"),    # ... and from 1024 tokens up 4 tokens per block, ragged
+    dict(T=70, d_in=1536, d_out=8, N=128, k=8, dtype="f32"),      # ... fp32, the most adapters
 ]
 
 
