@@ -458,6 +458,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "stream")) t.stream = value;
     else if (!strcmp(name, "pf")) t.pf = value;
     else if (!strcmp(name, "own_local")) t.own_local = value;
+    else if (!strcmp(name, "group_pairs")) t.group_pairs = value;
     else if (!strcmp(name, "bulk_deliver")) t.bulk_deliver = value;
     else if (!strcmp(name, "pair_decode")) t.pair_decode = value;
     else if (!strcmp(name, "wait_limit_us")) return set_wait_limit_us(value);

@@ -124,6 +124,7 @@ struct Tuning {
     int pdl = 1;
     int stream = 1;          // streamed decode kernel (two launches resident at a time): 0 never, 1 where the planner takes it,
                              // 2 the same kernel with one CTA per SM and a deep ring, 3 wherever the shape allows
+    int group_pairs = 0;     // prefill on pairs of SMs: row pairs per scheduling group (0: planner's choice; a large value = row-major order)
     int pair_decode = 0;     // streamed decode kernel, main CTAs in pairs (two-CTA MMA): 0 never (measured slower), 1 from 64 tokens up, 2 from 17
     int bulk_deliver = 0;    // streamed decode kernel: partial tiles leave through shared memory and bulk copies (1: where the row slices are equal; default plain stores)
     int own_local = 1;       // streamed decode kernel: a CTA keeps its own row slice of its accumulator in shared memory

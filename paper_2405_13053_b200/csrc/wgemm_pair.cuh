@@ -89,6 +89,7 @@ struct PairParams {
     int d_out, N, k, r;           // rank r: a multiple of 8
     int nblk, rb;                 // blocks of 8 expand columns: N * r / 8 in all, rb (even) per round
     int row_tiles;
+    int group_pairs;              // row pairs per scheduling group (see the kernel: which tile a pair of CTAs takes)
     int epi_off, slab_off;        // staging area behind the barriers; the B rows sit at slab_off inside it
     const int32_t* topk_idx;
     const float* uw;
@@ -117,8 +118,20 @@ k_wgemm_pair(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();
     const bool leader = rank == 0;
-    const int tile_m = (blockIdx.x >> 1) * 2 + (int)rank;         // own 128 rows of W0 / y
-    const int tok0 = blockIdx.y * kPairTokens;                    // the pair's 256 tokens
+    // Which tile this pair takes.  Pairs are dispatched in the order of p = blockIdx.y * (gridDim.x / 2) + blockIdx.x / 2;
+    // taken row-major (all row pairs of one token tile, then the next token tile) every token tile streams the whole of
+    // W0 again, and once W0 is about as large as the L2 each pass comes from HBM: 764 MB of DRAM reads per launch at
+    // 4096 -> 14336 with 2048 tokens, 6.5 times W0.  Instead the row pairs are cut into groups of `group_pairs`, and a
+    // group's row pairs run over ALL token tiles before the next group starts: the pairs resident at one time then
+    // share a few row pairs of W0 (read from HBM once, found in L2 by the other token tiles) and all of x (small).
+    const int row_pairs = (int)gridDim.x >> 1, tok_tiles = (int)gridDim.y;
+    const int lin = (int)blockIdx.y * row_pairs + ((int)blockIdx.x >> 1);
+    const int per_group = p.group_pairs * tok_tiles;
+    const int grp = lin / per_group, rem = lin - grp * per_group;
+    const int in_grp = min(p.group_pairs, row_pairs - grp * p.group_pairs);     // the last group may be smaller
+    const int tok_tile = rem / in_grp, row_pair = grp * p.group_pairs + rem - tok_tile * in_grp;
+    const int tile_m = row_pair * 2 + (int)rank;                  // own 128 rows of W0 / y
+    const int tok0 = tok_tile * kPairTokens;                      // the pair's 256 tokens
     const int tokh = tok0 + (int)rank * kPairHalf;                // own half of them
     const int niter = p.ksteps;
 
