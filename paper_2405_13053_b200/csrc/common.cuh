@@ -122,8 +122,8 @@ struct Tuning {
     int simt_expand = 0;   // 1: keep the LoRA expand on CUDA cores even for rank 8
     int force_simt = 0;
     int pdl = 1;
-    int stream = 1;          // streamed decode kernel (two launches resident at a time): 0 never, 1 where the planner takes it,
-                             // 2 the same kernel with one CTA per SM and a deep ring, 3 wherever the shape allows
+    int stream = 1;          // streamed decode kernel: 0 never, 1 the planner's choice of one or two CTAs per SM,
+                             // 2 / 4 always one CTA per SM (deep ring), 3 two per SM wherever they fit
     int group_pairs = 0;     // prefill on pairs of SMs: row pairs per scheduling group (0: planner's choice; a large value = row-major order)
     int pair_decode = 0;     // streamed decode kernel, main CTAs in pairs (two-CTA MMA): 0 never (measured slower), 1 from 64 tokens up, 2 from 17
     int bulk_deliver = 0;    // streamed decode kernel: partial tiles leave through shared memory and bulk copies (1: where the row slices are equal; default plain stores)

@@ -1623,12 +1623,6 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     sp.why = 1;
     if (!tn.fused || !tn.stream || tn.simt_expand) return sp;
     if (!tc_path_supported(s) || s.T > 128 || s.r % 8 != 0 || s.d_in % kBK != 0 || s.d_out <= 0) return sp;
-    // Two CTAs per SM means half the ring each.  Measured per call, this kernel against the cooperative one (one CTA
-    // per SM, twice the ring): 4096 -> 4096 (34 MB of W0) 11.8 / 12.7 / 16.7 us against 13.5 / 14.2 / 17.1 at 1 / 32 / 128
-    // tokens; 5120 -> 5120 (52 MB) 15.1 against 15.7 at one token but 19.3 against 18.0 at 64; 13824 -> 5120 (142 MB)
-    // 39.3 against 35.3 at 64: the longer the stream, the more the deeper ring counts and the less the set-up and the
-    // first tiles loaded under the call ahead.  Taken up to 40 MB of W0 (knob stream = 3: always).
-    if ((size_t)s.d_out * s.d_in * 2 > ((size_t)40 << 20) && tn.stream != 3) return sp;
     const int sms = std::min(sm_count(), 148);                   // the workspace holds partial tiles for 148 CTAs
     const int ksteps = s.d_in / kBK;
     sp.row_tiles = (s.d_out + kBM - 1) / kBM;
@@ -1697,8 +1691,19 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     const size_t ring_need = std::max(std::max(landing, (size_t)sp.BN * kBM * 4), aux_rows);
     const int n_it_max = (nst + S - 1) / S;
     const int nks_aux = (ksteps + sp.aux_slices - 1) / sp.aux_slices;
+    // Two CTAs per SM (the next call's CTAs resident under this call) or one with twice the ring?  Two hide the set-up
+    // and load the first tiles under the call ahead, but the in-order ring stalls on its slowest line and five
+    // stages run at 3.3 - 4 TB/s where eleven reach HBM's rate: the longer the stream, the more the deeper ring counts.
+    // Measured per call, two / one per SM (us): 4096 -> 4096 (34 MB of W0) 12.2 / 13.1 at 1 token, 12.4 / 13.2 at 8,
+    // 14.3 / 13.8 at 64, 16.6 / 16.4 at 128; 5120 -> 5120 (52 MB) 15.3 / 15.9 at 1, 15.4 / 16.1 at 16, 19.1 / 17.1 at 64;
+    // 4096 -> 1024 (8 MB) 10.3 / 10.3 at 1, 12.1 / 11.8 at 64; 4096 -> 14336 (117 MB) 30.3 / 26.7 at 1, 31.2 / 31.5 at 64;
+    // 5120 -> 13824 (142 MB) 36.5 / 31.8 at 1.  So: two per SM for 16 - 56 MB of W0 and up to 32 tokens, else one.
+    // (Knob stream: 2 or 4 always one per SM, 3 always two where they fit.)
+    const size_t w0_bytes = (size_t)s.d_out * s.d_in * 2;
+    const bool want_two = tn.stream == 3 || (tn.stream == 1 && s.T <= 32 && w0_bytes >= ((size_t)16 << 20) &&
+                                             w0_bytes <= ((size_t)56 << 20));
     for (int per_sm = 2; per_sm >= 1; --per_sm) {
-        if (per_sm == 2 && tn.stream == 2) continue;               // knob: one CTA per SM, deep ring
+        if (per_sm == 2 && !want_two) continue;
         const size_t budget = per_sm == 2 ? kTwoPerSmBytes : 226 * 1024;
         const size_t fixed = 1024 + sp.slab_off + slab_bytes;
         if (fixed + ring_need > budget || fixed + 2 * stage_bytes > budget) continue;
