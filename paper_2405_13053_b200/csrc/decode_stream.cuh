@@ -177,22 +177,14 @@ __device__ __forceinline__ void stream_count_out(const StreamParams& d) {
 #define STREAM_STAMP(slot) do { } while (0)
 #endif
 
-// Selection for one token whose partial stacked-shrink rows are in shared memory: sm[(z * tiles + tile) * ntl + tl]
-// is the 128-float row of slice z, tile `tile`, local token tl.  The slices are added in slice order, exactly as
-// select_token_narrow adds them, so both give the same bits.
-__device__ __forceinline__ void select_token_smem(const float* sm, int tl, int ntl, int tiles, int gate_tile, int gate_row0,
-                                                  int zsplits, int t, int N, int r, int k, float inv_tau, int lane,
-                                                  int32_t* topk_idx, float* topk_w, float* uw) {
-    const int zstride = tiles * ntl * kBM;
+// Selection for one token from its summed row of the stacked shrink in shared memory (row[R] for stacked row R of
+// [A_0 .. A_{N-1}], logit n at row[gate_tile * 128 + gate_row0 + n]): top-k, softmax over the picks (Eq. 3), uw.
+__device__ __forceinline__ void select_token_row(const float* row, int gate_tile, int gate_row0, int t, int N, int r, int k,
+                                                 float inv_tau, int lane, int32_t* topk_idx, float* topk_w, float* uw) {
     float v[kSelVals];
 #pragma unroll
-    for (int i = 0; i < kSelVals; ++i) {
-        v[i] = 0.f;
-        if (32 * i < N) {                                   // uniform across the warp
-            const float* src = sm + (gate_tile * ntl + tl) * kBM + gate_row0 + min(lane + 32 * i, N - 1);
-            for (int z = 0; z < zsplits; ++z) v[i] += src[z * zstride];
-        }
-    }
+    for (int i = 0; i < kSelVals; ++i)
+        v[i] = lane + 32 * i < N ? row[gate_tile * kBM + gate_row0 + lane + 32 * i] : 0.f;
     int idx;
     float w;
     warp_topk_softmax(v, N, k, inv_tau, lane, idx, w);
@@ -205,11 +197,7 @@ __device__ __forceinline__ void select_token_smem(const float* sm, int tl, int n
         const int j = c / r, q = c - j * r;
         const int ij = __shfl_sync(0xFFFFFFFFu, idx, j);
         const float wj = __shfl_sync(0xFFFFFFFFu, w, j);
-        const int R = ij * r + q;                           // row of the stacked matrix [A_0 .. A_{N-1}]
-        const float* src = sm + ((R / kBM) * ntl + tl) * kBM + (R % kBM);
-        float u = 0.f;
-        for (int z = 0; z < zsplits; ++z) u += src[z * zstride];
-        if (c0 + lane < k * r) uw[(size_t)t * k * r + c0 + lane] = wj * u;
+        if (c0 + lane < k * r) uw[(size_t)t * k * r + c0 + lane] = wj * row[ij * r + q];
     }
 }
 
@@ -387,25 +375,50 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             // This CTA's share of the tokens: their rows of every partial tile into the idle ring (one bulk copy per
             // tile and slice, a token range is contiguous there), then a warp per token selects from shared memory.
             const int t0 = d.T * aux_id / n_active, t1 = d.T * (aux_id + 1) / n_active, ntl = t1 - t0;
-            if (threadIdx.x == 0 && ntl > 0) {
-                mbar_expect_tx(bar_land, (uint32_t)(n_active * ntl * kBM * 4));
-                for (int q = 0; q < n_active; ++q)
-                    bulk_load_block(ring + (uint32_t)(q * ntl * kBM * 4), d.u_part + ((size_t)q * d.T + t0) * kBM,
-                                    (uint32_t)(ntl * kBM * 4), bar_land);
-            }
-            __syncthreads();                                         // (the staged accumulator tile has left the ring)
+            const uint32_t rows_bytes = (uint32_t)(n_active * ntl * kBM * 4);
+            __syncthreads();                                         // thread 0 has seen all partials; its staged tile has left the ring
             if (ntl > 0) {
+                // one copy per (slice, tile), each issued by a thread of its own (twenty issued by one thread took over a microsecond)
+                if (threadIdx.x == 0) mbar_expect_tx(bar_land, rows_bytes);
+                if ((int)threadIdx.x < n_active)
+                    bulk_load_block(ring + (uint32_t)((int)threadIdx.x * ntl * kBM * 4),
+                                    d.u_part + ((size_t)threadIdx.x * d.T + t0) * kBM, (uint32_t)(ntl * kBM * 4), bar_land);
                 bool ok = mbar_wait(bar_land, 0);
                 if (!ok && lane == 0) stream_flag_error(d, 4, 750);
                 ok = __all_sync(0xFFFFFFFFu, ok);                   // the selection is warp-collective
+                if (threadIdx.x == 0) STREAM_STAMP(6);
+                // All threads add the slices of the CTA's tokens' rows, four columns per item, every slice of an item in
+                // flight together, in slice order (the same sums in the same order as select_token_narrow: same bits); a
+                // warp per token then selects from the summed row.  (One warp doing both for its token took 1.7 us.)
+                const float4* sm4 = reinterpret_cast<const float4*>(ring_ptr);
+                float4* rows4 = reinterpret_cast<float4*>(ring_ptr + rows_bytes);      // [ntl][tiles * 128] floats
+                const int per_tok = d.aux_tiles * 32, zs4 = d.aux_tiles * ntl * 32;
+                for (int it = threadIdx.x; it < ntl * per_tok && ok; it += kThreads) {
+                    const int tl = it / per_tok, rem = it - tl * per_tok, tile = rem >> 5, l4 = rem & 31;
+                    const float4* src = sm4 + (tile * ntl + tl) * 32 + l4;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+                    for (int z = 0; z < d.aux_slices; ++z) {
+                        const float4 v = src[z * zs4];
+                        acc.x += v.x;
+                        acc.y += v.y;
+                        acc.z += v.z;
+                        acc.w += v.w;
+                    }
+                    rows4[it] = acc;
+                }
+                __syncthreads();
                 const int nwarps = kThreads / 32;
                 for (int tl = warp; tl < ntl && ok; tl += nwarps)
-                    select_token_smem(reinterpret_cast<const float*>(ring_ptr), tl, ntl, d.aux_tiles, d.gate_tile, d.gate_row0,
-                                      d.aux_slices, t0 + tl, d.N, d.r, d.k, d.inv_tau, lane, d.topk_idx, d.topk_w, d.uw);
+                    select_token_row(reinterpret_cast<const float*>(rows4 + tl * per_tok), d.gate_tile, d.gate_row0, t0 + tl, d.N,
+                                     d.r, d.k, d.inv_tau, lane, d.topk_idx, d.topk_w, d.uw);
+                if (threadIdx.x == 0) STREAM_STAMP(7);
             }
             __syncthreads();
             if (threadIdx.x == 0) {
+                STREAM_STAMP(8);
                 __threadfence();
+                STREAM_STAMP(9);
                 atomicAdd(d.ctr + 1, 1);
                 STREAM_STAMP(5);
             }

@@ -20,6 +20,7 @@ __device__ __forceinline__ void warp_topk_softmax(float (&v)[kSelVals], int N, i
     for (int i = 0; i < kSelVals; ++i) {
         taken[i] = lane + 32 * i >= N;
         if (!(v[i] > -CUDART_INF_F)) v[i] = -CUDART_INF_F;  // NaN never wins a comparison; treat it as -inf
+        v[i] += 0.f;                                        // -0 becomes +0: equal as floats, and equal as the keys below
     }
     float first = 0.f, sum = 0.f, my_e = 0.f;
     my_idx = 0;
@@ -29,12 +30,13 @@ __device__ __forceinline__ void warp_topk_softmax(float (&v)[kSelVals], int N, i
 #pragma unroll
         for (int i = 0; i < kSelVals; ++i)                   // ascending index: a later equal value does not replace
             if (!taken[i] && (bi == 0x7FFFFFFF || v[i] > bv)) { bv = v[i]; bi = lane + 32 * i; }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
-            const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
+        // Warp-wide arg-max by two reductions instead of a five-step butterfly of shuffles (a third of the latency):
+        // the largest value through an order-preserving integer key, then the lowest index among the lanes that hold it.
+        const uint32_t bits = __float_as_uint(bv);
+        const uint32_t key = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+        const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, key);
+        bi = __reduce_min_sync(0xFFFFFFFFu, key == kmax ? bi : 0x7FFFFFFF);
+        bv = __uint_as_float((kmax & 0x80000000u) ? (kmax & 0x7FFFFFFFu) : ~kmax);
         bi = min(bi, N - 1);
 #pragma unroll
         for (int i = 0; i < kSelVals; ++i)

@@ -1687,7 +1687,8 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     const size_t parts = (size_t)(S + 1) * ((size_t)sp.BN * 4 * nq_max * 4);   // (blocks hold the padded token count)
     const size_t landing = parts + align_up(align_up((size_t)ntok * s.k * 4, 16), 128) + (size_t)ntok * s.k * s.r * 4;
     // an aux CTA stages its accumulator tile there, later its tokens' rows of every partial tile of the stacked shrink
-    const size_t aux_rows = (size_t)sp.n_aux * ((s.T + sp.n_aux - 1) / sp.n_aux) * kBM * 4;
+    // (and the summed rows of those tokens behind them)
+    const size_t aux_rows = (size_t)(sp.n_aux + sp.aux_tiles) * ((s.T + sp.n_aux - 1) / sp.n_aux) * kBM * 4;
     const size_t ring_need = std::max(std::max(landing, (size_t)sp.BN * kBM * 4), aux_rows);
     const int n_it_max = (nst + S - 1) / S;
     const int nks_aux = (ksteps + sp.aux_slices - 1) / sp.aux_slices;
