@@ -39,7 +39,7 @@ NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, nominal
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "36438807b8c24de5", "bytes_per_launch": {"128": 38620416 + 64597}}
+NCU_TRAFFIC = {"kernel_sha": "c181bb98afb407ee", "bytes_per_launch": {"128": 38595925 + 20565, "1": 37555627 + 1451}}
 
 
 def parse_args():
