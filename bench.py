@@ -1024,6 +1024,8 @@ def run_decode_loop():
 
 def run_gate_backward_sweep():
     """meteora_gate_backward (gradient of the gate weights for a forward's routing) at the q_proj shape."""
+    import ctypes
+
     import torch
 
     from paper_2405_13053_b200 import binding as mb
@@ -1031,7 +1033,8 @@ def run_gate_backward_sweep():
     hbm, _ = measured_peaks()
     dt, es = torch.bfloat16, 2
     d_in = d_out = 4096
-    for T in (128, 2048, 8192):
+    lib = mb.load_library()
+    for T in (1, 128, 2048, 8192):
         g = torch.Generator(device="cuda").manual_seed(13)
         x = torch.randn(T, d_in, device="cuda", generator=g).to(dt)
         W0 = (0.02 * torch.randn(d_out, d_in, device="cuda", generator=g)).to(dt)
@@ -1041,25 +1044,50 @@ def run_gate_backward_sweep():
         dy = torch.randn(T, d_out, device="cuda", generator=g).to(dt)
         _, idx, w = mb.meteora_linear_forward(x, W0, A, B, Wg, TOPK, return_routing=True)
         idx, w = idx.clone(), w.clone()
-        for _ in range(3):
-            mb.meteora_gate_backward(x, A, B, dy, idx, w)
-        torch.cuda.synchronize()
-        iters = 20
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(iters):
-            mb.meteora_gate_backward(x, A, B, dy, idx, w)
-        e1.record()
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) * 1e3 / iters
+        Bt = mb.meteora_transpose_adapters_b(B)
+        shape = mb.make_shape(T, d_in, d_out, N_ADAPTERS, RANK, TOPK, dt)
+        ws = torch.zeros(lib.meteora_gate_backward_workspace_bytes(ctypes.byref(shape)), dtype=torch.uint8, device="cuda")
+
+        def timed(**kw):
+            """Per call from a CUDA graph of 8 calls (stream-ordered on one workspace), median of 5 regions."""
+            def eight():
+                for _ in range(8):
+                    mb.meteora_gate_backward(x, A, B, dy, idx, w, workspace=ws, **kw)
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                eight()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                eight()
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            out = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(5):
+                    graph.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                out.append(e0.elapsed_time(e1) * 1e3 / 40)
+            return sorted(out)[2]
+
+        us_b, us = timed(), timed(Bt=Bt)
         touched = int(torch.unique(idx).numel())
         # x is read for the shrink and again, once per pick, for the reduction over tokens; dy once; dWg written in fp32
         nbytes = ((1 + TOPK) * T * d_in + T * d_out + touched * RANK * (d_in + d_out)) * es + N_ADAPTERS * d_in * 4
-        print(json.dumps({"op": "meteora_gate_backward", "shape": "4096->4096", "T": T, "us_per_call": round(us, 2),
+        print(json.dumps({"op": "meteora_gate_backward_bt", "shape": "4096->4096", "T": T, "us_per_call": round(us, 2),
+                          "us_per_call_with_transposition": round(us_b, 2),
                           "tokens_per_s": round(T / us * 1e6), "bound": "hbm",
                           "roofline_us": round(nbytes / hbm / 1e3, 2),
                           "frac_of_roofline": round(nbytes / hbm / 1e3 / us, 3),
-                          "note": "bucketing, transpose of B, two stacked shrinks on the tensor cores, dlogit, reduction over tokens, copy; stream timing through the Python binding"}),
+                          "note": "B transposed beforehand (meteora_transpose_adapters_b); up to 256 tokens both stacked "
+                                  "shrinks as one launch and no bucketing, up to 1024 no bucketing; graph replay of 8 "
+                                  "stream-ordered calls"}),
               flush=True)
 
 
@@ -1084,14 +1112,18 @@ def run_variants():
     base = {"N": 28, "r": 8, "k": 2, "tau": 1.0}
     points = [dict(base)]
     points += [dict(base, k=k) for k in (1, 4)]
-    points += [dict(base, r=r) for r in (4, 16, 32, 64)]
+    points += [dict(base, r=4, pad="every call"), dict(base, r=4, pad="once")]
+    points += [dict(base, r=r) for r in (16, 32, 64)]
     points += [dict(base, N=N) for N in (8, 64, 128)]
     points += [dict(base, tau=20.0)]
     for T in (32, 2048):
         for pt in points:
             N, r, k, tau = pt["N"], pt["r"], pt["k"], pt["tau"]
             R = 8 if T <= 256 else 1
-            shape = mb.make_shape(T, d_in, d_out, N, r, k, dt, tau)
+            # a rank that is no multiple of 8: the forward pads the adapters on every call, or the caller padded
+            # them once (meteora_pad_adapters) and passes the padded rank
+            r_call = (r + 7) // 8 * 8 if pt.get("pad") == "once" else r
+            shape = mb.make_shape(T, d_in, d_out, N, r_call, k, dt, tau)
             g = torch.Generator(device="cuda").manual_seed(3)
             mods = []
             ws_shared = mb.alloc_workspace(shape)
@@ -1103,6 +1135,8 @@ def run_variants():
                              "B": (0.01 * torch.randn(N, d_out, r, device="cuda", generator=g)).to(dt),
                              "Wg": (torch.randn(N, d_in, device="cuda", generator=g) / d_in ** 0.5).to(dt),
                              "y": torch.empty(T, d_out, device="cuda", dtype=dt), "ws": ws_shared})
+                if pt.get("pad") == "once":
+                    mods[-1]["A"], mods[-1]["B"] = mb.meteora_pad_adapters(mods[-1]["A"], mods[-1]["B"])
 
             def step():
                 for m in mods:

@@ -195,6 +195,34 @@ int meteora_gate_backward(const void* x, const void* A, const void* B, const voi
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Zero-padding of the adapters' rank to the next multiple of 8, made ONCE instead of by every forward: a bf16 layer
+ * whose rank is no multiple of 8 (rank 4, say) runs on the tensor-core paths with A and B padded, and
+ * meteora_linear_forward pads them into its workspace on every call.  The adapters are fixed (Sec. 3.2), so a
+ * caller pads them once: A_pad[N, r8, d_in] and B_pad[N, d_out, r8] (bf16, device memory owned by the caller, 16-byte
+ * aligned, *a_bytes and *b_bytes from meteora_pad_adapters_bytes, which returns r8 = the padded rank, or 0 where
+ * the shape needs no padding or is invalid), then calls the forward with shape->r = r8 and the padded arrays: the
+ * added rank entries are zero in A (rows) and in B (columns), so y, the routing and every sum are bit-identical.
+ * Asynchronous on `stream`; reads N, r, d_in, d_out and dtype of the shape.
+ */
+int meteora_pad_adapters_bytes(const meteora_shape_t* shape, size_t* a_bytes, size_t* b_bytes);
+int meteora_pad_adapters(const void* A, const void* B, const meteora_shape_t* shape, void* A_pad, void* B_pad,
+                         void* stream);
+
+/*
+ * The same gradient with the adapters' B matrices transposed beforehand.  The adapters are fixed while the gates
+ * train (Sec. 3.2), so Bt[n, p, o] = B[n, o, p] (shape->dtype, [N, r, d_out], device memory of
+ * meteora_adapters_bt_bytes(shape) bytes, 16-byte aligned, owned by the caller) is made once per module with
+ * meteora_transpose_adapters_b (asynchronous on `stream`; only N, d_out, r and dtype of the shape are read) and
+ * every step then calls meteora_gate_backward_bt, which is meteora_gate_backward without its transposition of B
+ * (same arguments, results bit-identical to it, same workspace size).
+ */
+size_t meteora_adapters_bt_bytes(const meteora_shape_t* shape);
+int meteora_transpose_adapters_b(const void* B, const meteora_shape_t* shape, void* Bt, void* stream);
+int meteora_gate_backward_bt(const void* x, const void* A, const void* Bt, const void* dy, const int32_t* topk_idx,
+                             const float* topk_w, const meteora_shape_t* shape, float* dlogit, float* dWg,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same as meteora_linear_forward with the activations in HOST memory: x_host[T,d_in] is copied to
  * the device, the layer runs, y_host[T,d_out] is copied back, all on `stream` (pinned host memory
  * makes the copies asynchronous).  Weights and workspace stay device pointers.  The call does not

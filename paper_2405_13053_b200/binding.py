@@ -25,7 +25,8 @@ STATUS = {0: "METEORA_OK", -1: "METEORA_ERR_INVALID_ARG", -2: "METEORA_ERR_UNSUP
 EXPORTS = ["meteora_gate_topk", "meteora_route", "meteora_lora_delta", "meteora_lora_delta_static",
            "meteora_linear_forward", "meteora_linear_forward_group", "meteora_group_workspace_bytes",
            "meteora_group_workspace_routing", "meteora_group_plan", "meteora_gate_backward",
-           "meteora_gate_backward_workspace_bytes",
+           "meteora_gate_backward_workspace_bytes", "meteora_gate_backward_bt", "meteora_transpose_adapters_b",
+           "meteora_adapters_bt_bytes", "meteora_pad_adapters", "meteora_pad_adapters_bytes",
            "meteora_linear_forward_host", "meteora_workspace_bytes", "meteora_workspace_routing",
            "meteora_workspace_init", "meteora_workspace_status", "meteora_profile_begin", "meteora_profile_end",
            "meteora_describe_plan", "meteora_set_tuning", "meteora_status_string"]
@@ -66,6 +67,12 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_linear_forward_group.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
                                                  ctypes.POINTER(vp), ip, ci, shp, ctypes.POINTER(vp), vp, sz, vp]
     lib.meteora_gate_backward.argtypes = [vp, vp, vp, vp, vp, vp, shp, vp, vp, vp, sz, vp]
+    lib.meteora_gate_backward_bt.argtypes = [vp, vp, vp, vp, vp, vp, shp, vp, vp, vp, sz, vp]
+    lib.meteora_transpose_adapters_b.argtypes = [vp, shp, vp, vp]
+    lib.meteora_pad_adapters_bytes.argtypes = [shp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    lib.meteora_pad_adapters.argtypes = [vp, vp, shp, vp, vp, vp]
+    lib.meteora_adapters_bt_bytes.argtypes = [shp]
+    lib.meteora_adapters_bt_bytes.restype = sz
     lib.meteora_gate_backward_workspace_bytes.argtypes = [shp]
     lib.meteora_gate_backward_workspace_bytes.restype = sz
     lib.meteora_group_plan.argtypes = [shp, ip, ci]
@@ -85,7 +92,8 @@ def load_library() -> ctypes.CDLL:
     lib.meteora_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
         if name not in ("meteora_workspace_bytes", "meteora_group_workspace_bytes",
-                        "meteora_gate_backward_workspace_bytes", "meteora_status_string"):
+                        "meteora_gate_backward_workspace_bytes", "meteora_gate_backward_bt", "meteora_transpose_adapters_b",
+           "meteora_adapters_bt_bytes", "meteora_pad_adapters", "meteora_pad_adapters_bytes", "meteora_status_string"):
             getattr(lib, name).restype = ci
     _lib = lib
     return lib
@@ -236,26 +244,59 @@ def meteora_linear_forward(x, W0, A, B, Wg, k: int, temperature: float = 1.0,
     return y, idx, w
 
 
-def meteora_gate_backward(x, A, B, dy, topk_idx, topk_w, temperature: float = 1.0):
-    """dWg[N,d_in] (fp32) and dlogit[T,k] (fp32): gradient of the gate through Eq. 3 and Eq. 2 for the routing given."""
+def meteora_pad_adapters(A, B):
+    """(A_pad[N,r8,d_in], B_pad[N,d_out,r8]) with the rank zero-padded to the next multiple of 8, made once for a bf16
+    layer whose rank is none: a forward on the padded arrays gives the same bits without padding on every call.
+    Returns (A, B) themselves where the library would not pad."""
+    lib = load_library()
+    N, r, d_in = A.shape
+    d_out = B.shape[1]
+    shape = make_shape(0, d_in, d_out, N, r, 1, A.dtype)
+    a_bytes, b_bytes = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    r8 = lib.meteora_pad_adapters_bytes(ctypes.byref(shape), ctypes.byref(a_bytes), ctypes.byref(b_bytes))
+    if r8 == 0:
+        return A, B
+    A_pad = torch.empty((N, r8, d_in), dtype=A.dtype, device=A.device)
+    B_pad = torch.empty((N, d_out, r8), dtype=A.dtype, device=A.device)
+    assert A_pad.numel() * 2 == a_bytes.value and B_pad.numel() * 2 == b_bytes.value
+    _check(lib.meteora_pad_adapters(_dev(A, (N, r, d_in), A.dtype, "A"), _dev(B, (N, d_out, r), A.dtype, "B"),
+                                    ctypes.byref(shape), A_pad.data_ptr(), B_pad.data_ptr(), _stream()),
+           "meteora_pad_adapters")
+    return A_pad, B_pad
+
+
+def meteora_transpose_adapters_b(B):
+    """Bt[N,r,d_out] with Bt[n,p,o] = B[n,o,p]: made once per module for meteora_gate_backward(..., Bt=...)."""
+    lib = load_library()
+    N, d_out, r = B.shape
+    shape = make_shape(0, 1, d_out, N, r, 1, B.dtype)
+    Bt = torch.empty((N, r, d_out), dtype=B.dtype, device=B.device)
+    _check(lib.meteora_transpose_adapters_b(_dev(B, (N, d_out, r), B.dtype, "B"), ctypes.byref(shape), Bt.data_ptr(),
+                                            _stream()), "meteora_transpose_adapters_b")
+    return Bt
+
+
+def meteora_gate_backward(x, A, B, dy, topk_idx, topk_w, temperature: float = 1.0, Bt=None, workspace=None):
+    """dWg[N,d_in] (fp32) and dlogit[T,k] (fp32): gradient of the gate through Eq. 3 and Eq. 2 for the routing given.
+    With Bt (meteora_transpose_adapters_b(B)) the call skips its own transposition of B."""
     lib = load_library()
     T, d_in = x.shape
     N, r, _ = A.shape
-    d_out = B.shape[1]
+    d_out = B.shape[1] if Bt is None else Bt.shape[2]
     k = topk_idx.shape[1]
     shape = make_shape(T, d_in, d_out, N, r, k, x.dtype, temperature)
     n = lib.meteora_gate_backward_workspace_bytes(ctypes.byref(shape))
     if n == 0:
         raise MeteoraError(-1, "meteora_gate_backward_workspace_bytes")
-    ws = torch.empty(n, dtype=torch.uint8, device=x.device)
+    ws = torch.empty(n, dtype=torch.uint8, device=x.device) if workspace is None else workspace
     dWg = torch.empty((N, d_in), dtype=torch.float32, device=x.device)
     dlogit = torch.empty((T, k), dtype=torch.float32, device=x.device)
-    _check(lib.meteora_gate_backward(_dev(x, (T, d_in), x.dtype, "x"), _dev(A, (N, r, d_in), x.dtype, "A"),
-                                     _dev(B, (N, d_out, r), x.dtype, "B"), _dev(dy, (T, d_out), x.dtype, "dy"),
-                                     _dev(topk_idx, (T, k), torch.int32, "topk_idx"),
-                                     _dev(topk_w, (T, k), torch.float32, "topk_w"), ctypes.byref(shape),
-                                     dlogit.data_ptr(), dWg.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
-           "meteora_gate_backward")
+    fn = lib.meteora_gate_backward if Bt is None else lib.meteora_gate_backward_bt
+    b_arg = _dev(B, (N, d_out, r), x.dtype, "B") if Bt is None else _dev(Bt, (N, r, d_out), x.dtype, "Bt")
+    _check(fn(_dev(x, (T, d_in), x.dtype, "x"), _dev(A, (N, r, d_in), x.dtype, "A"), b_arg,
+              _dev(dy, (T, d_out), x.dtype, "dy"), _dev(topk_idx, (T, k), torch.int32, "topk_idx"),
+              _dev(topk_w, (T, k), torch.float32, "topk_w"), ctypes.byref(shape), dlogit.data_ptr(), dWg.data_ptr(),
+              ws.data_ptr(), ws.numel(), _stream()), "meteora_gate_backward")
     return dWg, dlogit
 
 

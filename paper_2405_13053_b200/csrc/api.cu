@@ -303,14 +303,16 @@ size_t meteora_gate_backward_workspace_bytes(const meteora_shape_t* shape) {
            align_up((size_t)shape->N * shape->d_out * r * elem_size(shape->dtype), 256);
 }
 
-int meteora_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
-                          const float* topk_w, const meteora_shape_t* shape, float* dlogit, float* dWg,
-                          void* workspace, size_t workspace_bytes, void* stream) {
+// B != nullptr: transposed into the workspace first; else Bt_ready holds the transposed adapters.
+static int gate_backward_impl(const void* x, const void* A, const void* B, const void* Bt_ready, const void* dy,
+                              const int32_t* topk_idx, const float* topk_w, const meteora_shape_t* shape,
+                              float* dlogit, float* dWg, void* workspace, size_t workspace_bytes, void* stream) {
     int rc = check_shape(shape, true, true);
     if (rc != METEORA_OK) return rc;
     if (!dWg || !workspace) return METEORA_ERR_INVALID_ARG;
-    if (shape->T > 0 && (!x || !A || !B || !dy || !topk_idx || !topk_w)) return METEORA_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(A) || !aligned16(B) || !aligned16(dy) || !aligned16(workspace))
+    const void* b_any = B ? B : Bt_ready;
+    if (shape->T > 0 && (!x || !A || !b_any || !dy || !topk_idx || !topk_w)) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(A) || !aligned16(b_any) || !aligned16(dy) || !aligned16(workspace))
         return METEORA_ERR_MISALIGNED;
     if (workspace_bytes < meteora_gate_backward_workspace_bytes(shape)) return METEORA_ERR_WORKSPACE_TOO_SMALL;
     const size_t S = (size_t)shape->T * shape->k, r = (size_t)shape->r;
@@ -323,20 +325,67 @@ int meteora_gate_backward(const void* x, const void* A, const void* B, const voi
     float* dl = (float*)take(S * 4);
     int32_t* perm = (int32_t*)take(S * 4);
     const size_t shrink_bytes = gate_backward_shrink_floats(*shape) * 4;
-    float* u = (float*)take(shrink_bytes);
-    float* z = (float*)take(shrink_bytes);
+    float* u = (float*)take(shrink_bytes);               // u and z are contiguous: the one-launch pair of stacked
+    float* z = (float*)take(shrink_bytes);               // shrinks writes both into the space of the two
     int32_t* counts = (int32_t*)take(((size_t)shape->N + 1) * 4);
     int32_t* offsets = (int32_t*)take(((size_t)shape->N + 1) * 4);
     void* Bt = take((size_t)shape->N * shape->d_out * r * elem_size(shape->dtype));
     cudaStream_t st = (cudaStream_t)stream;
     // the header's first words take the error flags of the tensor-core kernels
     if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) return METEORA_ERR_CUDA;
-    rc = launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, Bt, u, z, dl, counts, offsets, perm,
-                              (int32_t*)workspace, dWg, st);
+    return launch_gate_backward(x, A, B, dy, topk_idx, topk_w, *shape, B ? Bt : const_cast<void*>(Bt_ready), u, z, dl,
+                                S > 0 ? dlogit : nullptr, counts, offsets, perm, (int32_t*)workspace, dWg, st);
+}
+
+int meteora_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
+                          const float* topk_w, const meteora_shape_t* shape, float* dlogit, float* dWg,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    if (shape && shape->T > 0 && !B) return METEORA_ERR_INVALID_ARG;
+    return gate_backward_impl(x, A, B, nullptr, dy, topk_idx, topk_w, shape, dlogit, dWg, workspace, workspace_bytes,
+                              stream);
+}
+
+int meteora_pad_adapters_bytes(const meteora_shape_t* shape, size_t* a_bytes, size_t* b_bytes) {
+    if (check_shape(shape, true, true) != METEORA_OK || !rank_pad_applies(*shape)) return 0;
+    const meteora_shape_t e = rank_padded(*shape);
+    if (a_bytes) *a_bytes = (size_t)e.N * e.r * e.d_in * 2;
+    if (b_bytes) *b_bytes = (size_t)e.N * e.d_out * e.r * 2;
+    return e.r;
+}
+
+int meteora_pad_adapters(const void* A, const void* B, const meteora_shape_t* shape, void* A_pad, void* B_pad,
+                         void* stream) {
+    int rc = check_shape(shape, true, true);
     if (rc != METEORA_OK) return rc;
-    if (dlogit && S > 0)
-        return cuda_status(cudaMemcpyAsync(dlogit, dl, S * sizeof(float), cudaMemcpyDeviceToDevice, st));
-    return METEORA_OK;
+    if (!A || !B || !A_pad || !B_pad) return METEORA_ERR_INVALID_ARG;
+    if (!rank_pad_applies(*shape)) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(A) || !aligned16(A_pad) || !aligned16(B_pad)) return METEORA_ERR_MISALIGNED;
+    const meteora_shape_t e = rank_padded(*shape);
+    k_pad_rank<<<296, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)B,
+                                                      (__nv_bfloat16*)A_pad, (__nv_bfloat16*)B_pad, shape->N, shape->r,
+                                                      e.r, shape->d_in, shape->d_out);
+    return last_launch_status();
+}
+
+size_t meteora_adapters_bt_bytes(const meteora_shape_t* shape) {
+    if (check_shape(shape, true, true) != METEORA_OK) return 0;
+    return (size_t)shape->N * shape->d_out * shape->r * elem_size(shape->dtype);
+}
+
+int meteora_transpose_adapters_b(const void* B, const meteora_shape_t* shape, void* Bt, void* stream) {
+    int rc = check_shape(shape, true, true);
+    if (rc != METEORA_OK) return rc;
+    if (!B || !Bt) return METEORA_ERR_INVALID_ARG;
+    if (!aligned16(B) || !aligned16(Bt)) return METEORA_ERR_MISALIGNED;
+    return launch_transpose_b(B, *shape, Bt, (cudaStream_t)stream);
+}
+
+int meteora_gate_backward_bt(const void* x, const void* A, const void* Bt, const void* dy, const int32_t* topk_idx,
+                             const float* topk_w, const meteora_shape_t* shape, float* dlogit, float* dWg,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (shape && shape->T > 0 && !Bt) return METEORA_ERR_INVALID_ARG;
+    return gate_backward_impl(x, A, nullptr, Bt, dy, topk_idx, topk_w, shape, dlogit, dWg, workspace, workspace_bytes,
+                              stream);
 }
 
 int meteora_linear_forward_host(const void* x_host, const void* W0, const void* A, const void* B,

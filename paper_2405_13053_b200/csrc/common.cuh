@@ -60,8 +60,9 @@ int launch_select_from_stacked(const float* u_all, int ld_u, int col_logits, int
 // route.cu
 int launch_gate_backward(const void* x, const void* A, const void* B, const void* dy, const int32_t* topk_idx,
                          const float* topk_w, const meteora_shape_t& s, void* Bt, float* u, float* z, float* dlogit,
-                         int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* status, float* dWg,
-                         cudaStream_t st);
+                         float* dlogit_out, int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* status,
+                         float* dWg, cudaStream_t st);
+int launch_transpose_b(const void* B, const meteora_shape_t& s, void* Bt, cudaStream_t st);
 bool gate_backward_dense(const meteora_shape_t& s);            // both shrinks as dense products on the tensor cores
 size_t gate_backward_shrink_floats(const meteora_shape_t& s);  // floats of each of the two shrink outputs
 int launch_route(const int32_t* topk_idx, int T, int k, int N, int32_t* counts, int32_t* offsets, int32_t* perm,
@@ -80,6 +81,10 @@ int launch_gemm_simt(const void* x, const void* W0, const void* B, const int32_t
 bool tc_path_supported(const meteora_shape_t& s);
 int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits);  // row pitch (floats) of u_all
 int stacked_zsplits_bound(int T);                                  // upper bound of those copies, sizes the workspace
+bool stacked_dual_supported(const meteora_shape_t& s);            // both shrinks of the gate gradient in one launch?
+int stacked_dual_zsplits(const meteora_shape_t& s);               // copies of its output
+int launch_stacked_dual_tc(const void* x, const void* A, const void* dy, const void* Bt, const meteora_shape_t& s,
+                           float* out, int32_t* status, cudaStream_t st);
 int tc_stacked_zsplits(const meteora_shape_t& s);                 // copies of u_all the stacked shrink writes (<= 4)
 int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const meteora_shape_t& s,
                              const Workspace& ws, cudaStream_t st);

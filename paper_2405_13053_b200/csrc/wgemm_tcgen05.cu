@@ -92,6 +92,8 @@ struct WGemmParams {
     int32_t* status;
     int pdl_wait;        // epilogue waits for the preceding grid before reading its results
     int pdl_trigger;     // let the dependent grid start as soon as this one is resident
+    int x_alt;           // MODE_STACKED: row tiles >= split_tile multiply the tokens of the FOURTH tensor map over
+    int ksteps1;         //   ksteps1 k-steps (two stacked products with different token operands in one launch)
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -476,8 +478,10 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const int tok0 = blockIdx.y * p.BN;
     const int ntok = min(p.BN, p.T - tok0);
     // contraction range of this CTA: first cut by grid z, then by cluster rank
-    const int kz0 = (int)(((long long)p.ksteps * blockIdx.z) / p.zsplits);
-    const int kz1 = (int)(((long long)p.ksteps * (blockIdx.z + 1)) / p.zsplits);
+    const bool second_x = p.x_alt && tile_m >= p.split_tile;
+    const int ksteps_here = second_x ? p.ksteps1 : p.ksteps;
+    const int kz0 = (int)(((long long)ksteps_here * blockIdx.z) / p.zsplits);
+    const int kz1 = (int)(((long long)ksteps_here * (blockIdx.z + 1)) / p.zsplits);
     const int ks0 = kz0 + (int)(((long long)(kz1 - kz0) * split) / S);
     const int ks1 = kz0 + (int)(((long long)(kz1 - kz0) * (split + 1)) / S);
     const int nks = ks1 - ks0;
@@ -513,6 +517,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
         if (lane == 0) {
             const bool second = tile_m >= p.split_tile;
             const CUtensorMap* tmW = second ? &tmW1 : &tmW0;
+            const CUtensorMap* tmT = second_x ? &tmY : &tmX;
             const int row0 = (second ? tile_m - p.split_tile : tile_m) * kBM;
             int issued = 0;
             bool ok = true;
@@ -526,10 +531,10 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
                 mbar_expect_tx(full, stage_bytes);
                 if (p.maps3d) {      // one instruction per operand brings kc consecutive 64-element chunks
                     tma_load_3d(dst, tmW, 0, row0, kstep, full);
-                    tma_load_3d(dst + p.kc * kWTileBytes, &tmX, 0, tok0, kstep, full);
+                    tma_load_3d(dst + p.kc * kWTileBytes, tmT, 0, tok0, kstep, full);
                 } else {
                     tma_load_2d(dst, tmW, kstep * kBK, row0, full);
-                    tma_load_2d(dst + kWTileBytes, &tmX, kstep * kBK, tok0, full);
+                    tma_load_2d(dst + kWTileBytes, tmT, kstep * kBK, tok0, full);
                 }
                 issued = i + 1;
             }
@@ -822,7 +827,7 @@ int tc_stacked_pitch(const meteora_shape_t& s, int* col_logits) {
 
 struct Plan;
 static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi = false,
-                      int bn_force = 0, bool no_mma_expand = false);
+                      int bn_force = 0, bool no_mma_expand = false, int K2 = 0, int splits_force = 0, int zcap_force = 0);
 
 struct Plan {
     int BN, n_tiles, splits, zsplits, stages, kc, maps3d, tmem_cols;
@@ -844,16 +849,35 @@ int stacked_zsplits_bound(int T) {
     return std::min(kMaxZSplits, std::max(1, 148 / tiles));
 }
 
+// K2 > 0: part of the row tiles contracts over K2 instead of K (two stacked products in one launch); the plan is
+// made for the shorter of the two and its k-steps per stage divide both.  splits_force / zcap_force: cluster size and
+// bound of the grid-z slices chosen by the caller (the tuning knobs still win).
 static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int k, bool fused_epi, int bn_force,
-                      bool no_mma_expand) {
+                      bool no_mma_expand, int K2, int splits_force, int zcap_force) {
     const Tuning& tn = tuning();
     Plan pl = {};
+    const int ksteps_long = (std::max(K, K2) + kBK - 1) / kBK;
+    if (K2 > 0 && K2 < K) std::swap(K, K2);
     const int ksteps = (K + kBK - 1) / kBK;
-    // tokens per tile: a decode batch is one tile; a prefill batch uses 256-token tiles unless those leave SMs
-    // idle, then 128 (prefill tiles are never split along the contraction axis: summing 128 x 256 partial
-    // tiles across a cluster costs more than it gains)
+    // tokens per tile: a decode batch is one tile; a prefill batch uses 256-token tiles (never split along the
+    // contraction axis while they fill the SMs: summing 128 x 256 partial tiles across a cluster costs more than it
+    // gains there).
     int bn = tn.tile_tokens > 0 ? tn.tile_tokens : (T <= 256 ? (T + 15) / 16 * 16 : 256);
-    if (tn.tile_tokens == 0 && T > 256 && row_tiles * ((T + 255) / 256) < sm_count()) bn = 128;
+    // A prefill grid that leaves SMs idle with 256-token tiles: over a long contraction axis (from 8192) two CTAs
+    // share a 256-token tile's axis when that still fits the SMs, else 128-token tiles (and two CTAs per tile
+    // while those fill less than half of the SMs).  Measured on B200, whole layer: 14336 -> 4096 at 512 tokens 100.8 us
+    // with 128-token tiles, 82.4 with 256-token tiles on two CTAs each (106 on pairs of SMs); 4096 -> 1024 at 512
+    // tokens 31.7 -> 26.8 us and at 1024 tokens 39.4 -> 34.8 with two CTAs per 128-token tile; 4096 -> 4096 at 512
+    // tokens stays on 128-token tiles (33.6 us against 41.2).
+    bool prefill_split2 = false;
+    if (tn.tile_tokens == 0 && T > 256 && row_tiles * ((T + 255) / 256) < sm_count()) {
+        if (lora && K >= 8192 && row_tiles * ((T + 255) / 256) * 2 <= sm_count()) {
+            prefill_split2 = true;
+        } else {
+            bn = 128;
+            prefill_split2 = lora && row_tiles * ((T + 127) / 128) * 2 <= sm_count();
+        }
+    }
     if (bn_force > 0) bn = bn_force;
     bn = std::min(256, std::max(16, (bn + 15) / 16 * 16));
     pl.BN = bn;
@@ -861,11 +885,14 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     const int tiles = row_tiles * pl.n_tiles;
     const int sms = sm_count();
     int splits = 1;
-    if (tn.splits > 0) {
-        splits = tn.splits >= 8 ? 8 : tn.splits >= 4 ? 4 : tn.splits >= 2 ? 2 : 1;
+    if (tn.splits > 0 || splits_force > 0) {
+        const int want = tn.splits > 0 ? tn.splits : splits_force;
+        splits = want >= 8 ? 8 : want >= 4 ? 4 : want >= 2 ? 2 : 1;
     } else if (pl.n_tiles == 1) {
         while (splits < 8 && tiles * splits * 2 <= sms) splits *= 2;
         if (splits < 8 && tiles * splits * 4 < sms * 3 && tiles * splits * 2 <= 2 * sms) splits *= 2;
+    } else if (prefill_split2 && bn_force == 0) {
+        splits = 2;
     }
     while (splits > 1 && splits > ksteps) splits /= 2;
     pl.splits = splits;
@@ -880,7 +907,8 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
             splits = tn.splits > 0 ? splits : 1;
             pl.splits = splits;
         }
-        const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits) : (tn.stacked_direct ? kMaxZSplits : 4);
+        const int zcap = tn.zmax > 0 ? std::min(tn.zmax, kMaxZSplits)
+                         : zcap_force > 0 ? std::min(zcap_force, kMaxZSplits) : (tn.stacked_direct ? kMaxZSplits : 4);
         pl.zsplits = std::min(zcap, std::max(1, ksteps / splits / 2));
     } else if (!lora) {
         // Stacked shrink of a prefill batch: never a cluster (summing 128 x 256 partial tiles through
@@ -934,21 +962,21 @@ static Plan make_plan(int row_tiles, int T, int K, bool lora, int N, int r, int 
     // k-steps per stage: issuing a TMA copy costs about as much as moving 16 KB, so with the 3-D maps one
     // instruction per operand fetches up to 4 consecutive k-steps, as long as that count divides every
     // CTA's share of the contraction axis and at least two stages still fit.
-    pl.maps3d = (K % kBK) == 0 ? 1 : 0;
+    pl.maps3d = (K % kBK) == 0 && (K2 % kBK) == 0 ? 1 : 0;
     int kc = 1;
     const int parts = splits * pl.zsplits;
-    if (pl.maps3d && ksteps % parts == 0) {
-        const int per = ksteps / parts;
+    if (pl.maps3d && ksteps % parts == 0 && ksteps_long % parts == 0) {
+        const int per = ksteps / parts, per2 = ksteps_long / parts;
         for (int cand = 4; cand > 1; cand /= 2)
-            if (per % cand == 0 && (size_t)std::max(2, tn.stages) * cand * chunk_bytes <= avail) {
+            if (per % cand == 0 && per2 % cand == 0 && (size_t)std::max(2, tn.stages) * cand * chunk_bytes <= avail) {
                 kc = cand;
                 break;
             }
-        if (tn.kc > 0 && per % tn.kc == 0) kc = tn.kc;
+        if (tn.kc > 0 && per % tn.kc == 0 && per2 % tn.kc == 0) kc = tn.kc;
     }
     pl.kc = kc;
     const size_t stage_bytes = kc * chunk_bytes;
-    const int niter = (ksteps_cta + kc - 1) / kc + 1;
+    const int niter = (std::max(ksteps_cta, ksteps_long / (splits * pl.zsplits)) + kc - 1) / kc + 1;
     int stages;
     if (tn.stages > 0) {
         stages = tn.stages;
@@ -1146,6 +1174,53 @@ int launch_stacked_shrink_tc(const void* x, const void* A, const void* Wg, const
     p.pdl_wait = 0;
     p.pdl_trigger = tuning().pdl ? 1 : 0;
     return launch_wgemm(mA, mG, mX, mX, p, row_tiles, pl, false, st);
+}
+
+// Two stacked shrinks with different token operands as ONE launch, for the gate gradient of a decode batch:
+// out[z][t][col] with col = e*r + p for [A_0; ..; A_{N-1}] x (contraction over d_in) and col = half + e*r + p for
+// [Bt_0; ..; Bt_{N-1}] dy (contraction over d_out), half = the A rows padded to whole 128-row tiles, row pitch
+// 2 * half.  Batches of one token tile only (T <= 256).
+bool stacked_dual_supported(const meteora_shape_t& s) {
+    meteora_shape_t sb = s;
+    sb.d_in = s.d_out;
+    return s.T <= 256 && !tuning().stacked_direct && tc_path_supported(s) && tc_path_supported(sb);
+}
+
+static Plan make_dual_plan(const meteora_shape_t& s) {
+    const int a_tiles = (s.N * s.r + kBM - 1) / kBM;
+    // Measured on B200 (4096 -> 4096, 128 tokens; the whole gradient per call): clusters of 8 with 4 slices 30.6 us,
+    // clusters of 4: 23.5, of 2 with 16 slices: 24.0, no cluster and 16 slices, each stored straight to its copy of
+    // the output: 21.9 (32 slices: 25.5).
+    return make_plan(2 * a_tiles, s.T, s.d_in, false, s.N, s.r, s.k, false, 0, false, s.d_out, 1, 16);
+}
+
+int stacked_dual_zsplits(const meteora_shape_t& s) { return make_dual_plan(s).zsplits; }
+
+int launch_stacked_dual_tc(const void* x, const void* A, const void* dy, const void* Bt, const meteora_shape_t& s,
+                           float* out, int32_t* status, cudaStream_t st) {
+    const int a_rows = s.N * s.r;
+    const int a_tiles = (a_rows + kBM - 1) / kBM;
+    const Plan pl = make_dual_plan(s);
+    if (pl.n_tiles != 1) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    CUtensorMap mA, mB, mX, mD;
+    int rc;
+    if ((rc = get_tensor_map(A, s.d_in, a_rows, kBM, pl.maps3d ? pl.kc : 0, &mA)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Bt, s.d_out, a_rows, kBM, pl.maps3d ? pl.kc : 0, &mB)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, pl.BN, pl.maps3d ? pl.kc : 0, &mX)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(dy, s.d_out, s.T, pl.BN, pl.maps3d ? pl.kc : 0, &mD)) != METEORA_OK) return rc;
+    WGemmParams p = {};
+    fill_common(p, pl, s.T, s.d_in, status);
+    p.split_tile = a_tiles;
+    p.rows0 = p.rows1 = a_rows;
+    p.mode = MODE_STACKED;
+    p.u_all = out;
+    p.ld_u = 2 * a_tiles * kBM;
+    p.u_all_zstride = (size_t)s.T * p.ld_u;
+    p.col1 = a_tiles * kBM;
+    p.x_alt = 1;
+    p.ksteps1 = (s.d_out + kBK - 1) / kBK;
+    p.pdl_trigger = 1;                      // the kernel that follows waits for this grid before it reads
+    return launch_wgemm(mA, mB, mX, mD, p, 2 * a_tiles, pl, false, st);
 }
 
 // Prefill batches on pairs of SMs (wgemm_pair.cuh): 256 x 256 tiles, ranks that are multiples of 8, y stored by TMA.

@@ -34,6 +34,11 @@ def dy_like(w, seed):
     dict(T=33, d_in=128, d_out=100, N=10, r=8, k=2, dtype="bf16"),               # d_out no multiple of 8: grouped shrink
     dict(T=130, d_in=1024, d_out=256, N=64, r=24, k=4, dtype="bf16"),            # 1536 stacked rows, rank 24
     dict(T=90, d_in=256, d_out=512, N=128, r=8, k=3, dtype="bf16"),              # 128 adapters
+    dict(T=128, d_in=1024, d_out=640, N=28, r=8, k=2, dtype="bf16"),             # both shrinks in one launch, 16 / 10 k-steps
+    dict(T=256, d_in=640, d_out=2048, N=28, r=8, k=2, dtype="bf16"),             # the same, the longer axis second
+    dict(T=1024, d_in=512, d_out=512, N=28, r=8, k=2, dtype="bf16"),             # the most slots without buckets
+    dict(T=1025, d_in=512, d_out=512, N=28, r=8, k=2, dtype="bf16"),             # the fewest with
+    dict(T=16, d_in=4096, d_out=4096, N=28, r=8, k=2, dtype="bf16"),             # a decode batch at config 1's shape
 ])
 def test_gate_backward_matches_oracle(case):
     kw = dict(case)
@@ -45,8 +50,13 @@ def test_gate_backward_matches_oracle(case):
     dy = torch.from_numpy(dy_np).to("cuda").to(x.dtype)
     dWg, dlogit = mb.meteora_gate_backward(x, A, B, dy, idx, wts, w.temperature)
     dWg2, _ = mb.meteora_gate_backward(x, A, B, dy, idx, wts, w.temperature)
+    # the adapters transposed beforehand (they are fixed while the gates train): the same numbers, bit for bit
+    Bt = mb.meteora_transpose_adapters_b(B)
+    assert torch.equal(Bt, B.transpose(1, 2).contiguous())
+    dWg3, dlogit3 = mb.meteora_gate_backward(x, A, None, dy, idx, wts, w.temperature, Bt=Bt)
     torch.cuda.synchronize()
     assert torch.equal(dWg, dWg2)                                     # fixed summation order
+    assert torch.equal(dWg, dWg3) and torch.equal(dlogit, dlogit3)
     o_dlogit, o_dWg = oracle.gate_backward(w["x"], w["A"], w["B"], w["Wg"], dy_np, idx.cpu().numpy(), w.temperature)
     if w.k == 1:
         assert float(dWg.abs().max()) == 0.0 and np.all(o_dWg == 0.0)
@@ -66,3 +76,8 @@ def test_gate_backward_argument_errors():
     p = buf.data_ptr()
     assert lib.meteora_gate_backward(p, p, p, p, p, p, ctypes.byref(shape), None, None, p, buf.numel(), None) == -1
     assert lib.meteora_gate_backward(p, p, p, p, p, p, ctypes.byref(shape), None, p, p, 64, None) == -4
+    assert lib.meteora_gate_backward(p, p, None, p, p, p, ctypes.byref(shape), None, p, p, buf.numel(), None) == -1
+    assert lib.meteora_gate_backward_bt(p, p, None, p, p, p, ctypes.byref(shape), None, p, p, buf.numel(), None) == -1
+    assert lib.meteora_gate_backward_bt(p, p, p, p, p, p, ctypes.byref(shape), None, p, p, 64, None) == -4
+    assert lib.meteora_transpose_adapters_b(None, ctypes.byref(shape), p, None) == -1
+    assert lib.meteora_adapters_bt_bytes(ctypes.byref(shape)) == 8 * 64 * 8 * 2

@@ -214,6 +214,8 @@ FORWARD_CASES = [
     dict(T=20, d_in=256, d_out=128, N=8, r=8, k=1, dtype="bf16"),                 # top-1
     dict(T=40, d_in=512, d_out=256, N=28, r=32, k=4, dtype="bf16"),               # rank 32, top-4, decode batch
     dict(T=30, d_in=512, d_out=384, N=28, r=4, k=2, dtype="bf16"),                # rank 4: adapters zero-padded to 8
+    dict(T=300, d_in=1024, d_out=256, N=28, r=8, k=2, dtype="bf16"),              # short prefill grid: two CTAs per 128-token tile
+    dict(T=700, d_in=8192, d_out=512, N=28, r=8, k=2, dtype="bf16"),              # long axis: two CTAs per 256-token tile
     dict(T=300, d_in=256, d_out=256, N=12, r=12, k=3, dtype="bf16"),              # rank 12 -> 16, prefill batch
     dict(T=600, d_in=512, d_out=200, N=28, r=64, k=2, dtype="bf16"),              # rank 64 prefill, d_out % 8 == 0 only
     dict(T=24, d_in=256, d_out=136, N=4, r=8, k=4, dtype="bf16", temperature=20.0),  # k = N with temperature
