@@ -104,7 +104,8 @@ def kernel_sha():
     white space removed, so that an edit of a comment does not void the figure and an edit of the code does."""
     import re
     h = hashlib.sha256()
-    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "decode_stream.cuh", "wgemm_pair.cuh", "select.cuh"):
+    for name in ("wgemm_tcgen05.cu", "decode_fused.cuh", "decode_stream.cuh", "decode_cluster.cuh", "wgemm_pair.cuh",
+                 "select.cuh"):
         with open(os.path.join(ROOT, "paper_2405_13053_b200", "csrc", name), "r") as fh:
             text = fh.read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)

@@ -310,6 +310,20 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *                    the kernel is launched without it (pdl_decode_refused in the plan string counts these).
  *   "pair"           default 1 = prefill base product on pairs of SMs (two-CTA MMA, 256 x 256 tiles)
  *                    where the pairs cover a quarter of the SMs; 0 = never; 2 = wherever the shape allows
+ *   "stream"         decode batches up to 128 tokens on the streamed one-launch kernel: default 1 = planner's
+ *                    choice of one or two CTAs per SM, 0 = never (the cooperative kernel takes them), 2 = always one
+ *                    CTA per SM with a deep ring, 3 = two per SM wherever they fit
+ *   "pf"             L2 prefetch of the weights beyond the streamed kernel's ring: default 0 / -1 = none, n > 0 = cap in MB
+ *   "own_local"      default 1 = a CTA's own row slice of its partial tile stays in shared memory; 0 = through scratch
+ *   "bulk_deliver"   1 = the partial tiles leave through shared memory and bulk copies instead of plain stores
+ *   "pair_decode"    streamed kernel on pairs of CTAs (two-CTA MMA, half a token tile each): default 0 = never,
+ *                    1 = from 64 tokens up, 2 = from 17 tokens up
+ *   "cluster_decode" decode batches on the clustered one-launch kernel (the CTAs of a row tile exchange their partial
+ *                    tiles through distributed shared memory, the stacked shrink is spread over all CTAs):
+ *                    default 0 = never (measured slower than the streamed kernel except for the largest layers),
+ *                    other = wherever the device can hold all clusters at once
+ *   "group_pairs"    > 0 = row pairs per scheduling group of the prefill kernel on pairs of SMs (0 = planner's choice)
+ *   "wait_limit_us"  > 0 = limit of every bounded device-side wait in microseconds (0 = the default of about a second)
  * Unknown names return METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
  */
 int meteora_set_tuning(const char* name, int value);

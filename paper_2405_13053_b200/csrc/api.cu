@@ -109,6 +109,15 @@ static int forward_device(const void* x, const void* W0, const void* A, const vo
     }
     Profile& pf = profile();
     const bool timed = pf.open && 2 * (pf.used + 1) <= (int)pf.ev.size();
+    if (decode_cluster_supported(s)) {
+        if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
+        rc = launch_decode_cluster(x, W0, A, B, Wg, s, ws, y, st);
+        if (rc != kLaunchRefused) {
+            if (timed) cudaEventRecord(pf.ev[2 * pf.used++ + 1], st);
+            return rc;
+        }
+        tuning().fused_refused += 1;   // the cluster launch was refused: the streamed kernel takes the call
+    }
     if (decode_stream_supported(s)) {
         if (timed) cudaEventRecord(pf.ev[2 * pf.used], st);
         rc = launch_decode_stream(x, W0, A, B, Wg, s, ws, y, st);
@@ -510,6 +519,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "group_pairs")) t.group_pairs = value;
     else if (!strcmp(name, "bulk_deliver")) t.bulk_deliver = value;
     else if (!strcmp(name, "pair_decode")) t.pair_decode = value;
+    else if (!strcmp(name, "cluster_decode")) t.cluster_decode = value;
     else if (!strcmp(name, "wait_limit_us")) return set_wait_limit_us(value);
     else if (!strcmp(name, "coop")) t.coop = value;
     else if (!strcmp(name, "no_hold")) t.no_hold = value;

@@ -112,6 +112,9 @@ int set_wait_limit_us(int us);   // limit of the bounded device-side waits on th
 int launch_decode_fused(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                         const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
 // streamed decode kernel (wgemm_tcgen05.cu + decode_stream.cuh): up to 128 tokens, two launches resident at a time
+bool decode_cluster_supported(const meteora_shape_t& s);
+int launch_decode_cluster(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                          const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
 bool decode_stream_supported(const meteora_shape_t& s);
 int launch_decode_stream(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
                          const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st);
@@ -143,6 +146,7 @@ struct Tuning {
     int no_hold = 0;         // decode kernel, head start of the aux CTAs: 0 planner's choice, 1 none, 64 counter wait, other = nanoseconds
     int hold_after = 0;      // decode kernel: ring stages of W0 the main CTAs request before the aux CTAs' head start (0: planner, -1: none)
     int narrow_select = 0;   // decode kernel's selection: 0 by batch size, 1 always two narrow round trips, -1 always one wide one
+    int cluster_decode = 0;  // decode batches on clusters that exchange through distributed shared memory (0: never)
     int pdl_decode = 1;      // the decode kernel is launched with programmatic stream serialization as well (0: not)
     int pdl_decode_refused = 0;   // launches the driver refused with both attributes (repeated without it)
     int fused_refused = 0;   // cooperative launches the driver refused (the chain ran instead)

@@ -706,6 +706,7 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
 #include "decode_fused.cuh"
 #include "wgemm_pair.cuh"
 #include "decode_stream.cuh"
+#include "decode_cluster.cuh"
 
 namespace meteora {
 
@@ -1917,9 +1918,214 @@ int launch_decode_stream(const void* x, const void* W0, const void* A, const voi
     return cuda_status(cudaLaunchKernelEx(&cfg, k_decode_stream<false>, mW, mA, mAt, mG, mX, mX1, d));
 }
 
+// ------------------------------------------------------------------------------------------------
+// Clustered decode launch (decode_cluster.cuh): the CTAs of a row tile exchange through distributed shared memory.
+// ------------------------------------------------------------------------------------------------
+struct ClusterPlan {
+    bool ok;
+    int why;       // why not: 1 knob/shape, 2 clusters do not fit the device, 5 shared memory
+    int BN, stages, tmem_cols, acc2_col, S, row_tiles, n_cta;
+    int a_tiles, aux_tiles, gate_tile, gate_row0, SL, n_sel;
+    int slab_off, recv_off, delta_off, route_off, ring_bytes;
+    size_t smem;
+};
+
+// How many clusters of `S` CTAs with `smem` bytes of dynamic shared memory the device holds at once (0: unknown).
+static int cluster_capacity(int S, size_t smem) {
+    static int cache[64][9][2] = {};                             // [device][S][smem above / below 113 KB]
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || S < 1 || S > 8) return 0;
+    int& slot = cache[dev][S][smem > kTwoPerSmBytes ? 0 : 1];
+    if (slot != 0) return slot;
+    if (cudaFuncSetAttribute(k_decode_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S * 148);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem > kTwoPerSmBytes ? 226 * 1024 : kTwoPerSmBytes;   // the most a plan of that class may ask for
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, k_decode_cluster, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    slot = n > 0 ? n : -1;
+    return slot;
+}
+
+static ClusterPlan make_cluster_plan(const meteora_shape_t& s) {
+    const Tuning& tn = tuning();
+    ClusterPlan cp = {};
+    cp.why = 1;
+    if (!tn.fused || !tn.cluster_decode || tn.simt_expand) return cp;
+    if (!tc_path_supported(s) || s.T > 128 || s.r % 8 != 0 || s.d_in % kBK != 0 || s.d_out <= 0) return cp;
+    const int sms = std::min(sm_count(), 148);
+    const int ksteps = s.d_in / kBK;
+    cp.row_tiles = (s.d_out + kBM - 1) / kBM;
+    cp.a_tiles = (s.N * s.r + kBM - 1) / kBM;
+    const int tail_rows = s.N * s.r - (cp.a_tiles - 1) * kBM;
+    const bool merged = tail_rows % 8 == 0 && tail_rows + s.N <= kBM;
+    cp.aux_tiles = merged ? cp.a_tiles : cp.a_tiles + 1;
+    cp.gate_tile = cp.aux_tiles - 1;
+    cp.gate_row0 = merged ? tail_rows : 0;
+    if (cp.row_tiles < cp.aux_tiles || cp.row_tiles > sms) return cp;       // every stacked tile needs a cluster
+    cp.SL = std::min(std::min(cp.row_tiles / cp.aux_tiles, 16), ksteps);
+    if (cp.SL * cp.aux_tiles > kEpiThreads) return cp;                      // one thread issues each partial's copy
+    cp.BN = (s.T + 15) / 16 * 16;
+    int cols = 32;
+    while (cols < cp.BN) cols *= 2;
+    cp.acc2_col = cols;
+    cp.tmem_cols = 2 * cols;
+    cp.why = 2;
+    // cluster size: as many CTAs per row tile as the SMs allow (at most 8), and the device must hold all clusters at once
+    int S = tn.splits > 0 ? std::min(tn.splits, 8) : std::min(8, sms / cp.row_tiles);
+    S = std::min(S, ksteps);
+    for (; S >= 1; --S) {
+        const int cap = cluster_capacity(S, 226 * 1024);
+        if (cap >= cp.row_tiles) break;
+    }
+    if (S < 1) return cp;
+    cp.S = S;
+    cp.n_cta = cp.row_tiles * S;
+    cp.n_sel = std::min(s.T, cp.n_cta);
+    cp.why = 5;
+    const int cpa = s.r / 8;
+    const int nq_max = (32 + S - 1) / S;
+    const size_t slab_bytes = (size_t)s.N * cpa * 4 * nq_max * 16;
+    const size_t blk_max = (size_t)cp.BN * 4 * nq_max * 4;
+    // what the selection puts into the receive blocks: its tokens' rows of all partials and their sums behind them
+    const int ntl_max = (s.T + cp.n_cta - 1) / cp.n_cta;
+    const size_t sel_bytes = (size_t)(cp.SL * cp.aux_tiles + cp.aux_tiles) * ntl_max * kBM * 4;
+    const size_t recv_bytes = align_up(std::max((size_t)S * blk_max, sel_bytes), 128);
+    const size_t route_bytes = align_up(align_up((size_t)s.T * s.k * 4, 16), 128) + (size_t)s.T * s.k * s.r * 4;
+    cp.slab_off = (int)align_up((size_t)(2 * kStreamBarSlots + 7) * 8 + 16, 128);
+    cp.recv_off = (int)align_up(cp.slab_off + slab_bytes, 128);
+    cp.delta_off = (int)(cp.recv_off + recv_bytes);
+    cp.route_off = (int)align_up(cp.delta_off + blk_max, 128);
+    const size_t tail_bytes = cp.route_off + align_up(route_bytes, 128);
+    const size_t stage_bytes = kWTileBytes + (size_t)cp.BN * 128;
+    const size_t budget = 226 * 1024;
+    if (1024 + tail_bytes + 2 * stage_bytes > budget) return cp;
+    const int n_it_max = (ksteps + S - 1) / S + (ksteps / S + cp.SL - 1) / cp.SL + 1;
+    int stages = (int)std::min<size_t>((budget - 1024 - tail_bytes) / stage_bytes, (size_t)std::min(kStreamBarSlots, n_it_max));
+    if (tn.stages > 0) stages = std::min(tn.stages, stages);
+    if (stages < 2) return cp;
+    cp.stages = stages;
+    cp.ring_bytes = (int)(stages * stage_bytes);
+    cp.smem = 1024 + cp.ring_bytes + tail_bytes;
+    cp.why = 0;
+    cp.ok = true;
+    return cp;
+}
+
+bool decode_cluster_supported(const meteora_shape_t& s) { return make_cluster_plan(s).ok; }
+
+int launch_decode_cluster(const void* x, const void* W0, const void* A, const void* B, const void* Wg,
+                          const meteora_shape_t& s, const Workspace& ws, void* y, cudaStream_t st) {
+    const ClusterPlan cp = make_cluster_plan(s);
+    if (!cp.ok) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    CUtensorMap mW, mA, mAt, mG, mX;
+    int rc;
+    const int tail_box = cp.gate_row0 > 0 ? cp.gate_row0 : kBM, gate_box = kBM - cp.gate_row0;
+    if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, 1, &mW)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, kBM, 1, &mA)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(A, s.d_in, s.N * s.r, tail_box, 1, &mAt)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(Wg, s.d_in, s.N, gate_box, 1, &mG)) != METEORA_OK) return rc;
+    if ((rc = get_tensor_map(x, s.d_in, s.T, cp.BN, 1, &mX)) != METEORA_OK) return rc;
+    ClusterParams d = {};
+    d.T = s.T;
+    d.BN = cp.BN;
+    d.ksteps = s.d_in / kBK;
+    d.stages = cp.stages;
+    d.tmem_cols = cp.tmem_cols;
+    d.acc2_col = cp.acc2_col;
+    d.N = s.N;
+    d.r = s.r;
+    d.k = s.k;
+    d.d_out = s.d_out;
+    d.row_tiles = cp.row_tiles;
+    d.S = cp.S;
+    d.aux_tiles = cp.aux_tiles;
+    d.a_tiles = cp.a_tiles;
+    d.gate_tile = cp.gate_tile;
+    d.gate_row0 = cp.gate_row0;
+    d.SL = cp.SL;
+    d.n_stk = cp.SL * cp.aux_tiles * cp.S;
+    d.n_sel = cp.n_sel;
+    d.ring_bytes = cp.ring_bytes;
+    d.bar_slots = kStreamBarSlots;
+    d.slab_off = cp.slab_off;
+    d.recv_off = cp.recv_off;
+    d.delta_off = cp.delta_off;
+    d.route_off = cp.route_off;
+    d.inv_tau = 1.0f / s.temperature;
+    d.B = (const __nv_bfloat16*)B;
+    d.y = (__nv_bfloat16*)y;
+    d.topk_idx = ws.topk_idx;
+    d.topk_w = ws.topk_w;
+    d.uw = ws.uw;
+    d.u_part = ws.u_all;
+    d.ctr = ws.status + 16;
+    d.status = ws.status;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return METEORA_ERR_UNSUPPORTED_SHAPE;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(k_decode_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(k_decode_cluster, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+            return METEORA_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cp.n_cta);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = cp.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    const bool want_pdl = tuning().pdl_decode != 0;
+    int na = 0;
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = cp.S;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+    if (want_pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    d.pdl = want_pdl ? 1 : 0;
+#ifdef METEORA_TRACE
+    static int trace_calls = 0;
+    d.trace_call = trace_calls++;
+#endif
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, k_decode_cluster, mW, mA, mAt, mG, mX, d);
+    if (err != cudaSuccess && launch_config_refused(err)) {
+        cudaGetLastError();
+        return kLaunchRefused;
+    }
+    return cuda_status(err);
+}
+
 // Human-readable launch plan of meteora_linear_forward for this shape (for logs and benchmark records).
 int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     if (!tc_path_supported(s)) return snprintf(buf, n, "path=simt");
+    const ClusterPlan cp = make_cluster_plan(s);
+    if (cp.ok)
+        return snprintf(buf, n,
+                        "path=cluster_decode launches=1 ctas=%d row_tiles=%d cluster=%d stacked_tiles=%d stacked_slices=%d "
+                        "tile_tokens=%d stages=%d smem=%zu",
+                        cp.n_cta, cp.row_tiles, cp.S, cp.aux_tiles, cp.SL, cp.BN, cp.stages, cp.smem);
     const StreamPlan sp = make_stream_plan(s);
     if (sp.ok)
         return snprintf(buf, n,

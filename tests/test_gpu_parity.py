@@ -539,6 +539,98 @@ def test_streamed_decode_calls_share_one_workspace_back_to_back():
         assert rel_l2(y.float().cpu().numpy(), ref) <= 1e-2
 
 
+# --------------------------------------------------------------------------------------- clustered decode kernel
+# The decode kernel whose CTAs of a row tile form a thread-block cluster and exchange through distributed shared
+# memory, with the stacked shrink spread over all CTAs.  Shapes for every way its work splits: clusters of 1, 2, 3,
+# 4, 5, 7 and 8 (even and uneven row slices), k-steps that do not divide by the cluster size (17), fewer k-steps per
+# CTA than clusters per stacked tile (512: 8 k-steps), more clusters than stacked slices are used (71 row tiles),
+# a ragged last tile (1000, 1001 rows), one token, a token count that is no multiple of 16, the full 128, more
+# tokens than CTAs (128 tokens on 10 x 2 CTAs: several tokens per selecting CTA).
+@pytest.fixture
+def clustered_decode_kernel():
+    mb.meteora_set_tuning("cluster_decode", 2)
+    mb.meteora_set_tuning("wait_limit_us", 200000)                   # a wait that cannot end gives up after 0.2 s
+    yield
+    mb.meteora_set_tuning("wait_limit_us", 0)
+    mb.meteora_set_tuning("cluster_decode", CLUSTER_DEFAULT)
+
+
+CLUSTER_DEFAULT = 0
+
+
+@pytest.mark.parametrize("d_in,d_out,T,per_tile", [
+    (1024, 640, 1, 0), (1024, 640, 8, 0), (1024, 640, 100, 0), (1024, 640, 128, 0),
+    (1536, 1000, 37, 0), (1088, 768, 16, 0), (2048, 4224, 5, 0), (2048, 4224, 128, 0),
+    (512, 9000, 24, 0), (1024, 1280, 64, 1), (1024, 1280, 128, 2), (1024, 1280, 77, 3), (1024, 1001, 50, 5),
+    (1024, 384, 128, 7), (1024, 384, 19, 8), (4096, 1024, 128, 0), (4096, 4096, 128, 0), (4096, 4096, 1, 0),
+])
+def test_clustered_decode_kernel_matches_oracle(d_in, d_out, T, per_tile, clustered_decode_kernel):
+    w = workloads.make_workload("cluster", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="rms",
+                                seed=350 + T + d_out, b_std=0.3)
+    mb.meteora_set_tuning("splits", per_tile)
+    try:
+        shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+        plan = mb.meteora_describe_plan(shape)
+        assert "cluster_decode" in plan
+        if per_tile:
+            assert f"cluster={per_tile} " in plan
+        check_forward(w, y_tol=1e-2)
+        y1, i1, w1 = run_forward(w)
+        y2, i2, w2 = run_forward(w)
+        np.testing.assert_array_equal(y1, y2)                        # fixed summation order: reproducible bit for bit
+        np.testing.assert_array_equal(i1, i2)
+        np.testing.assert_array_equal(w1, w2)
+    finally:
+        mb.meteora_set_tuning("splits", 0)
+
+
+@pytest.mark.parametrize("N,k,T,r", [(4, 2, 9, 8), (16, 4, 40, 8), (33, 3, 128, 8), (2, 1, 3, 8), (28, 2, 20, 16),
+                                     (12, 2, 128, 32), (10, 3, 64, 24), (64, 8, 7, 8), (28, 1, 128, 8), (28, 2, 33, 8)])
+def test_clustered_decode_kernel_adapter_counts(N, k, T, r, clustered_decode_kernel):
+    w = workloads.make_workload("cluster_n", T=T, d_in=768, d_out=896, N=N, k=k, r=r, dtype="bf16", x_kind="normal",
+                                seed=2900 + N + r, b_std=0.3, temperature=1.0 if N != 16 else 15.0)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16, w.temperature)
+    assert "cluster_decode" in mb.meteora_describe_plan(shape)
+    check_forward(w, y_tol=1e-2)
+
+
+@pytest.mark.parametrize("knob,value", [("stages", 2), ("pdl_decode", 0), ("splits", 2)])
+def test_clustered_decode_kernel_planner_choices(knob, value, clustered_decode_kernel):
+    w = workloads.make_workload("cluster_knobs", T=70, d_in=2048, d_out=640, dtype="bf16", x_kind="normal", seed=3234,
+                                b_std=0.3)
+    shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+    y0, i0, _ = run_forward(w)
+    mb.meteora_set_tuning(knob, value)
+    try:
+        assert "cluster_decode" in mb.meteora_describe_plan(shape)
+        check_forward(w, y_tol=1e-2)
+        y1, i1, _ = run_forward(w)
+    finally:
+        mb.meteora_set_tuning(knob, {"pdl_decode": 1}.get(knob, 0))
+    same = assert_same_outside_the_band(w, i0, i1)
+    assert same.mean() > 0.97
+    assert rel_l2(y1[same], y0[same]) < 4e-3
+
+
+def test_clustered_decode_calls_share_one_workspace_back_to_back(clustered_decode_kernel):
+    T, d_in, d_out = 96, 1024, 768
+    ws_list = [workloads.make_workload(f"shared_cl{i}", T=T, d_in=d_in, d_out=d_out, dtype="bf16", x_kind="normal",
+                                       seed=8100 + i, b_std=0.3) for i in range(8)]
+    shape = mb.make_shape(T, d_in, d_out, 28, 8, 2, torch.bfloat16)
+    assert "cluster_decode" in mb.meteora_describe_plan(shape)
+    dev = [to_dev(w, "x", "W0", "A", "B", "Wg") for w in ws_list]
+    workspace = mb.alloc_workspace(shape)
+    ys = [mb.meteora_linear_forward(*t, 2, workspace=workspace) for t in dev]
+    torch.cuda.synchronize()
+    assert mb.meteora_workspace_status(workspace) == 0
+    for w, t, y in zip(ws_list, dev, ys):
+        y_alone, idx, _ = mb.meteora_linear_forward(*t, 2, return_routing=True)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(y.float().cpu().numpy(), y_alone.float().cpu().numpy())
+        ref = oracle.linear_forward_routed(w["x"], w["W0"], w["A"], w["B"], w["Wg"], idx.cpu().numpy())
+        assert rel_l2(y.float().cpu().numpy(), ref) <= 1e-2
+
+
 # Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
 # one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
 # (257), a contraction length that is no multiple of 64, and adapters up to an odd count.  The stacked shrink of
