@@ -316,6 +316,8 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *   "pf"             L2 prefetch of the weights beyond the streamed kernel's ring: default 0 / -1 = none, n > 0 = cap in MB
  *   "own_local"      default 1 = a CTA's own row slice of its partial tile stays in shared memory; 0 = through scratch
  *   "bulk_deliver"   1 = the partial tiles leave through shared memory and bulk copies instead of plain stores
+ *   "aux_plain"      default 1 = the stacked shrink's partial tiles leave the aux CTAs as plain stores; 0 = staged in
+ *                    shared memory and sent as one bulk copy each
  *   "pair_decode"    streamed kernel on pairs of CTAs (two-CTA MMA, half a token tile each): default 0 = never,
  *                    1 = from 64 tokens up, 2 = from 17 tokens up
  *   "cluster_decode" decode batches on the clustered one-launch kernel (the CTAs of a row tile exchange their partial

@@ -51,6 +51,7 @@ struct StreamParams {
     int32_t* tile_ctr;         // [row tiles] partials delivered
     int32_t* status;
     int bulk_deliver;          // the other CTAs' row slices leave through shared memory and bulk copies instead of plain stores
+    int aux_plain;             // the aux CTAs' partial tiles leave as plain stores instead of one bulk copy
     int own_local;             // the CTA's own row slice of its accumulator stays in shared memory (else through scratch like the others)
     int pdl;
     int trace_call;
@@ -350,14 +351,36 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             if (!acc_ok && lane == 0) stream_flag_error(d, 3, 600);
             acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
             tc_fence_after();
-            // the accumulator tile as it is, [token][128 rows] fp32, through the idle ring and one bulk copy
+            // the accumulator tile as it is, [token][128 rows] fp32
             const int trow = quad * 32 + lane;
-            float* stage = reinterpret_cast<float*>(ring_ptr);
-            // (all BN columns are written: the bulk copy below moves T of them, the rest are zero rows of the x tile)
-            tmem_rows_out(tmem_base + ((uint32_t)(quad * 32) << 16), c_begin, c_end, acc_ok && niter > 0, nullptr,
-                          ring + (uint32_t)trow * 4u, true, kBM);
-            (void)stage;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (d.aux_plain) {
+                // straight from registers: lane = row, a warp writes 128 contiguous bytes per token (the scratch holds
+                // BN token rows per tile, so nothing is predicated)
+                if (d.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+                float* dst = d.u_part + (((size_t)slice * d.aux_tiles + tile) * d.T) * kBM + trow;
+                for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+                    float v[16];
+                    if (acc_ok && niter > 0) {
+                        tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                    }
+                    if (c0 + 16 <= d.T) {                                      // warp-uniform: whole chunks unpredicated
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) dst[(size_t)(c0 + i) * kBM] = v[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (c0 + i < d.T) dst[(size_t)(c0 + i) * kBM] = v[i];
+                    }
+                }
+            } else {
+                // through the idle ring and one bulk copy (all BN columns are written: the copy moves T of them)
+                tmem_rows_out(tmem_base + ((uint32_t)(quad * 32) << 16), c_begin, c_end, acc_ok && niter > 0, nullptr,
+                              ring + (uint32_t)trow * 4u, true, kBM);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
         }
         __syncwarp();
         __syncthreads();
@@ -365,7 +388,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             if (d.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");     // every thread below touches the scratch
             if (threadIdx.x == 0) {
                 float* dst = d.u_part + (((size_t)slice * d.aux_tiles + tile) * d.T) * kBM;
-                bulk_store_block(dst, ring, (uint32_t)d.T * kBM * 4u);
+                if (!d.aux_plain) bulk_store_block(dst, ring, (uint32_t)d.T * kBM * 4u);
                 __threadfence();
                 atomicAdd(d.ctr + 0, 1);
                 STREAM_STAMP(3);
@@ -407,7 +430,9 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
                     }
                     rows4[it] = acc;
                 }
+                if (threadIdx.x == 0) STREAM_STAMP(10);
                 __syncthreads();
+                if (threadIdx.x == 0) STREAM_STAMP(11);
                 const int nwarps = kThreads / 32;
                 for (int tl = warp; tl < ntl && ok; tl += nwarps)
                     select_token_row(reinterpret_cast<const float*>(rows4 + tl * per_tok), d.gate_tile, d.gate_row0, t0 + tl, d.N,
@@ -640,6 +665,7 @@ k_decode_stream(const __grid_constant__ CUtensorMap tmW0, const __grid_constant_
             }
             // LoRA expand of the slice (Eq. 2) while the partials are on their way: routing and B rows are here.
             bool ok = mbar_wait(bar_route, 0);
+            if (etid == 0) STREAM_STAMP(15);
             if (!ok && lane == 0) stream_flag_error(d, 4, 850);
             const int* s_idx = reinterpret_cast<const int*>(ring_ptr + idx_off);
             const float4* s_uw4 = reinterpret_cast<const float4*>(ring_ptr + uw_off);

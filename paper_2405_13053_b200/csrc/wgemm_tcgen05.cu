@@ -1869,6 +1869,7 @@ int launch_decode_stream(const void* x, const void* W0, const void* A, const voi
     // slices have the same size) instead of plain stores.  Measured at 4096 -> 4096: the same 2.2 - 2.6 us from the
     // accumulator to the counter at 128 tokens either way, 0.3 us slower at one token; off by default.
     d.bulk_deliver = sp.S > 1 && 32 % sp.S == 0 && tuning().bulk_deliver > 0 ? 1 : 0;
+    d.aux_plain = tuning().aux_plain ? 1 : 0;
     d.own_local = tuning().own_local && sp.S > 1 ? 1 : 0;
     if (d.bulk_deliver) d.own_local = 1;
     if (sp.S == 1) d.own_local = 1;                             // the tile is the CTA's alone: nothing goes through scratch

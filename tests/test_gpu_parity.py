@@ -479,13 +479,14 @@ def test_streamed_decode_kernel_adapter_counts(N, k, T, r):
 # change the result beyond the order of the fp32 sums of the stacked shrink's slices.  (pair_decode = 1 runs the 70
 # tokens on pairs of CTAs with a two-CTA MMA, own_local = 0 sends a CTA's own row slice through scratch too.)
 @pytest.mark.parametrize("knob,value", [("stages", 2), ("kc", 2), ("pf", -1), ("pf", 1), ("stream", 2), ("aux_ctas", 4),
-                                        ("aux_ctas", 40), ("pdl_decode", 0), ("pair_decode", 1), ("own_local", 0), ("bulk_deliver", 1)])
+                                        ("aux_ctas", 40), ("pdl_decode", 0), ("pair_decode", 1), ("own_local", 0), ("bulk_deliver", 1),
+                                        ("aux_plain", 0)])
 def test_streamed_decode_kernel_planner_choices(knob, value):
     w = workloads.make_workload("stream_knobs", T=70, d_in=2048, d_out=640, dtype="bf16", x_kind="normal", seed=2234,
                                 b_std=0.3)
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
     y0, i0, _ = run_forward(w)
-    default = {"stream": 1, "pdl_decode": 1, "own_local": 1}.get(knob, 0)
+    default = {"stream": 1, "pdl_decode": 1, "own_local": 1, "aux_plain": 1}.get(knob, 0)
     mb.meteora_set_tuning(knob, value)
     try:
         assert "stream_decode" in mb.meteora_describe_plan(shape)
