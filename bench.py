@@ -39,7 +39,7 @@ NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, nominal
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "c181bb98afb407ee", "bytes_per_launch": {"128": 38595925 + 20565, "1": 37555627 + 1451}}
+NCU_TRAFFIC = {"kernel_sha": "fb61f1e632daa184", "bytes_per_launch": {"128": 38597803 + 13397, "1": 37557163 + 85}}
 
 
 def parse_args():
@@ -68,6 +68,8 @@ def parse_args():
                          "the axes of the paper's synthetic sweep (App. A.7); one JSON line each")
     ap.add_argument("--knob", action="append", default=[], metavar="NAME=VALUE",
                     help="set a measurement knob of the library (meteora_set_tuning) before timing; repeatable")
+    ap.add_argument("--gate-backward", action="store_true",
+                    help="meteora_gate_backward / _bt at 1 - 8192 tokens (4096 -> 4096), per call from a CUDA graph")
     ap.add_argument("--standalone", action="store_true",
                     help="time the standalone entry points (gate + top-k, bucketing, LoRA term by segments) beside the fused "
                          "forward's stacked shrink + selection; also part of --sweep")
@@ -1219,6 +1221,8 @@ def main():
         run_layer()
     elif args.standalone:
         run_standalone_sweep()
+    elif args.gate_backward:
+        run_gate_backward_sweep()
     elif args.decode_loop:
         run_decode_loop()
     elif args.sweep:

@@ -50,19 +50,29 @@ k_gate_dlogit(const float* __restrict__ u, const float* __restrict__ z, const in
               int zsplits_u, int zsplits_z, size_t zstride, float* __restrict__ dlogit, float* __restrict__ dlogit2) {
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
-    // launched ahead of the end of the shrinks, and lets the last kernel become resident in turn; both wait here
-    // (no-ops without the launch attribute)
+    // launched ahead of the end of the shrinks, and lets the last kernel become resident in turn (no-ops without
+    // the launch attribute)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (t >= T) return;
     const bool spread = r <= 32 && (32 % r) == 0;
     const int nq = spread ? 32 / r : 1, qg = spread ? lane / r : 0;
-    float g[METEORA_MAX_K];
-    float mean = 0.f;
-    for (int j = 0; j < k; ++j) {
-        const int e = min(max(topk_idx[(size_t)t * k + j], 0), N - 1);
-        const size_t row = dense ? (size_t)t * ld + (size_t)e * r : ((size_t)t * k + j) * r;
-        float acc = 0.f;
+    // every load of the token goes out before the first reduction: the picks' adapters and weights (inputs of the
+    // call: read while the shrinks still run), then the copies of both shrink outputs for all picks (the kernel is
+    // a chain of dependent loads otherwise)
+    int e[METEORA_MAX_K];
+    float w[METEORA_MAX_K], g[METEORA_MAX_K];
+#pragma unroll
+    for (int j = 0; j < METEORA_MAX_K; ++j) {
+        const bool live = j < k && t < T;
+        e[j] = live ? min(max(topk_idx[(size_t)t * k + j], 0), N - 1) : 0;
+        w[j] = live ? topk_w[(size_t)t * k + j] : 0.f;
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (t >= T) return;
+#pragma unroll
+    for (int j = 0; j < METEORA_MAX_K; ++j) {
+        g[j] = 0.f;
+        if (j >= k) continue;
+        const size_t row = dense ? (size_t)t * ld + (size_t)e[j] * r : ((size_t)t * k + j) * r;
         if (spread) {
             const int p = lane - qg * r;
             float uv = 0.f, zv = 0.f;
@@ -72,21 +82,28 @@ k_gate_dlogit(const float* __restrict__ u, const float* __restrict__ z, const in
                 uv += __shfl_xor_sync(0xFFFFFFFFu, uv, o);
                 zv += __shfl_xor_sync(0xFFFFFFFFu, zv, o);
             }
-            acc = qg == 0 ? uv * zv : 0.f;
+            g[j] = qg == 0 ? uv * zv : 0.f;
         } else {
             for (int p = lane; p < r; p += 32) {
                 float uv = 0.f, zv = 0.f;
                 for (int q = 0; q < zsplits_u; ++q) uv += u[q * zstride + row + p];
                 for (int q = 0; q < zsplits_z; ++q) zv += z[q * zstride + row + p];
-                acc = fmaf(uv, zv, acc);
+                g[j] = fmaf(uv, zv, g[j]);
             }
         }
-        g[j] = warp_sum(acc);
-        mean = fmaf(topk_w[(size_t)t * k + j], g[j], mean);
+    }
+    float mean = 0.f;
+#pragma unroll
+    for (int j = 0; j < METEORA_MAX_K; ++j) {
+        if (j >= k) continue;
+        g[j] = warp_sum(g[j]);
+        mean = fmaf(w[j], g[j], mean);
     }
     if (lane == 0)
-        for (int j = 0; j < k; ++j) {
-            const float v = topk_w[(size_t)t * k + j] * (g[j] - mean) * inv_tau;
+#pragma unroll
+        for (int j = 0; j < METEORA_MAX_K; ++j) {
+            if (j >= k) continue;
+            const float v = w[j] * (g[j] - mean) * inv_tau;
             dlogit[(size_t)t * k + j] = v;
             if (dlogit2) dlogit2[(size_t)t * k + j] = v;
         }
