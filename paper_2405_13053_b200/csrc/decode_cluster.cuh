@@ -321,7 +321,7 @@ k_decode_cluster(const __grid_constant__ CUtensorMap tmW0, const __grid_constant
                     cluster_flag_error(d, 4, 1400);
                     ok = false;
                 }
-                tmem_slot[1] = ok ? 1u : 0u;                               // thread 0's verdict for the other threads
+                tmem_slot[1] = ok ? 1u : 0u;                               // what thread 0 found, for the other threads
                 mbar_expect_tx(bar_sel, ok ? rows_bytes : 0u);
                 CL_STAMP(8);
             }
