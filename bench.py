@@ -224,7 +224,7 @@ def whole_job_value(modules, tokens, world, steps, ms_total):
 
 def prefill_line(mb, lib, tc_peak, tc_kind, hbm_peak):
     """One prefill figure for the default line (the headline workload is a decode batch and HBM-bound): config 2's
-    gate/up shape, 4096 -> 14336 with 2048 tokens from 4 clusters, the whole MeteoRA linear per call (three launches:
+    gate/up shape, 4096 -> 14336 with 2048 tokens from 4 clusters, the whole MeteoRA linear per call (three or four launches:
     stacked shrink, selection, base product with the expand) against the sustained bf16 tensor peak, and the
     base-product kernel alone from event pairs around its launches."""
     import ctypes
@@ -282,7 +282,7 @@ def prefill_line(mb, lib, tc_peak, tc_kind, hbm_peak):
             "frac_of_nominal": flops / us_call / 1e6 / NOMINAL_BF16_TFLOPS,
             "base_product_kernel": {"us_per_launch": us_base, "achieved": flops_base / us_base / 1e6,
                                     "frac": flops_base / us_base / 1e6 / tc_peak, "launches_timed": n},
-            "launches_per_call": 3, "plan": plan}
+            "launches_per_call": int(plan.split("launches=")[1].split()[0]) if "launches=" in plan else 3, "plan": plan}
 
 
 # --------------------------------------------------------------------------------------------- our arm

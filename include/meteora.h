@@ -325,6 +325,8 @@ int meteora_describe_plan(const meteora_shape_t* shape, char* buf, size_t buf_by
  *                    default 0 = never (measured slower than the streamed kernel except for the largest layers),
  *                    other = wherever the device can hold all clusters at once
  *   "group_pairs"    > 0 = row pairs per scheduling group of the prefill kernel on pairs of SMs (0 = planner's choice)
+ *   "tail_carve"     prefill on pairs of SMs: 0 = the planner carves the tiles of a nearly empty last wave out of the
+ *                    pair launch (they follow as a launch of small tiles), -1 = never, n > 0 = the last token tile of n row pairs
  *   "wait_limit_us"  > 0 = limit of every bounded device-side wait in microseconds (0 = the default of about a second)
  * Unknown names return METEORA_ERR_INVALID_ARG.  The defaults are what the benchmarks measure.
  */

@@ -521,6 +521,7 @@ int meteora_set_tuning(const char* name, int value) {
     else if (!strcmp(name, "pair_decode")) t.pair_decode = value;
     else if (!strcmp(name, "cluster_decode")) t.cluster_decode = value;
     else if (!strcmp(name, "aux_plain")) t.aux_plain = value;
+    else if (!strcmp(name, "tail_carve")) t.tail_carve = value;
     else if (!strcmp(name, "wait_limit_us")) return set_wait_limit_us(value);
     else if (!strcmp(name, "coop")) t.coop = value;
     else if (!strcmp(name, "no_hold")) t.no_hold = value;

@@ -146,6 +146,7 @@ struct Tuning {
     int no_hold = 0;         // decode kernel, head start of the aux CTAs: 0 planner's choice, 1 none, 64 counter wait, other = nanoseconds
     int hold_after = 0;      // decode kernel: ring stages of W0 the main CTAs request before the aux CTAs' head start (0: planner, -1: none)
     int narrow_select = 0;   // decode kernel's selection: 0 by batch size, 1 always two narrow round trips, -1 always one wide one
+    int tail_carve = 0;      // prefill on pairs of SMs: 0 = the planner carves a nearly empty last wave out, -1 = never, n = n row pairs
     int aux_plain = 1;       // streamed kernel: the aux CTAs' partial tiles leave as plain stores (0: staged, one bulk copy)
     int cluster_decode = 0;  // decode batches on clusters that exchange through distributed shared memory (0: never)
     int pdl_decode = 1;      // the decode kernel is launched with programmatic stream serialization as well (0: not)

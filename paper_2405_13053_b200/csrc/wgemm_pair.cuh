@@ -96,6 +96,8 @@ struct PairParams {
     const __nv_bfloat16* B;
     int32_t* status;
     int pdl_wait;
+    int skip_rp0, skip_tt0;       // tiles with row pair >= skip_rp0 AND token tile >= skip_tt0 are another launch's
+    int pdl_trigger;              // that launch follows: let it become resident as this launch's last wave drains
 };
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads)
@@ -130,6 +132,9 @@ k_wgemm_pair(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CU
     const int grp = lin / per_group, rem = lin - grp * per_group;
     const int in_grp = min(p.group_pairs, row_pairs - grp * p.group_pairs);     // the last group may be smaller
     const int tok_tile = rem / in_grp, row_pair = grp * p.group_pairs + rem - tok_tile * in_grp;
+    // The tiles of a last, nearly empty wave are carved out of this launch (a launch of small tiles takes them): both
+    // CTAs of such a pair leave before they touch a barrier or TMEM.
+    if (row_pair >= p.skip_rp0 && tok_tile >= p.skip_tt0) return;
     const int tile_m = row_pair * 2 + (int)rank;                  // own 128 rows of W0 / y
     const int tok0 = tok_tile * kPairTokens;                      // the pair's 256 tokens
     const int tokh = tok0 + (int)rank * kPairHalf;                // own half of them
@@ -157,6 +162,7 @@ k_wgemm_pair(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CU
     cluster_sync();                                               // both CTAs' barriers exist before anyone signals
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+    if (p.pdl_trigger && threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)

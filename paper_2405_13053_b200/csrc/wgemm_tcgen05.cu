@@ -92,6 +92,7 @@ struct WGemmParams {
     int32_t* status;
     int pdl_wait;        // epilogue waits for the preceding grid before reading its results
     int pdl_trigger;     // let the dependent grid start as soon as this one is resident
+    int row_tile0, tok_base;   // the launch covers row tiles from row_tile0 and tokens from tok_base (a rectangle of y)
     int x_alt;           // MODE_STACKED: row tiles >= split_tile multiply the tokens of the FOURTH tensor map over
     int ksteps1;         //   ksteps1 k-steps (two stacked products with different token operands in one launch)
 };
@@ -474,8 +475,8 @@ k_wgemm(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtens
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.splits;
     const int split = (int)cluster_rank();
-    const int tile_m = blockIdx.x / S;
-    const int tok0 = blockIdx.y * p.BN;
+    const int tile_m = p.row_tile0 + blockIdx.x / S;
+    const int tok0 = p.tok_base + blockIdx.y * p.BN;
     const int ntok = min(p.BN, p.T - tok0);
     // contraction range of this CTA: first cut by grid z, then by cluster rank
     const bool second_x = p.x_alt && tile_m >= p.split_tile;
@@ -1258,7 +1259,8 @@ static PairPlan make_pair_plan(const meteora_shape_t& s) {
 }
 
 static int launch_base_lora_pair(const void* x, const void* W0, const void* B, const meteora_shape_t& s,
-                                 const Workspace& ws, void* y, const PairPlan& pp, bool pdl, cudaStream_t st) {
+                                 const Workspace& ws, void* y, const PairPlan& pp, bool pdl, cudaStream_t st,
+                                 int skip_rp0, int skip_tt0) {
     const int row_tiles = (s.d_out + kBM - 1) / kBM;
     CUtensorMap mW, mX, mY;
     int rc;
@@ -1293,6 +1295,9 @@ static int launch_base_lora_pair(const void* x, const void* W0, const void* B, c
     p.B = (const __nv_bfloat16*)B;
     p.status = ws.status;
     p.pdl_wait = pdl ? 1 : 0;
+    p.skip_rp0 = skip_rp0;
+    p.skip_tt0 = skip_tt0;
+    p.pdl_trigger = skip_rp0 != 0x7FFFFFFF && tuning().pdl ? 1 : 0;
     static int smem_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return METEORA_ERR_CUDA;
@@ -1315,12 +1320,21 @@ static int launch_base_lora_pair(const void* x, const void* W0, const void* B, c
     return cuda_status(cudaLaunchKernelEx(&cfg, k_wgemm_pair, mW, mX, mY, p));
 }
 
-int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
-                        void* y, bool pdl, cudaStream_t st) {
-    const PairPlan pp = make_pair_plan(s);
-    if (pp.ok) return launch_base_lora_pair(x, W0, B, s, ws, y, pp, pdl, st);
-    const int row_tiles = (s.d_out + kBM - 1) / kBM;
-    const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
+// Base product + LoRA expand of the rectangle of y [row tiles row_tile0 .. + n_row_tiles) x [tokens tok_base .. + n_tok) on
+// k_wgemm (one CTA, or a cluster along the contraction axis, per tile); bn_force > 0 fixes the tokens per tile.
+static int launch_base_lora_rect(const void* x, const void* W0, const void* B, const meteora_shape_t& s,
+                                 const Workspace& ws, void* y, int row_tile0, int n_row_tiles, int tok_base, int n_tok,
+                                 int bn_force, bool pdl, cudaStream_t st) {
+    const int row_tiles = n_row_tiles;
+    // a carved-out rectangle of small tiles: clusters along the contraction axis until the tiles fill the SMs (a
+    // 128 x 64 tile alone takes in 1.5 MB over 64 k-steps, 23 us on one SM)
+    int splits_force = 0;
+    if (bn_force > 0) {
+        const int tiles = row_tiles * ((n_tok + bn_force - 1) / bn_force);
+        splits_force = 1;
+        while (splits_force < 8 && tiles * splits_force * 2 <= sm_count()) splits_force *= 2;
+    }
+    const Plan pl = make_plan(row_tiles, n_tok, s.d_in, true, s.N, s.r, s.k, false, bn_force, false, 0, splits_force);
     CUtensorMap mW, mX;
     int rc;
     if ((rc = get_tensor_map(W0, s.d_in, s.d_out, kBM, pl.maps3d ? pl.kc : 0, &mW)) != METEORA_OK) return rc;
@@ -1341,6 +1355,8 @@ int launch_base_lora_tc(const void* x, const void* W0, const void* B, const mete
     p.k = s.k;
     p.pdl_wait = pdl ? 1 : 0;
     p.pdl_trigger = 0;
+    p.row_tile0 = row_tile0;
+    p.tok_base = tok_base;
     CUtensorMap mY = mX;
     p.tma_store = 0;
     if (pl.splits == 1 && pl.lora_mma && s.d_out % 8 == 0 && !tuning().no_tma_store) {
@@ -1348,6 +1364,41 @@ int launch_base_lora_tc(const void* x, const void* W0, const void* B, const mete
         p.tma_store = 1;
     }
     return launch_wgemm(mW, mW, mX, mY, p, row_tiles, pl, pdl, st);
+}
+
+// A last wave that is nearly empty costs a whole tile time: 448 pair tiles on 74 pairs of SMs are 6 waves and 4 tiles.
+// Those tiles (the last token tile of the last `rem` row pairs) are carved out of the pair launch and follow as 128 x 64
+// tiles of k_wgemm, which take a fraction of a pair tile's time on a few SMs.  Returns the row pairs to carve.
+static int pair_tail_carve(const meteora_shape_t& s) {
+    const int row_tiles = (s.d_out + kBM - 1) / kBM, row_pairs = (row_tiles + 1) / 2;
+    const int tok_tiles = (s.T + kPairTokens - 1) / kPairTokens;
+    const int resident = std::max(1, sm_count() / 2), tiles = row_pairs * tok_tiles;
+    const int rem = tiles % resident;
+    const int knob = tuning().tail_carve;                        // 0: planner, -1: never, n > 0: carve n row pairs
+    int carve = 0;
+    if (knob >= 0 && tiles > resident && rem > 0 && rem <= row_pairs && 4 * rem <= resident) carve = rem;
+    if (knob > 0) carve = std::min(knob, row_pairs);
+    if (tok_tiles < 2) carve = 0;
+    return carve;
+}
+
+int launch_base_lora_tc(const void* x, const void* W0, const void* B, const meteora_shape_t& s, const Workspace& ws,
+                        void* y, bool pdl, cudaStream_t st) {
+    const PairPlan pp = make_pair_plan(s);
+    if (pp.ok) {
+        const int row_tiles = (s.d_out + kBM - 1) / kBM, row_pairs = (row_tiles + 1) / 2;
+        const int tok_tiles = (s.T + kPairTokens - 1) / kPairTokens;
+        const int carve = pair_tail_carve(s);
+        int rc = launch_base_lora_pair(x, W0, B, s, ws, y, pp, pdl, st, carve > 0 ? row_pairs - carve : 0x7FFFFFFF,
+                                       tok_tiles - 1);
+        if (rc != METEORA_OK || carve == 0) return rc;
+        const int row_tile0 = 2 * (row_pairs - carve), tok_base = (tok_tiles - 1) * kPairTokens;
+        // (launched programmatically dependent: its main loops run on the SMs the pair launch's last wave frees first;
+        // its epilogue waits for the pair launch, and with it for the routing, before it reads the routing)
+        return launch_base_lora_rect(x, W0, B, s, ws, y, row_tile0, row_tiles - row_tile0, tok_base, s.T - tok_base, 64,
+                                     tuning().pdl != 0, st);
+    }
+    return launch_base_lora_rect(x, W0, B, s, ws, y, 0, (s.d_out + kBM - 1) / kBM, 0, s.T, 0, pdl, st);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2145,9 +2196,11 @@ int describe_plan(const meteora_shape_t& s, char* buf, size_t n) {
     const PairPlan pp = make_pair_plan(s);
     if (pp.ok)
         return snprintf(buf, n,
-                        "path=chain(not fused: reason %d) launches=3 base=pairs_of_ctas pairs=%d tile=256x256 stages=%d "
-                        "smem=%zu expand=mma",
-                        fp.why, (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens), pp.stages, pp.smem);
+                        "path=chain(not fused: reason %d) launches=%d base=pairs_of_ctas pairs=%d tile=256x256 stages=%d "
+                        "smem=%zu expand=mma tail_pairs_as_small_tiles=%d",
+                        fp.why, pair_tail_carve(s) > 0 ? 4 : 3,
+                        (row_tiles + 1) / 2 * ((s.T + kPairTokens - 1) / kPairTokens) - pair_tail_carve(s), pp.stages,
+                        pp.smem, pair_tail_carve(s));
     const Plan pl = make_plan(row_tiles, s.T, s.d_in, true, s.N, s.r, s.k);
     return snprintf(buf, n,
                     "path=chain(not fused: reason %d) launches=3 base_ctas=%d cluster=%d tile_tokens=%d stages=%d kc=%d "

@@ -632,6 +632,33 @@ def test_clustered_decode_calls_share_one_workspace_back_to_back(clustered_decod
         assert rel_l2(y.float().cpu().numpy(), ref) <= 1e-2
 
 
+def test_a_nearly_empty_last_wave_of_pair_tiles_runs_as_small_tiles():
+    # 8 row pairs x 10 token tiles = 80 pair tiles on 74 pairs of SMs: the planner carves the 6 tiles of the second
+    # wave (last token tile of the last 6 row pairs) out of the pair launch; a launch of 128 x 64 tiles follows.
+    # Forced to other sizes as well (1 row pair, all 8), with a ragged last token tile and rank 16.
+    for T, r, carve in ((2560, 8, 0), (2500, 8, 1), (2500, 16, 8), (700, 8, 3)):
+        w = workloads.make_workload("carve", T=T, d_in=512, d_out=2048, N=28, k=2, r=r, dtype="bf16", x_kind="normal",
+                                    seed=9100 + T + carve, b_std=0.3)
+        mb.meteora_set_tuning("pair", 2)
+        mb.meteora_set_tuning("tail_carve", carve)
+        try:
+            shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+            plan = mb.meteora_describe_plan(shape)
+            assert "pairs_of_ctas" in plan
+            want = carve if carve else 6
+            assert f"tail_pairs_as_small_tiles={want}" in plan, plan
+            check_forward(w, y_tol=1e-2)
+            y1, i1, _ = run_forward(w)
+            mb.meteora_set_tuning("tail_carve", -1)                      # the same call with every tile on pairs
+            assert "tail_pairs_as_small_tiles=0" in mb.meteora_describe_plan(shape)
+            y0, i0, _ = run_forward(w)
+            np.testing.assert_array_equal(i0, i1)
+            assert rel_l2(y1, y0) < 2e-3
+        finally:
+            mb.meteora_set_tuning("pair", 1)
+            mb.meteora_set_tuning("tail_carve", 0)
+
+
 # Prefill base product on pairs of SMs (256 x 256 tiles): an odd number of row tiles (640 = 5, the last pair has
 # one idle half), a ragged last token tile, a token count that leaves the second half of a pair's tokens empty
 # (257), a contraction length that is no multiple of 64, and adapters up to an odd count.  The stacked shrink of
