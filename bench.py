@@ -39,7 +39,7 @@ NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, nominal
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "fb61f1e632daa184", "bytes_per_launch": {"128": 38597803 + 13397, "1": 37557163 + 85}}
+NCU_TRAFFIC = {"kernel_sha": "6c268f4db48b4a04", "bytes_per_launch": {"128": 38597547 + 13739, "1": 37557248 + 256}}
 
 
 def parse_args():
