@@ -3,7 +3,7 @@
 Every wait of the kernels (mbarrier phases, workspace counters) gives up after a limit, records it in the
 workspace's status word, and the kernel drains and returns.  Here that limit is shortened to a few milliseconds
 (knob wait_limit_us) and one counter of a workspace header is biased on the host so that it cannot reach its
-target: the aux CTAs' "all partials are in" wait then expires.  Nothing waits forever: every waiter in the
+target: the "all partials are in" wait of the CTAs that select then expires.  Nothing waits forever: every waiter in the
 kernels is bounded by the same limit.  The call must return, meteora_workspace_status must report
 METEORA_ERR_TIMEOUT, and after meteora_workspace_init the next call on that workspace must match the oracle.
 """
@@ -19,20 +19,23 @@ from .gpu_util import rel_l2, to_dev
 
 pytestmark = pytest.mark.gpu
 
-COUNTER_WORD = 16          # header word of the "stacked-shrink partials delivered" counter of both decode kernels
+COUNTER_WORD = 16          # header word of the "stacked-shrink partials delivered" counter of all three decode kernels
 
 
-@pytest.mark.parametrize("stream_kernel", [1, 0])
+@pytest.mark.parametrize("stream_kernel", [1, 0, "cluster"])
 def test_an_expired_wait_is_reported_and_the_workspace_recovers(stream_kernel):
     w = workloads.make_workload("bounded", T=40, d_in=1024, d_out=640, dtype="bf16", x_kind="normal", seed=8800,
                                 b_std=0.3)
     x, W0, A, B, Wg = to_dev(w, "x", "W0", "A", "B", "Wg")
     shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
     ws = mb.alloc_workspace(shape)
-    mb.meteora_set_tuning("stream", stream_kernel)
+    cluster = stream_kernel == "cluster"
+    mb.meteora_set_tuning("stream", 1 if cluster else stream_kernel)
+    mb.meteora_set_tuning("cluster_decode", 2 if cluster else 0)
     mb.meteora_set_tuning("wait_limit_us", 3000)
     try:
-        assert ("stream_decode" if stream_kernel else "fused_decode") in mb.meteora_describe_plan(shape)
+        assert ("cluster_decode" if cluster else "stream_decode" if stream_kernel else "fused_decode") in \
+            mb.meteora_describe_plan(shape)
         ws[:4096].view(torch.int32)[COUNTER_WORD] = -1000000         # the counter can no longer reach its target
         torch.cuda.synchronize()
         mb.meteora_linear_forward(x, W0, A, B, Wg, w.k, workspace=ws)
@@ -52,3 +55,4 @@ def test_an_expired_wait_is_reported_and_the_workspace_recovers(stream_kernel):
         np.testing.assert_array_equal(y.float().cpu().numpy(), y2.float().cpu().numpy())
     finally:
         mb.meteora_set_tuning("stream", 1)
+        mb.meteora_set_tuning("cluster_decode", 0)
