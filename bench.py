@@ -39,7 +39,7 @@ NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, nominal
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by tokens; valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernel_sha": "6c268f4db48b4a04", "bytes_per_launch": {"128": 38597547 + 13739, "1": 37557248 + 256}}
+NCU_TRAFFIC = {"kernel_sha": "50d161f11a52512d", "bytes_per_launch": {"128": 38597888 + 16128, "1": 37557333 + 427}}
 
 
 def parse_args():

@@ -1744,7 +1744,7 @@ struct StreamPlan {
 constexpr int kStreamBarSlots = 16;
 constexpr size_t kTwoPerSmBytes = 113 * 1024;    // dynamic shared memory with which two CTAs share an SM
 
-static StreamPlan make_stream_plan(const meteora_shape_t& s) {
+static StreamPlan make_stream_plan_with(const meteora_shape_t& s, int aux_budget_forced) {
     const Tuning& tn = tuning();
     StreamPlan sp = {};
     sp.why = 1;
@@ -1763,6 +1763,7 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     sp.gate_row0 = merged ? tail_rows : 0;
     sp.why = 2;
     int aux_budget = std::max(20, 4 * sp.aux_tiles);
+    if (aux_budget_forced > 0) aux_budget = std::max(aux_budget_forced, sp.aux_tiles);
     if (tn.aux_ctas > 0) aux_budget = std::max(tn.aux_ctas, sp.aux_tiles);
     aux_budget = std::min(aux_budget, sms - 8);
     sp.aux_slices = std::min(std::min(aux_budget / sp.aux_tiles, ksteps), 16);
@@ -1833,6 +1834,9 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     for (int per_sm = 2; per_sm >= 1; --per_sm) {
         if (per_sm == 2 && !want_two) continue;
         const size_t budget = per_sm == 2 ? kTwoPerSmBytes : 226 * 1024;
+        // all CTAs wait for one another through the workspace: they must all be resident (a forced split can ask for
+        // more CTAs than one per SM holds)
+        if (sp.n_main + sp.n_aux > per_sm * sms) continue;
         const size_t fixed = 1024 + sp.slab_off + slab_bytes;
         if (fixed + ring_need > budget || fixed + 2 * stage_bytes > budget) continue;
         const size_t avail = budget - fixed;
@@ -1861,6 +1865,16 @@ static StreamPlan make_stream_plan(const meteora_shape_t& s) {
     sp.pf_aux = cap > 0 ? std::max(0, nks_aux - sp.aux_stages) : 0;
     sp.why = 0;
     sp.ok = true;
+    return sp;
+}
+
+// Large ranks (64 at N = 28): with the usual four aux CTAs per stacked tile the main CTAs are few, each has many output
+// rows, and the B rows of all adapters for them do not fit beside the ring.  One aux CTA per stacked tile leaves more
+// main CTAs with fewer rows each (measured at 4096 -> 4096, 32 tokens, rank 64: 34.4 us against 41.6 on the three-launch
+// chain; an expand that reads the picked adapters' rows from L2 instead of staging them took 68 - 78 us).
+static StreamPlan make_stream_plan(const meteora_shape_t& s) {
+    StreamPlan sp = make_stream_plan_with(s, 0);
+    if (!sp.ok && sp.why == 5 && tuning().aux_ctas == 0) sp = make_stream_plan_with(s, 20);
     return sp;
 }
 

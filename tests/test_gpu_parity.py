@@ -474,6 +474,19 @@ def test_streamed_decode_kernel_adapter_counts(N, k, T, r):
     check_forward(w, y_tol=1e-2)
 
 
+def test_streamed_decode_kernel_rank_64_takes_one_aux_cta_per_stacked_tile():
+    # 28 adapters of rank 64: 15 tiles of stacked rows.  With four aux CTAs per tile only two main CTAs per row tile
+    # remain and the B rows of all adapters for a CTA's 64 output rows (229 KB) do not fit; the planner falls back
+    # to one aux CTA per stacked tile, four main CTAs per row tile and 114 KB of staged rows.
+    for T in (32, 1, 64):                                            # (at 128 tokens the landing area no longer fits either)
+        w = workloads.make_workload("stream_r64", T=T, d_in=512, d_out=4096, N=28, k=2, r=64, dtype="bf16",
+                                    x_kind="normal", seed=2700 + T, b_std=0.3)
+        shape = mb.make_shape(w.T, w.d_in, w.d_out, w.N, w.r, w.k, torch.bfloat16)
+        plan = mb.meteora_describe_plan(shape)
+        assert "stream_decode" in plan and "aux_ctas=15 " in plan and "ctas_per_tile=4 " in plan, plan
+        check_forward(w, y_tol=1e-2)
+
+
 # Its planner's choices forced the other way: a shallow ring, two k-steps per stage, no L2 prefetch, a small prefetch
 # cap, one CTA per SM with a deep ring, few and many aux CTAs, no programmatic dependent launch.  None of them may
 # change the result beyond the order of the fp32 sums of the stacked shrink's slices.  (pair_decode = 1 runs the 70
