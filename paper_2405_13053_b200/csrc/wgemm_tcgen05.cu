@@ -1829,7 +1829,10 @@ static StreamPlan make_stream_plan_with(const meteora_shape_t& s, int aux_budget
     // 5120 -> 13824 (142 MB) 36.5 / 31.8 at 1.  So: two per SM for 16 - 56 MB of W0 and up to 32 tokens, else one.
     // (Knob stream: 2 or 4 always one per SM, 3 always two where they fit.)
     const size_t w0_bytes = (size_t)s.d_out * s.d_in * 2;
-    const bool want_two = tn.stream == 3 || (tn.stream == 1 && s.T <= 32 && w0_bytes >= ((size_t)16 << 20) &&
+    // (later, at 4096 -> 4096: 12.9 / 13.3 at 48 tokens, 13.4 / 13.5 at 64, 14.4 / 14.3 at 80; at 5120 -> 5120 16.8 / 16.6 at 48
+    // and 18.6 / 16.8 at 64: up to 64 tokens for the layers up to 40 MB.)
+    const int two_tokens = w0_bytes <= ((size_t)40 << 20) ? 64 : 32;
+    const bool want_two = tn.stream == 3 || (tn.stream == 1 && s.T <= two_tokens && w0_bytes >= ((size_t)16 << 20) &&
                                              w0_bytes <= ((size_t)56 << 20));
     for (int per_sm = 2; per_sm >= 1; --per_sm) {
         if (per_sm == 2 && !want_two) continue;

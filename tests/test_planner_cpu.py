@@ -20,7 +20,7 @@ def no_gpu_planning_only():
         pytest.skip("the planner asks the device for its SM count; these pins are for the 148-SM default")
 
 
-@pytest.mark.parametrize("T,per_sm", [(1, 2), (8, 2), (32, 2), (64, 1), (128, 1)])
+@pytest.mark.parametrize("T,per_sm", [(1, 2), (8, 2), (32, 2), (64, 2), (80, 1), (128, 1)])
 def test_decode_batches_of_the_headline_shape_take_the_streamed_kernel(T, per_sm):
     p = plan(T, 4096, 4096)
     assert "path=stream_decode launches=1 main_ctas=128 row_tiles=32 ctas_per_tile=4 aux_ctas=20 aux_slices=10" in p
@@ -31,7 +31,8 @@ def test_wide_layers_stream_with_one_cta_per_row_tile_and_one_per_sm():
     p = plan(1, 4096, 14336)
     assert "path=stream_decode" in p and "row_tiles=112 ctas_per_tile=1 " in p and "ctas_per_sm=1 " in p, p
     p = plan(64, 5120, 5120)
-    assert "path=stream_decode" in p and "row_tiles=40 ctas_per_tile=3 " in p, p
+    assert "path=stream_decode" in p and "row_tiles=40 ctas_per_tile=3 " in p and "ctas_per_sm=1 " in p, p
+    assert "ctas_per_sm=2 " in plan(32, 5120, 5120)
 
 
 def test_batches_above_128_tokens_leave_the_streamed_kernel():
